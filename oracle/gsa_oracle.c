@@ -1,0 +1,252 @@
+/*
+ * CPU oracle for the forward path of Gated Sparse Attention.
+ *
+ * TEST INFRASTRUCTURE ONLY.  Plain loops, fp64 arithmetic, no blocking, no fusion.
+ * It shares no code with the CUDA library and must never be called from the product
+ * path: only the tests, the smoke check and the benchmark's CPU-baseline leg use it.
+ *
+ * Inputs arrive as fp32 arrays holding exactly the bf16 / fp32 values the GPU reads
+ * (widening is exact); every sum, exponential and division below is done in double.
+ *
+ * Steps, in the paper's order:
+ *   Eq. 7   gated lightning indexer     I[t,s] = sum_j w[t,j] * sigmoid(q^I[t,j] . k^I[s] + b_j)
+ *   Eq. 8   adaptive budget             k_t = clamp(floor(k_base * Var(I[t,:]) / Vbar), k_min, k_max)
+ *   Eq. 4   top-k_t selection           S_t = the k_t positions with the largest I[t,s]
+ *   Eq. 9   value gate G2               V'[s] = V[s] * sigmoid(g2[s])      (elementwise)
+ *   Eq. 11  softmax over S_t            A[t,s] = exp(Q_t.K_s/sqrt(d_k)) / sum_{j in S_t} exp(...)
+ *   Eq. 12  aggregation                 O[t] = sum_{s in S_t} A[t,s] V'[s]
+ *   Eq. 10  output gate G1              out[t,h] = O[t,h] * sigmoid(g1[t,h]) (elementwise)
+ *
+ * Readings where the paper is silent (each is also listed in the design notes):
+ *   - query t of Lq sees keys s = 0 .. Lk-Lq+t (causal; decode is Lq = 1);
+ *   - Var is the population variance over the visible scores only;
+ *   - k_eff = min(k_t, number of visible keys);
+ *   - ties in I are broken towards the lower position; S_t is emitted ascending;
+ *   - one S_t per query position, shared by all heads (I has no head index);
+ *   - k_mode 0 is Eq. 8 as printed; k_mode 1 is the direction the prose describes
+ *     (k_base * Vbar / Var; Var = 0 gives k_max); k_mode 2 is a fixed k = k_base.
+ *
+ * Pins (tests/test_oracle_pins.py): closed-form sigmoid values on one-hot inputs,
+ * the reflection identity I(q)+I(-q)=sum_j w_j, the open range (0, sum w), two-valued
+ * rows with known variance, clamp edges, monotonicity per mode, brute-force top-k
+ * with exact ties, reduction to library softmax attention when S_t is everything
+ * and gates are saturated, single-key and equal-logit closed forms, g1 = -40 -> 0.
+ * Parity unpinned: nothing (every function above has at least one such pin); the
+ * absolute values on random data have no printed reference in the paper.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+typedef struct {
+    int32_t B, Lq, Lk;
+    int32_t n_h, n_kv, d_h;
+    int32_t HI, dI;
+    int32_t k_base, k_min, k_max;
+    int32_t k_mode;
+    double v_bar;
+    double sm_scale; /* <= 0: 1/sqrt(d_h) */
+} gsa_oracle_params;
+
+static double sigmoid_d(double x) { return 1.0 / (1.0 + exp(-x)); }
+
+int gsa_oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* number of keys query t may look at */
+int gsa_oracle_visible(const gsa_oracle_params *p, int t) { return p->Lk - p->Lq + t + 1; }
+
+/* ---- Eq. 7 -------------------------------------------------------------- */
+/* qI_t: [HI, dI] of this query; kI_b: [Lk, dI] of this batch element; w_t: [HI]. */
+void gsa_oracle_score_row(const gsa_oracle_params *p, const float *qI_t, const float *kI_b,
+                          const float *w_t, const float *bI, int n_t, double *I_row)
+{
+    for (int s = 0; s < n_t; ++s) {
+        double acc = 0.0;
+        for (int j = 0; j < p->HI; ++j) {
+            double x = bI ? (double)bI[j] : 0.0;
+            for (int c = 0; c < p->dI; ++c)
+                x += (double)qI_t[j * p->dI + c] * (double)kI_b[(size_t)s * p->dI + c];
+            acc += (double)w_t[j] * sigmoid_d(x);
+        }
+        I_row[s] = acc;
+    }
+}
+
+/* ---- Eq. 8 -------------------------------------------------------------- */
+void gsa_oracle_budget(const gsa_oracle_params *p, const double *I_row, int n_t,
+                       double *var_out, double *r_out, int32_t *k_t_out, int32_t *k_eff_out)
+{
+    double mean = 0.0;
+    for (int s = 0; s < n_t; ++s) mean += I_row[s];
+    mean /= (double)n_t;
+    double var = 0.0;
+    for (int s = 0; s < n_t; ++s) var += (I_row[s] - mean) * (I_row[s] - mean);
+    var /= (double)n_t;
+
+    double r;
+    if (p->k_mode == 0)      r = (double)p->k_base * var / p->v_bar;
+    else if (p->k_mode == 1) r = var > 0.0 ? (double)p->k_base * p->v_bar / var : INFINITY;
+    else                     r = (double)p->k_base;
+
+    double f = floor(r);
+    int32_t k;
+    if (!(f < (double)p->k_max)) k = p->k_max;          /* also catches +inf */
+    else if (f < (double)p->k_min) k = p->k_min;
+    else k = (int32_t)f;
+    if (var_out) *var_out = var;
+    if (r_out) *r_out = r;
+    *k_t_out = k;
+    *k_eff_out = k < n_t ? k : n_t;
+}
+
+/* ---- Eq. 4 -------------------------------------------------------------- */
+typedef struct { double score; int32_t pos; } scored_t;
+
+static int by_score_desc_pos_asc(const void *a, const void *b)
+{
+    const scored_t *x = (const scored_t *)a, *y = (const scored_t *)b;
+    if (x->score > y->score) return -1;
+    if (x->score < y->score) return 1;
+    return (x->pos > y->pos) - (x->pos < y->pos);
+}
+static int by_int_asc(const void *a, const void *b)
+{
+    int32_t x = *(const int32_t *)a, y = *(const int32_t *)b;
+    return (x > y) - (x < y);
+}
+
+/* full sort of the row; the first k_eff entries are S_t; written ascending, rest -1 */
+void gsa_oracle_topk(const double *I_row, int n_t, int k_eff, int32_t *idx_out, int k_pad)
+{
+    scored_t *a = (scored_t *)malloc(sizeof(scored_t) * (size_t)n_t);
+    for (int s = 0; s < n_t; ++s) { a[s].score = I_row[s]; a[s].pos = s; }
+    qsort(a, (size_t)n_t, sizeof(scored_t), by_score_desc_pos_asc);
+    for (int i = 0; i < k_eff; ++i) idx_out[i] = a[i].pos;
+    qsort(idx_out, (size_t)k_eff, sizeof(int32_t), by_int_asc);
+    for (int i = k_eff; i < k_pad; ++i) idx_out[i] = -1;
+    free(a);
+}
+
+/* ---- Eq. 9, 11, 12, 10 --------------------------------------------------- */
+/* Q_t, g1_t: [n_h, d_h]; K_b, V_b, g2_b: [Lk, n_kv, d_h]; idx: k_eff positions. */
+void gsa_oracle_attn_row(const gsa_oracle_params *p, const float *Q_t, const float *K_b,
+                         const float *V_b, const float *g1_t, const float *g2_b,
+                         const int32_t *idx, int k_eff, double *out_t)
+{
+    const int d = p->d_h, grp = p->n_h / p->n_kv;
+    const double scale = p->sm_scale > 0.0 ? p->sm_scale : 1.0 / sqrt((double)d);
+    double *z = (double *)malloc(sizeof(double) * (size_t)(k_eff > 0 ? k_eff : 1));
+    for (int h = 0; h < p->n_h; ++h) {
+        const int g = h / grp;
+        double zmax = -INFINITY;
+        for (int i = 0; i < k_eff; ++i) {
+            const float *Ks = K_b + ((size_t)idx[i] * p->n_kv + g) * d;
+            double dot = 0.0;
+            for (int c = 0; c < d; ++c) dot += (double)Q_t[h * d + c] * (double)Ks[c];
+            z[i] = dot * scale;
+            if (z[i] > zmax) zmax = z[i];
+        }
+        double den = 0.0;
+        for (int i = 0; i < k_eff; ++i) { z[i] = exp(z[i] - zmax); den += z[i]; }
+        for (int c = 0; c < d; ++c) {
+            double o = 0.0;
+            for (int i = 0; i < k_eff; ++i) {
+                const size_t at = ((size_t)idx[i] * p->n_kv + g) * d + c;
+                const double vg = (double)V_b[at] * sigmoid_d((double)g2_b[at]);   /* Eq. 9 */
+                o += (z[i] / den) * vg;                                             /* Eq. 11-12 */
+            }
+            out_t[h * d + c] = o * sigmoid_d((double)g1_t[h * d + c]);            /* Eq. 10 */
+        }
+    }
+    free(z);
+}
+
+/* ---- drivers over a list of (batch, query) rows -------------------------- */
+
+/* scores of the listed rows: out[r, 0..n_t) in a [n_rows, Lk] double array */
+void gsa_oracle_scores_rows(const gsa_oracle_params *p, const float *qI, const float *kI,
+                            const float *w, const float *bI, const int32_t *rows_b,
+                            const int32_t *rows_t, int n_rows, double *scores_out)
+{
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int r = 0; r < n_rows; ++r) {
+        const int b = rows_b[r], t = rows_t[r];
+        const int n_t = gsa_oracle_visible(p, t);
+        gsa_oracle_score_row(p, qI + ((size_t)b * p->Lq + t) * p->HI * p->dI,
+                             kI + (size_t)b * p->Lk * p->dI, w + ((size_t)b * p->Lq + t) * p->HI,
+                             bI, n_t, scores_out + (size_t)r * p->Lk);
+    }
+}
+
+/* Eq. 8 + Eq. 4 on externally supplied fp32 score rows ("staged" mode): row r of
+ * `scores` (stride in floats) belongs to query rows_t[r]. */
+void gsa_oracle_select_rows_f32(const gsa_oracle_params *p, const float *scores, int64_t stride,
+                                const int32_t *rows_t, int n_rows, int32_t *idx_out,
+                                int32_t *kt_out, int32_t *keff_out, double *var_out,
+                                double *r_out)
+{
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int r = 0; r < n_rows; ++r) {
+        const int n_t = gsa_oracle_visible(p, rows_t[r]);
+        double *row = (double *)malloc(sizeof(double) * (size_t)n_t);
+        for (int s = 0; s < n_t; ++s) row[s] = (double)scores[(size_t)r * stride + s];
+        gsa_oracle_budget(p, row, n_t, var_out + r, r_out + r, kt_out + r, keff_out + r);
+        gsa_oracle_topk(row, n_t, keff_out[r], idx_out + (size_t)r * p->k_max, p->k_max);
+        free(row);
+    }
+}
+
+/* Eq. 9-12, 10 for the listed rows with given index sets (idx: [n_rows, k_max]) */
+void gsa_oracle_attn_rows(const gsa_oracle_params *p, const float *Q, const float *K,
+                          const float *V, const float *g1, const float *g2,
+                          const int32_t *rows_b, const int32_t *rows_t, int n_rows,
+                          const int32_t *idx, const int32_t *keff, double *out)
+{
+    const size_t qrow = (size_t)p->n_h * p->d_h, kvb = (size_t)p->Lk * p->n_kv * p->d_h;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int r = 0; r < n_rows; ++r) {
+        const int b = rows_b[r], t = rows_t[r];
+        gsa_oracle_attn_row(p, Q + ((size_t)b * p->Lq + t) * qrow, K + b * kvb, V + b * kvb,
+                            g1 + ((size_t)b * p->Lq + t) * qrow, g2 + b * kvb,
+                            idx + (size_t)r * p->k_max, keff[r], out + (size_t)r * qrow);
+    }
+}
+
+/* the whole path, end to end, for the listed rows.  scores_out may be NULL. */
+void gsa_oracle_forward_rows(const gsa_oracle_params *p, const float *Q, const float *K,
+                             const float *V, const float *qI, const float *kI, const float *w,
+                             const float *bI, const float *g1, const float *g2,
+                             const int32_t *rows_b, const int32_t *rows_t, int n_rows,
+                             double *out, int32_t *idx_out, int32_t *kt_out, int32_t *keff_out,
+                             double *var_out, double *r_out, double *scores_out)
+{
+    const size_t qrow = (size_t)p->n_h * p->d_h, kvb = (size_t)p->Lk * p->n_kv * p->d_h;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int r = 0; r < n_rows; ++r) {
+        const int b = rows_b[r], t = rows_t[r];
+        const int n_t = gsa_oracle_visible(p, t);
+        double *row = scores_out ? scores_out + (size_t)r * p->Lk
+                                 : (double *)malloc(sizeof(double) * (size_t)n_t);
+        gsa_oracle_score_row(p, qI + ((size_t)b * p->Lq + t) * p->HI * p->dI,
+                             kI + (size_t)b * p->Lk * p->dI, w + ((size_t)b * p->Lq + t) * p->HI,
+                             bI, n_t, row);
+        gsa_oracle_budget(p, row, n_t, var_out + r, r_out + r, kt_out + r, keff_out + r);
+        int32_t *idx = idx_out + (size_t)r * p->k_max;
+        gsa_oracle_topk(row, n_t, keff_out[r], idx, p->k_max);
+        gsa_oracle_attn_row(p, Q + ((size_t)b * p->Lq + t) * qrow, K + b * kvb, V + b * kvb,
+                            g1 + ((size_t)b * p->Lq + t) * qrow, g2 + b * kvb, idx, keff_out[r],
+                            out + (size_t)r * qrow);
+        if (!scores_out) free(row);
+    }
+}

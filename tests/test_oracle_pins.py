@@ -1,0 +1,359 @@
+"""Pins for the CPU oracle: checks against what the paper and the mathematics fix,
+none of which re-type the oracle's own formulas with the oracle's own routine.
+
+  Eq. 7   closed-form sigmoid values on one-hot inputs; the reflection identity;
+          the open range (0, sum_j w_j) which lies inside the paper's (0, H^I)
+  Eq. 8   rows with a known variance (two-valued rows), clamp edges, direction
+  Eq. 4   brute force on tiny rows with exact ties
+  Eq. 9-12, 10   reduction to library softmax attention, single-key / equal-logit
+          closed forms, the "do nothing" pathway of the output gate
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import OracleParams
+from paper_2601_15305_b200.inputs import CONFIGS, make_inputs
+
+LN3 = math.log(3.0)
+
+
+def small_params(**kw):
+    base = dict(B=1, Lq=6, Lk=6, n_h=4, n_kv=2, d_h=8, HI=3, dI=4, k_base=4, k_min=1, k_max=6,
+                k_mode=0, v_bar=1.0)
+    base.update(kw)
+    return OracleParams(**base)
+
+
+# ----------------------------------------------------------------------------- Eq. 7
+def test_indexer_closed_form_one_hot():
+    """q^I one-hot on component c with amplitude a picks a * k^I[s, c]; logits chosen as
+    0, +ln3, -ln3 give sigmoid 1/2, 3/4, 1/4 exactly.  Every index (t, j, c, s) is distinct,
+    so a transposed or shifted operand changes the expected value."""
+    p = small_params(Lq=3, Lk=3, HI=3, dI=4)
+    qI = np.zeros((1, 3, 3, 4), np.float32)
+    kI = np.zeros((1, 3, 4), np.float32)
+    w = np.array([[[0.5, 0.25, 0.125], [1.0, 0.5, 0.25], [0.75, 0.5, 0.0625]]], np.float32)
+    # query t=2: head 0 looks at component 1, head 1 at component 3, head 2 at component 0
+    qI[0, 2, 0, 1] = 2.0
+    qI[0, 2, 1, 3] = -1.0
+    qI[0, 2, 2, 0] = 4.0
+    # key s=1: components chosen so the three logits are ln3, -ln3, 0
+    kI[0, 1] = [0.0, LN3 / 2.0, 7.0, LN3]
+    # key s=0: logits 0, 0, ln3 ;  key s=2: logits -ln3, ln3, -ln3
+    kI[0, 0] = [LN3 / 4.0, 0.0, -3.0, 0.0]
+    kI[0, 2] = [-LN3 / 4.0, -LN3 / 2.0, 1.0, -LN3]
+    sc = oracle.scores(p, qI, kI, w, None, rows_t=[2])
+    w2 = w[0, 2].astype(np.float64)
+    # kI is stored in fp32, so ln3 carries fp32 rounding: tolerance 1e-7
+    exp_s1 = w2[0] * 0.75 + w2[1] * 0.25 + w2[2] * 0.5
+    exp_s0 = w2[0] * 0.5 + w2[1] * 0.5 + w2[2] * 0.75
+    exp_s2 = w2[0] * 0.25 + w2[1] * 0.75 + w2[2] * 0.25
+    np.testing.assert_allclose(sc[0, :3], [exp_s0, exp_s1, exp_s2], rtol=0, atol=2e-7)
+    # rows t=0,1 have zero queries: every visible score is sum_j w_j / 2; the rest stays NaN
+    sc01 = oracle.scores(p, qI, kI, w, None, rows_t=[0, 1])
+    np.testing.assert_allclose(sc01[0, :1], w[0, 0].sum() / 2, atol=1e-15)
+    np.testing.assert_allclose(sc01[1, :2], w[0, 1].sum() / 2, atol=1e-15)
+    assert np.isnan(sc01[0, 1:]).all() and np.isnan(sc01[1, 2:]).all()
+
+
+def test_indexer_bias_shifts_logit():
+    """b_j enters inside the sigmoid: zero query, bias (ln3, -ln3) gives w0*3/4 + w1/4."""
+    p = small_params(Lq=1, Lk=1, HI=2, dI=4)
+    qI = np.zeros((1, 1, 2, 4), np.float32)
+    kI = np.ones((1, 1, 4), np.float32)
+    w = np.array([[[0.5, 0.25]]], np.float32)
+    b = np.array([LN3, -LN3], np.float32)
+    sc = oracle.scores(p, qI, kI, w, b, rows_t=[0])
+    assert abs(sc[0, 0] - (0.5 * 0.75 + 0.25 * 0.25)) < 1e-7
+
+
+def test_indexer_reflection_and_range():
+    """sigmoid(x) + sigmoid(-x) = 1  =>  I(q) + I(-q) = sum_j w_j for b = 0;
+    every score lies strictly inside (0, sum_j w_j) which is inside (0, H^I)."""
+    cfg = CONFIGS["tiny"]
+    x = make_inputs(cfg)
+    p = OracleParams.from_config(cfg)
+    rows = [0, 1, 17, 255, 511]
+    a = oracle.scores(p, x["qI"], x["kI"], x["w"], None, rows)
+    b = oracle.scores(p, -x["qI"].float(), x["kI"], x["w"], None, rows)
+    wsum = x["w"][0, rows].double().sum(-1).numpy()
+    for i, t in enumerate(rows):
+        n = t + 1
+        np.testing.assert_allclose(a[i, :n] + b[i, :n], wsum[i], rtol=0, atol=1e-14)
+        assert (a[i, :n] > 0).all() and (a[i, :n] < wsum[i]).all() and wsum[i] < cfg.HI
+        assert np.isnan(a[i, n:]).all()
+
+
+def test_indexer_matches_library_matmul():
+    """The contraction inside the sigmoid is an ordinary matrix product: compare with
+    torch's fp64 einsum + library sigmoid on random data (an independent routine)."""
+    cfg = CONFIGS["tiny"]
+    x = make_inputs(cfg)
+    p = OracleParams.from_config(cfg)
+    rows = [5, 100, 511]
+    a = oracle.scores(p, x["qI"], x["kI"], x["w"], None, rows)
+    q = x["qI"][0, rows].double()
+    logits = torch.einsum("tjc,sc->tjs", q, x["kI"][0].double())
+    ref = (x["w"][0, rows].double()[:, :, None] * torch.sigmoid(logits)).sum(1).numpy()
+    for i, t in enumerate(rows):
+        np.testing.assert_allclose(a[i, : t + 1], ref[i, : t + 1], rtol=1e-13, atol=0)
+
+
+def test_decode_sees_whole_cache():
+    """Lq = 1 over Lk keys: the single query sees all Lk keys."""
+    p = small_params(Lq=1, Lk=5, HI=1, dI=1)
+    sc = oracle.scores(p, np.zeros((1, 1, 1, 1), np.float32), np.ones((1, 5, 1), np.float32),
+                       np.full((1, 1, 1), 0.5, np.float32), None, rows_t=[0])
+    np.testing.assert_allclose(sc[0], 0.25, atol=1e-15)
+
+
+# ----------------------------------------------------------------------------- Eq. 8
+def _select(p, row, t):
+    return oracle.select_f32(p, np.asarray(row, np.float32)[None, :], [t])
+
+
+def test_budget_two_valued_row():
+    """A row with n1 entries at a and n0 at b has population variance p(1-p)(a-b)^2."""
+    n, n1, a, b = 64, 16, 1.5, 0.5           # p = 1/4: Var = 3/16
+    row = np.full(n, b, np.float32)
+    row[:n1] = a
+    for k_base, v_bar, want in [(160, 1.0, 30), (100, 0.5, 37), (7, 3.0 / 16.0, 7)]:
+        p = small_params(Lq=n, Lk=n, k_base=k_base, k_min=2, k_max=60, v_bar=v_bar)
+        r = _select(p, row, n - 1)
+        assert abs(r["var"][0] - 3.0 / 16.0) < 1e-15
+        assert r["kt"][0] == want, (k_base, v_bar, r["kt"][0])
+    # sample variance (n-1) would give 160*0.1905 = 30.47 -> still 30; use a case that splits them
+    p = small_params(Lq=n, Lk=n, k_base=336, k_min=2, k_max=64, v_bar=1.0)   # 336*3/16 = 63 exactly
+    assert _select(p, row, n - 1)["kt"][0] == 63                               # 336*0.190476 = 64 if /(n-1)
+
+
+def test_budget_clamps_and_constant_row():
+    n = 40
+    p = small_params(Lq=n, Lk=n, k_base=16, k_min=5, k_max=12, v_bar=1.0)
+    const = np.full(n, 0.7, np.float32)
+    r = _select(p, const, n - 1)
+    assert r["var"][0] == 0.0 and r["kt"][0] == 5            # Var 0 -> floor(0) -> k_min
+    wide = np.zeros(n, np.float32)
+    wide[::2] = 4.0                                          # Var = 4 -> 64 -> k_max
+    assert _select(p, wide, n - 1)["kt"][0] == 12
+    # fewer visible keys than k_t: everything visible is selected
+    r = _select(p, wide[:3].tolist() + [0.0] * (n - 3), 2)
+    assert r["kt"][0] in (5, 12) and r["keff"][0] == 3
+    assert r["idx"][0, :3].tolist() == [0, 1, 2] and (r["idx"][0, 3:] == -1).all()
+
+
+def test_budget_uses_visible_scores_only():
+    """Entries past the causal limit are not part of the statistic."""
+    n = 32
+    p = small_params(Lq=n, Lk=n, k_base=64, k_min=1, k_max=32, v_bar=1.0)
+    row = np.full(n, 1.0, np.float32)
+    row[20:] = 100.0                       # garbage beyond t = 19
+    r = _select(p, row, 19)
+    assert r["var"][0] == 0.0 and r["kt"][0] == 1
+
+
+def test_budget_direction_per_mode():
+    """Eq. 8 as printed grows k_t with the row's variance (mode 0); the prose describes
+    the opposite (mode 1); mode 2 ignores the variance."""
+    n = 256
+    rng = np.random.default_rng(0)
+    base = rng.standard_normal(n).astype(np.float32) * 0.05 + 2.0
+    ks = {0: [], 1: [], 2: []}
+    for spread in (0.5, 1.0, 2.0, 4.0):
+        row = (2.0 + (base - 2.0) * spread).astype(np.float32)
+        for mode in ks:
+            p = small_params(Lq=n, Lk=n, k_base=64, k_min=4, k_max=200, v_bar=0.05 ** 2 * 1.0, k_mode=mode)
+            ks[mode].append(int(_select(p, row, n - 1)["kt"][0]))
+    assert ks[0] == sorted(ks[0]) and ks[0][0] < ks[0][-1]
+    assert ks[1] == sorted(ks[1], reverse=True) and ks[1][0] > ks[1][-1]
+    assert ks[2] == [64] * 4
+    # factor 2 in spread = factor 4 in variance = factor 4 in the unclamped budget
+    assert abs(ks[0][1] / ks[0][0] - 4.0) < 0.3 and ks[0][3] == 200
+    # mode 1 with zero variance saturates at k_max
+    p = small_params(Lq=8, Lk=8, k_base=4, k_min=1, k_max=6, v_bar=1.0, k_mode=1)
+    assert _select(p, np.ones(8, np.float32), 7)["kt"][0] == 6
+
+
+# ----------------------------------------------------------------------------- Eq. 4
+def test_topk_bruteforce_with_ties():
+    rng = np.random.default_rng(1)
+    for trial in range(40):
+        n = int(rng.integers(1, 60))
+        # few distinct values -> many exact ties
+        row = rng.integers(0, 5, size=n).astype(np.float32) * 0.25 + 0.25
+        k = int(rng.integers(1, n + 1))
+        p = small_params(Lq=n, Lk=n, k_mode=2, k_base=k, k_min=1, k_max=max(k, 1))
+        r = _select(p, row, n - 1)
+        order = sorted(range(n), key=lambda s: (-float(row[s]), s))     # python's own sort
+        want = sorted(order[:k])
+        assert r["keff"][0] == k
+        assert r["idx"][0, :k].tolist() == want
+        assert (r["idx"][0, k:] == -1).all()
+
+
+def test_topk_nested_and_threshold_property():
+    """top-k sets are nested in k, and every selected score >= every rejected score."""
+    cfg = CONFIGS["tiny"]
+    x = make_inputs(cfg)
+    p0 = OracleParams.from_config(cfg)
+    sc = oracle.scores(p0, x["qI"], x["kI"], x["w"], None, [511]).astype(np.float32)
+    prev = set()
+    for k in (1, 2, 17, 64, 300, 512):
+        p = OracleParams.from_config(cfg, k_mode=2, k_base=k, k_min=1, k_max=512)
+        r = oracle.select_f32(p, sc, [511])
+        cur = set(r["idx"][0, :k].tolist())
+        assert len(cur) == k and prev <= cur
+        rest = sorted(set(range(512)) - cur)
+        if rest:
+            assert sc[0, sorted(cur)].min() >= sc[0, rest].max()
+        prev = cur
+
+
+def test_planted_needle_is_selected():
+    """A key built as 0.8*q^I[t, j*] + noise, with a large head weight, scores among the best."""
+    cfg = CONFIGS["tiny"]
+    x = make_inputs(cfg)
+    x["w"][0, 400, :] = 0.05
+    x["w"][0, 400, 2] = 0.95
+    x["kI"][0, 123] = (4.0 * x["qI"][0, 400, 2].float()).to(torch.bfloat16)
+    p = OracleParams.from_config(cfg)
+    r = oracle.forward(p, **x, rows_t=[400])
+    assert 123 in r["idx"][0, : r["keff"][0]].tolist()
+
+
+# ----------------------------------------------------------------------------- Eq. 9-12, 10
+def _textbook_attention(Q, K, V, scale):
+    """softmax(Q K^T * scale) V with torch's library softmax / matmul in fp64 (Eq. 2)."""
+    return torch.softmax((Q @ K.transpose(-1, -2)) * scale, dim=-1) @ V
+
+
+def _rand_attn_inputs(p, seed=0):
+    g = torch.Generator().manual_seed(seed)
+    r = lambda *s: torch.randn(*s, generator=g).to(torch.bfloat16)
+    return dict(Q=r(p.B, p.Lq, p.n_h, p.d_h), K=r(p.B, p.Lk, p.n_kv, p.d_h), V=r(p.B, p.Lk, p.n_kv, p.d_h),
+                g1=r(p.B, p.Lq, p.n_h, p.d_h), g2=r(p.B, p.Lk, p.n_kv, p.d_h))
+
+
+def test_attn_saturated_gates_reduce_to_textbook_sdpa():
+    """Logit +40 makes sigmoid exactly 1.0 in double; with S_t = all visible keys the
+    layer is plain causal GQA attention (Eq. 2)."""
+    p = small_params(B=2, Lq=7, Lk=7, n_h=4, n_kv=2, d_h=8, k_max=7)
+    x = _rand_attn_inputs(p, 3)
+    x["g1"] = torch.full_like(x["g1"], 40.0)
+    x["g2"] = torch.full_like(x["g2"], 40.0)
+    for b in range(p.B):
+        for t in (0, 3, 6):
+            idx = np.full((1, p.k_max), -1, np.int32)
+            idx[0, : t + 1] = np.arange(t + 1)
+            got = oracle.attn(p, **x, idx=idx, keff=[t + 1], rows_t=[t], rows_b=[b])[0]
+            for h in range(p.n_h):
+                g = h // (p.n_h // p.n_kv)
+                ref = _textbook_attention(x["Q"][b, t, h].double()[None], x["K"][b, : t + 1, g].double(),
+                                          x["V"][b, : t + 1, g].double(), 1.0 / math.sqrt(p.d_h))[0]
+                np.testing.assert_allclose(got[h], ref.numpy(), rtol=1e-12, atol=1e-14)
+
+
+def test_attn_subset_equals_library_attention_on_gathered_rows():
+    """Sparse attention over S_t is dense gated attention on the gathered rows (Eq. 5, 9-12)."""
+    p = small_params(B=1, Lq=12, Lk=12, n_h=4, n_kv=2, d_h=8, k_max=6)
+    x = _rand_attn_inputs(p, 4)
+    t = 11
+    sel = [0, 3, 4, 9, 11]
+    idx = np.full((1, p.k_max), -1, np.int32)
+    idx[0, : len(sel)] = sel
+    got = oracle.attn(p, **x, idx=idx, keff=[len(sel)], rows_t=[t])[0]
+    Vg = x["V"][0].double() * torch.sigmoid(x["g2"][0].double())
+    for h in range(p.n_h):
+        g = h // 2
+        ref = _textbook_attention(x["Q"][0, t, h].double()[None], x["K"][0, sel, g].double(), Vg[sel, g],
+                                  1.0 / math.sqrt(p.d_h))[0] * torch.sigmoid(x["g1"][0, t, h].double())
+        np.testing.assert_allclose(got[h], ref.numpy(), rtol=1e-12, atol=1e-14)
+    # custom softmax scale is honoured
+    p2 = small_params(B=1, Lq=12, Lk=12, n_h=4, n_kv=2, d_h=8, k_max=6, sm_scale=0.3)
+    got2 = oracle.attn(p2, **x, idx=idx, keff=[len(sel)], rows_t=[t])[0]
+    ref2 = _textbook_attention(x["Q"][0, t, 1].double()[None], x["K"][0, sel, 0].double(), Vg[sel, 0], 0.3)[0] \
+        * torch.sigmoid(x["g1"][0, t, 1].double())
+    np.testing.assert_allclose(got2[1], ref2.numpy(), rtol=1e-12, atol=1e-14)
+
+
+def test_attn_single_key_and_equal_logits_closed_forms():
+    p = small_params(B=1, Lq=4, Lk=4, n_h=2, n_kv=1, d_h=4, k_max=4)
+    x = _rand_attn_inputs(p, 5)
+    # one selected key: softmax is 1, output = V[s]*sigmoid(g2[s]) * sigmoid(g1[t])
+    x["g2"][0, 2] = torch.tensor([0.0, LN3, -LN3, 40.0]).to(torch.bfloat16)
+    x["g1"][0, 3, 0] = torch.tensor([LN3, 0.0, 40.0, -LN3]).to(torch.bfloat16)
+    idx = np.array([[2, -1, -1, -1]], np.int32)
+    got = oracle.attn(p, **x, idx=idx, keff=[1], rows_t=[3])[0]
+    s = lambda v: 1.0 / (1.0 + math.exp(-float(v)))
+    v = x["V"][0, 2, 0].double().numpy()
+    want = v * [s(u) for u in x["g2"][0, 2, 0]] * np.array([s(u) for u in x["g1"][0, 3, 0]])
+    np.testing.assert_allclose(got[0], want, rtol=1e-14)
+    # equal keys => equal logits => plain average of the gated values
+    x["K"][0, 1] = x["K"][0, 0]
+    idx = np.array([[0, 1, -1, -1]], np.int32)
+    x["g1"][:] = 40.0
+    x["g2"][:] = 40.0
+    got = oracle.attn(p, **x, idx=idx, keff=[2], rows_t=[3])[0]
+    np.testing.assert_allclose(got[1], (x["V"][0, 0, 0].double() + x["V"][0, 1, 0].double()).numpy() / 2, rtol=1e-14)
+
+
+def test_output_gate_do_nothing_pathway():
+    """g1 = -40 suppresses the output whatever the attention distribution is."""
+    p = small_params(B=1, Lq=5, Lk=5, n_h=4, n_kv=2, d_h=8, k_max=5)
+    x = _rand_attn_inputs(p, 6)
+    x["g1"][:] = -40.0
+    idx = np.array([[0, 1, 2, 3, 4]], np.int32)
+    got = oracle.attn(p, **x, idx=idx, keff=[5], rows_t=[4])
+    assert np.abs(got).max() < 1e-15
+
+
+def test_forward_large_budget_is_dense_gated_attention():
+    """k_min >= L: S_t is every visible key and the whole layer is dense gated attention."""
+    cfg = CONFIGS["tiny"].with_(Lq=96, Lk=96, k_base=96, k_min=96, k_max=96)
+    x = make_inputs(cfg)
+    p = OracleParams.from_config(cfg)
+    rows = [0, 1, 50, 95]
+    r = oracle.forward(p, **x, rows_t=rows)
+    Vg = x["V"][0].double() * torch.sigmoid(x["g2"][0].double())
+    for i, t in enumerate(rows):
+        assert r["keff"][i] == t + 1 and r["idx"][i, : t + 1].tolist() == list(range(t + 1))
+        for h in range(cfg.n_h):
+            ref = _textbook_attention(x["Q"][0, t, h].double()[None], x["K"][0, : t + 1, 0].double(),
+                                      Vg[: t + 1, 0], 1.0 / math.sqrt(cfg.d_h))[0] \
+                * torch.sigmoid(x["g1"][0, t, h].double())
+            np.testing.assert_allclose(r["out"][i, h], ref.numpy(), rtol=1e-12, atol=1e-15)
+
+
+def test_forward_is_composition_of_stages():
+    cfg = CONFIGS["tiny"]
+    x = make_inputs(cfg)
+    p = OracleParams.from_config(cfg)
+    rows = [0, 15, 16, 127, 128, 300, 511]
+    r = oracle.forward(p, **x, rows_t=rows, want_scores=True)
+    assert r["kt"].min() >= cfg.k_min and r["kt"].max() <= cfg.k_max
+    assert len(set(r["kt"].tolist())) > 2                     # the budget really adapts
+    out2 = oracle.attn(p, x["Q"], x["K"], x["V"], x["g1"], x["g2"], r["idx"], r["keff"], rows)
+    np.testing.assert_array_equal(out2, r["out"])
+    for i, t in enumerate(rows):
+        assert r["keff"][i] == min(r["kt"][i], t + 1)
+        want_k = min(max(math.floor(cfg.k_base * np.var(r["scores"][i, : t + 1]) / cfg.v_bar), cfg.k_min), cfg.k_max)
+        assert r["kt"][i] == want_k
+
+
+# ----------------------------------------------------------------------------- printed numbers
+def test_paper_printed_cost_model():
+    """Appendix A prints d^I H^I/(d n_h) ~ 0.002 and a 12.8x speed-up for its parameters."""
+    vals = {}
+    with open(__file__.rsplit("/", 1)[0] + "/golden/paper_cost_model.txt") as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                k, v = line.split("=")
+                vals[k.strip()] = float(v.split("#")[0])
+    ratio = vals["dI"] * vals["HI"] / (vals["d"] * vals["n_h"])
+    assert abs(ratio - vals["printed_ratio"]) < 5e-4
+    sp = (vals["d"] / (vals["dI"] * vals["HI"])) / (1.0 + vals["k"] * vals["d"] / (vals["L"] * vals["dI"] * vals["HI"]))
+    assert abs(sp - vals["printed_speedup"]) < 0.1
