@@ -1,0 +1,171 @@
+/*
+ * gsa.h -- C ABI of the B200 (sm_100a) forward path of Gated Sparse Attention.
+ *
+ * Three stages and their fusion, named after the paper's notation:
+ *   gsa_indexer_scores         gated lightning indexer                     (Eq. 7)
+ *   gsa_adaptive_topk          adaptive budget k_t and top-k_t selection   (Eq. 8, Eq. 4)
+ *   gsa_sparse_gated_attn_fwd  value gate G2, sparse softmax attention over
+ *                              S_t, output gate G1                         (Eq. 9, 11, 12, 10)
+ *   gsa_forward                all of the above for a whole batch          (Sec. 3.2, Eq. 6 pipeline)
+ *
+ * Conventions common to every call
+ *   - Every data pointer is DEVICE memory owned by the caller, 16-byte aligned and
+ *     contiguous in the stated layout, unless the argument says "host".
+ *   - The library allocates no memory, keeps no state between calls and never
+ *     synchronises the device (except gsa_forward_host and gsa_device_status, which
+ *     wait for `stream`).  Work is enqueued on `stream` (a cudaStream_t passed as
+ *     void*; NULL is the legacy default stream).
+ *   - Return value: GSA_OK or a negative gsa_status.  Argument errors are detected on
+ *     the host before anything is launched.  Conditions only the device can see
+ *     (a bounded wait that ran out inside a tensor-core pipeline) are recorded in a
+ *     status word at the start of the workspace; read it with gsa_device_status.
+ *   - bf16 tensors are passed as void*; fp32 accumulation everywhere; outputs are
+ *     rounded to bf16 once (round to nearest even).
+ *   - Query t (0-based, of Lq) may look at keys s = 0 .. Lk-Lq+t ("visible keys",
+ *     n_t = Lk-Lq+t+1).  Prefill is Lq == Lk; decode is Lq == 1 over an Lk-token cache.
+ *
+ * Supported shapes: d_h in {64, 128}; dI in {32, 64}; HI in {1, 2, 4, 8};
+ * n_h / n_kv in {1, 2, 4, 8}; k_max <= 4096; 1 <= Lq <= Lk < 2^24.
+ */
+#ifndef GSA_H_
+#define GSA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    GSA_OK = 0,
+    GSA_ERR_INVALID_ARG = -1,      /* NULL / misaligned pointer, inconsistent sizes          */
+    GSA_ERR_UNSUPPORTED_SHAPE = -2,/* a shape outside the list above                         */
+    GSA_ERR_WORKSPACE = -3,        /* workspace missing or smaller than gsa_workspace_bytes  */
+    GSA_ERR_CUDA = -4,             /* a CUDA runtime / driver call failed                    */
+    GSA_ERR_DEVICE_TIMEOUT = -5    /* a bounded device-side wait expired (see device status) */
+} gsa_status;
+
+/* Hyper-parameters (Table 1 of the paper) plus the call's geometry. */
+typedef struct gsa_params {
+    int32_t B;          /* batch                                                             */
+    int32_t Lq, Lk;     /* query positions, key positions per batch element                  */
+    int32_t n_h;        /* query heads                                                       */
+    int32_t n_kv;       /* key/value heads; head h uses KV head h / (n_h / n_kv)             */
+    int32_t d_h;        /* head dimension d_k                                                */
+    int32_t HI;         /* indexer heads H^I                                                 */
+    int32_t dI;         /* indexer dimension d^I                                             */
+    int32_t k_base;     /* base selection budget                                             */
+    int32_t k_min;      /* budget bounds, 1 <= k_min <= k_max                                */
+    int32_t k_max;
+    int32_t k_mode;     /* 0: Eq. 8 as printed, k ~ Var/Vbar.  1: the direction the paper's
+                           prose describes, k ~ Vbar/Var (Var = 0 gives k_max).
+                           2: fixed k = k_base                                               */
+    float v_bar;        /* Vbar of Eq. 8: caller-owned running mean of score variance, > 0   */
+    float sm_scale;     /* softmax scale of Eq. 11; <= 0 means 1/sqrt(d_h)                   */
+    int32_t q_begin;    /* per-stage calls process query rows q_begin <= t < q_end of every  */
+    int32_t q_end;      /* batch element; q_end <= 0 means Lq.  gsa_forward ignores both.    */
+} gsa_params_t;
+
+/*
+ * Bytes of device workspace gsa_forward (and the per-stage calls) need for `p`.
+ * `slab_rows` is the number of query rows whose fp32 score rows gsa_forward keeps
+ * resident at a time (0 = library default, chosen so the slab stays near the L2 size).
+ * Host call; writes *bytes.
+ */
+int gsa_workspace_bytes(const gsa_params_t *p, int32_t slab_rows, size_t *bytes);
+
+/*
+ * Gated lightning indexer, Eq. 7:
+ *     I[t,s] = sum_j w[t,j] * sigmoid(qI[t,j,:] . kI[s,:] + bI[j]),   s visible to t.
+ *   qI     [B, Lq, HI, dI] bf16        kI  [B, Lk, dI] bf16 (one key shared by all heads)
+ *   w      [B, Lq, HI]     fp32, the already-activated head weights sigmoid(h_t W^Iw_j)
+ *   bI     [HI] fp32 or NULL (= zeros)
+ *   scores fp32; the row of (b, t) starts at scores[((b * R) + (t - q_begin)) * row_stride]
+ *          with R = q_end - q_begin and row_stride >= Lk, a multiple of 4.  Entries beyond
+ *          the row's visible keys are left unwritten.
+ *   ws     workspace (device status word lives at its start); ws_bytes >= 256.
+ */
+int gsa_indexer_scores(const gsa_params_t *p, const void *qI, const void *kI, const float *w,
+                       const float *bI, float *scores, int64_t row_stride, void *ws,
+                       size_t ws_bytes, void *stream);
+
+/*
+ * Adaptive sparsity controller, Eq. 8 then Eq. 4, one row at a time:
+ *     Var_t = population variance of the n_t visible scores (accumulated in fp64),
+ *     k_t   = clamp(floor(k_base * Var_t / v_bar), k_min, k_max)   (k_mode 0),
+ *     S_t   = the min(k_t, n_t) positions with the largest scores; equal scores are
+ *             ordered by position, lower first.
+ *   scores as written by gsa_indexer_scores (same q_begin / q_end / row_stride)
+ *   idx    [B, R, k_max] int32: S_t in ascending position order, then -1
+ *   kt     [B, R] int32: |S_t| = min(k_t, n_t)
+ *   var    [B, R] fp32 or NULL: Var_t (for the caller's running mean)
+ */
+int gsa_adaptive_topk(const gsa_params_t *p, const float *scores, int64_t row_stride,
+                      int32_t *idx, int32_t *kt, float *var, void *ws, size_t ws_bytes,
+                      void *stream);
+
+/*
+ * Sparse gated attention, Eq. 9, 11, 12, 10, for query rows q_begin..q_end:
+ *     V'[s]   = V[s] * sigmoid(g2[s])                       (elementwise, G2)
+ *     A[t,s]  = softmax over s in S_t of  sm_scale * Q[t,h,:] . K[s,g(h),:]
+ *     out[t,h,:] = (sum_s A[t,s] V'[s,g(h),:]) * sigmoid(g1[t,h,:])   (G1)
+ *   Q, g1_logits [B, Lq, n_h, d_h] bf16;  K, V, g2_logits [B, Lk, n_kv, d_h] bf16
+ *   g2_logits may be NULL: V is then taken as already gated.
+ *   idx [B, R, k_max], kt [B, R] as written by gsa_adaptive_topk (R = q_end - q_begin)
+ *   out [B, Lq, n_h, d_h] bf16 (rows outside q_begin..q_end untouched)
+ */
+int gsa_sparse_gated_attn_fwd(const gsa_params_t *p, const void *Q, const void *K, const void *V,
+                              const void *g1_logits, const void *g2_logits, const int32_t *idx,
+                              const int32_t *kt, void *out, void *ws, size_t ws_bytes,
+                              void *stream);
+
+/*
+ * The whole forward path (pipeline of Sec. 3.2): G2, indexer, budget, top-k, sparse
+ * attention, G1, for all B * Lq queries.  Score rows are produced and consumed slab by
+ * slab inside the workspace and never leave it.
+ *   idx_out [B, Lq, k_max] int32 or NULL;  kt_out [B, Lq] int32 or NULL;
+ *   var_out [B, Lq] fp32 or NULL.
+ *   slab_rows as in gsa_workspace_bytes (must be the value the workspace was sized with).
+ */
+int gsa_forward(const gsa_params_t *p, const void *Q, const void *K, const void *V,
+                const void *qI, const void *kI, const float *w, const float *bI,
+                const void *g1_logits, const void *g2_logits, void *out, int32_t *idx_out,
+                int32_t *kt_out, float *var_out, int32_t slab_rows, void *ws, size_t ws_bytes,
+                void *stream);
+
+/*
+ * gsa_forward on HOST buffers (pinned memory recommended): copies the nine inputs to a
+ * caller-provided device arena, runs gsa_forward there, copies `out` (and kt_out if
+ * not NULL) back and waits for `stream`.  All tensor pointers are host pointers.
+ * `arena` is device memory of at least gsa_forward_host_arena_bytes(p, slab_rows).
+ */
+int gsa_forward_host_arena_bytes(const gsa_params_t *p, int32_t slab_rows, size_t *bytes);
+int gsa_forward_host(const gsa_params_t *p, const void *Q, const void *K, const void *V,
+                     const void *qI, const void *kI, const float *w, const float *bI,
+                     const void *g1_logits, const void *g2_logits, void *out, int32_t *kt_out,
+                     int32_t slab_rows, void *arena, size_t arena_bytes, void *stream);
+
+/*
+ * Waits for `stream`, reads the device status word at the start of `ws` into
+ * *status_out (host) and returns GSA_OK / GSA_ERR_DEVICE_TIMEOUT accordingly.
+ * The word is cleared by every call that takes `ws`.
+ */
+int gsa_device_status(const void *ws, void *stream, int32_t *status_out);
+
+/* Number of kernel launches the library has enqueued so far in this process (host counter). */
+int64_t gsa_launch_count(void);
+
+/*
+ * Debug knob: 0 = tensor-core (tcgen05) indexer where the shape allows it (default),
+ * 1 = plain CUDA-core indexer.  Process-wide; not meant for production use.
+ */
+void gsa_debug_set_indexer_path(int32_t path);
+
+/* Static string for a gsa_status value. */
+const char *gsa_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GSA_H_ */

@@ -1,0 +1,319 @@
+// C ABI of the library (declared in include/gsa.h): argument checks, workspace plan,
+// the slab loop of gsa_forward, and the host-buffer variant.
+#include <math.h>
+#include <stdio.h>
+
+#include "gsa_common.cuh"
+
+namespace gsa {
+
+int64_t g_launches = 0;
+static int32_t g_indexer_path = 0;
+
+cudaError_t launch_indexer_simple(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* qI,
+                                  const __nv_bfloat16* kI, const float* w, const float* bI,
+                                  float* scores, int64_t row_stride, cudaStream_t st);
+bool indexer_tc_supported(const gsa_params_t& p);
+cudaError_t launch_indexer_tc(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* qI,
+                              const __nv_bfloat16* kI, const float* w, const float* bI,
+                              float* scores, int64_t row_stride, int32_t* dev_status,
+                              cudaStream_t st);
+
+cudaError_t launch_indexer(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* qI,
+                           const __nv_bfloat16* kI, const float* w, const float* bI, float* scores,
+                           int64_t row_stride, int32_t* dev_status, cudaStream_t st) {
+    if (g_indexer_path == 0 && indexer_tc_supported(p))
+        return launch_indexer_tc(p, rr, qI, kI, w, bI, scores, row_stride, dev_status, st);
+    return launch_indexer_simple(p, rr, qI, kI, w, bI, scores, row_stride, st);
+}
+
+namespace {
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool one_of(int v, std::initializer_list<int> l) {
+    for (int x : l) if (x == v) return true;
+    return false;
+}
+
+int check_params(const gsa_params_t* p) {
+    if (!p) return GSA_ERR_INVALID_ARG;
+    if (p->B < 1 || p->Lq < 1 || p->Lk < p->Lq || p->n_h < 1 || p->n_kv < 1) return GSA_ERR_INVALID_ARG;
+    if (p->n_h % p->n_kv != 0) return GSA_ERR_INVALID_ARG;
+    if (p->k_min < 1 || p->k_min > p->k_max || p->k_base < 1) return GSA_ERR_INVALID_ARG;
+    if (p->k_mode < 0 || p->k_mode > 2) return GSA_ERR_INVALID_ARG;
+    if (p->k_mode != 2 && !(p->v_bar > 0.f)) return GSA_ERR_INVALID_ARG;
+    if (!one_of(p->d_h, {64, 128}) || !one_of(p->dI, {32, 64}) || !one_of(p->HI, {1, 2, 4, 8}))
+        return GSA_ERR_UNSUPPORTED_SHAPE;
+    if (!one_of(p->n_h / p->n_kv, {1, 2, 4, 8}) || !one_of(p->n_kv, {1, 2, 4, 8}))
+        return GSA_ERR_UNSUPPORTED_SHAPE;
+    if (p->k_max > 4096 || p->Lk >= (1 << 24)) return GSA_ERR_UNSUPPORTED_SHAPE;
+    if ((int64_t)p->B * p->Lq >= (1ll << 31)) return GSA_ERR_UNSUPPORTED_SHAPE;
+    return GSA_OK;
+}
+
+int row_range(const gsa_params_t* p, RowRange* rr) {
+    const int qe = p->q_end <= 0 ? p->Lq : p->q_end;
+    if (p->q_begin < 0 || p->q_begin >= qe || qe > p->Lq) return GSA_ERR_INVALID_ARG;
+    rr->b0 = 0; rr->nb = p->B; rr->q_begin = p->q_begin; rr->R = qe - p->q_begin;
+    return GSA_OK;
+}
+
+struct WsPlan {
+    int64_t row_stride;
+    int32_t slab_rows;
+    bool prepass;                  // Eq. 9 as a pre-pass (prefill) or inside the gather (decode)
+    size_t slab_off, vg_off, idx_off, kt_off, total;
+};
+
+WsPlan plan_ws(const gsa_params_t& p, int32_t slab_rows) {
+    WsPlan w;
+    w.row_stride = (int64_t)align_up((size_t)p.Lk, 32);
+    const int64_t rows_total = (int64_t)p.B * p.Lq;
+    if (slab_rows <= 0) {
+        const int64_t target = 64ll << 20;
+        int64_t r = target / (w.row_stride * 4);
+        r = r / 32 * 32;
+        slab_rows = (int32_t)(r < 32 ? 32 : r);
+    }
+    if (slab_rows > rows_total) slab_rows = (int32_t)rows_total;
+    w.slab_rows = slab_rows;
+    // gating the whole V once costs 3 passes over it; gating inside the gather costs one more
+    // gathered row per selected key.
+    w.prepass = (int64_t)p.Lq * p.k_base > 3ll * p.Lk;
+    size_t off = kStatusBytes;
+    w.slab_off = off; off += align_up((size_t)slab_rows * w.row_stride * 4, 256);
+    w.vg_off = off;   off += w.prepass ? align_up((size_t)p.B * p.Lk * p.n_kv * p.d_h * 2, 256) : 0;
+    w.idx_off = off;  off += align_up((size_t)rows_total * p.k_max * 4, 256);
+    w.kt_off = off;   off += align_up((size_t)rows_total * 4, 256);
+    w.total = off;
+    return w;
+}
+
+int cuda_rc(cudaError_t e) {
+    if (e == cudaSuccess) return GSA_OK;
+    fprintf(stderr, "gsa: CUDA error: %s\n", cudaGetErrorString(e));
+    return GSA_ERR_CUDA;
+}
+
+}  // namespace
+}  // namespace gsa
+
+using namespace gsa;
+typedef __nv_bfloat16 bf16;
+
+extern "C" {
+
+int gsa_workspace_bytes(const gsa_params_t* p, int32_t slab_rows, size_t* bytes) {
+    int rc = check_params(p);
+    if (rc) return rc;
+    if (!bytes || slab_rows < 0) return GSA_ERR_INVALID_ARG;
+    *bytes = plan_ws(*p, slab_rows).total;
+    return GSA_OK;
+}
+
+int gsa_indexer_scores(const gsa_params_t* p, const void* qI, const void* kI, const float* w,
+                       const float* bI, float* scores, int64_t row_stride, void* ws,
+                       size_t ws_bytes, void* stream) {
+    int rc = check_params(p);
+    if (rc) return rc;
+    RowRange rr;
+    if ((rc = row_range(p, &rr))) return rc;
+    if (!qI || !kI || !w || !scores || !aligned16(qI) || !aligned16(kI) || !aligned16(w) || !aligned16(scores))
+        return GSA_ERR_INVALID_ARG;
+    if (row_stride < p->Lk || row_stride % 4 != 0) return GSA_ERR_INVALID_ARG;
+    if (!ws || ws_bytes < (size_t)kStatusBytes || !aligned16(ws)) return GSA_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, st);
+    if (e != cudaSuccess) return cuda_rc(e);
+    return cuda_rc(launch_indexer(*p, rr, (const bf16*)qI, (const bf16*)kI, w, bI, scores, row_stride,
+                                  (int32_t*)ws, st));
+}
+
+int gsa_adaptive_topk(const gsa_params_t* p, const float* scores, int64_t row_stride, int32_t* idx,
+                      int32_t* kt, float* var, void* ws, size_t ws_bytes, void* stream) {
+    int rc = check_params(p);
+    if (rc) return rc;
+    RowRange rr;
+    if ((rc = row_range(p, &rr))) return rc;
+    if (!scores || !idx || !kt || !aligned16(scores) || !aligned16(idx)) return GSA_ERR_INVALID_ARG;
+    if (row_stride < p->Lk || row_stride % 4 != 0) return GSA_ERR_INVALID_ARG;
+    (void)ws; (void)ws_bytes;
+    IdxLayout il{0, rr.q_begin, rr.R};
+    return cuda_rc(launch_select(*p, rr, scores, row_stride, idx, kt, var, il, (cudaStream_t)stream));
+}
+
+int gsa_sparse_gated_attn_fwd(const gsa_params_t* p, const void* Q, const void* K, const void* V,
+                              const void* g1_logits, const void* g2_logits, const int32_t* idx,
+                              const int32_t* kt, void* out, void* ws, size_t ws_bytes, void* stream) {
+    int rc = check_params(p);
+    if (rc) return rc;
+    RowRange rr;
+    if ((rc = row_range(p, &rr))) return rc;
+    if (!Q || !K || !V || !g1_logits || !idx || !kt || !out) return GSA_ERR_INVALID_ARG;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(g1_logits) || !aligned16(out) ||
+        !aligned16(idx) || (g2_logits && !aligned16(g2_logits)))
+        return GSA_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    IdxLayout il{0, rr.q_begin, rr.R};
+    const bf16* Vuse = (const bf16*)V;
+    const bf16* g2use = (const bf16*)g2_logits;
+    if (g2_logits) {
+        const WsPlan wp = plan_ws(*p, 0);
+        // pre-pass when it pays and the caller gave room for V'; otherwise gate inside the gather
+        const size_t vg_bytes = (size_t)p->B * p->Lk * p->n_kv * p->d_h * 2;
+        if (wp.prepass && ws && aligned16(ws) && ws_bytes >= (size_t)kStatusBytes + vg_bytes) {
+            bf16* Vg = (bf16*)((char*)ws + kStatusBytes);
+            cudaError_t e = launch_value_gate((const bf16*)V, (const bf16*)g2_logits, Vg,
+                                              (int64_t)p->B * p->Lk * p->n_kv * p->d_h, st);
+            if (e != cudaSuccess) return cuda_rc(e);
+            Vuse = Vg;
+            g2use = nullptr;
+        }
+    }
+    return cuda_rc(launch_sparse_attn(*p, rr, (const bf16*)Q, (const bf16*)K, Vuse, (const bf16*)g1_logits,
+                                      g2use, idx, kt, il, (bf16*)out, st));
+}
+
+int gsa_forward(const gsa_params_t* p, const void* Q, const void* K, const void* V, const void* qI,
+                const void* kI, const float* w, const float* bI, const void* g1_logits,
+                const void* g2_logits, void* out, int32_t* idx_out, int32_t* kt_out, float* var_out,
+                int32_t slab_rows, void* ws, size_t ws_bytes, void* stream) {
+    int rc = check_params(p);
+    if (rc) return rc;
+    if (!Q || !K || !V || !qI || !kI || !w || !g1_logits || !out || slab_rows < 0) return GSA_ERR_INVALID_ARG;
+    const void* ptrs[] = {Q, K, V, qI, kI, w, g1_logits, g2_logits, out, idx_out, kt_out, var_out};
+    for (const void* q : ptrs) if (q && !aligned16(q)) return GSA_ERR_INVALID_ARG;
+    const WsPlan wp = plan_ws(*p, slab_rows);
+    if (!ws || !aligned16(ws) || ws_bytes < wp.total) return GSA_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    char* wsb = (char*)ws;
+    cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, st);
+    if (e != cudaSuccess) return cuda_rc(e);
+
+    float* slab = (float*)(wsb + wp.slab_off);
+    int32_t* idx = idx_out ? idx_out : (int32_t*)(wsb + wp.idx_off);
+    int32_t* kt = kt_out ? kt_out : (int32_t*)(wsb + wp.kt_off);
+    const IdxLayout il{0, 0, p->Lq};
+
+    // Eq. 9: value gate (independent of the indexer)
+    const bf16* Vuse = (const bf16*)V;
+    const bf16* g2use = (const bf16*)g2_logits;
+    if (g2_logits && wp.prepass) {
+        bf16* Vg = (bf16*)(wsb + wp.vg_off);
+        e = launch_value_gate((const bf16*)V, (const bf16*)g2_logits, Vg,
+                              (int64_t)p->B * p->Lk * p->n_kv * p->d_h, st);
+        if (e != cudaSuccess) return cuda_rc(e);
+        Vuse = Vg;
+        g2use = nullptr;
+    }
+
+    // Eq. 7, 8, 4 slab by slab: score rows live only inside the workspace
+    if (wp.slab_rows >= p->Lq) {
+        const int nb_per = wp.slab_rows / p->Lq;
+        for (int b0 = 0; b0 < p->B; b0 += nb_per) {
+            RowRange rr{b0, (p->B - b0 < nb_per ? p->B - b0 : nb_per), 0, p->Lq};
+            if ((e = launch_indexer(*p, rr, (const bf16*)qI, (const bf16*)kI, w, bI, slab, wp.row_stride,
+                                    (int32_t*)ws, st)) != cudaSuccess) return cuda_rc(e);
+            if ((e = launch_select(*p, rr, slab, wp.row_stride, idx, kt, var_out, il, st)) != cudaSuccess)
+                return cuda_rc(e);
+        }
+    } else {
+        for (int b = 0; b < p->B; ++b)
+            for (int q0 = 0; q0 < p->Lq; q0 += wp.slab_rows) {
+                RowRange rr{b, 1, q0, (p->Lq - q0 < wp.slab_rows ? p->Lq - q0 : wp.slab_rows)};
+                if ((e = launch_indexer(*p, rr, (const bf16*)qI, (const bf16*)kI, w, bI, slab, wp.row_stride,
+                                        (int32_t*)ws, st)) != cudaSuccess) return cuda_rc(e);
+                if ((e = launch_select(*p, rr, slab, wp.row_stride, idx, kt, var_out, il, st)) != cudaSuccess)
+                    return cuda_rc(e);
+            }
+    }
+
+    // Eq. 11, 12, 10 over all rows
+    RowRange all{0, p->B, 0, p->Lq};
+    return cuda_rc(launch_sparse_attn(*p, all, (const bf16*)Q, (const bf16*)K, Vuse, (const bf16*)g1_logits,
+                                      g2use, idx, kt, il, (bf16*)out, st));
+}
+
+int gsa_forward_host_arena_bytes(const gsa_params_t* p, int32_t slab_rows, size_t* bytes) {
+    int rc = check_params(p);
+    if (rc) return rc;
+    if (!bytes || slab_rows < 0) return GSA_ERR_INVALID_ARG;
+    const size_t q = (size_t)p->B * p->Lq * p->n_h * p->d_h * 2, kv = (size_t)p->B * p->Lk * p->n_kv * p->d_h * 2;
+    size_t t = 0;
+    t += 3 * align_up(q, 256);                                   // Q, g1, out
+    t += 3 * align_up(kv, 256);                                  // K, V, g2
+    t += align_up((size_t)p->B * p->Lq * p->HI * p->dI * 2, 256);  // qI
+    t += align_up((size_t)p->B * p->Lk * p->dI * 2, 256);          // kI
+    t += align_up((size_t)p->B * p->Lq * p->HI * 4, 256);          // w
+    t += 256;                                                    // bI
+    t += align_up((size_t)p->B * p->Lq * 4, 256);                  // kt
+    t += plan_ws(*p, slab_rows).total;
+    *bytes = t;
+    return GSA_OK;
+}
+
+int gsa_forward_host(const gsa_params_t* p, const void* Q, const void* K, const void* V, const void* qI,
+                     const void* kI, const float* w, const float* bI, const void* g1_logits,
+                     const void* g2_logits, void* out, int32_t* kt_out, int32_t slab_rows, void* arena,
+                     size_t arena_bytes, void* stream) {
+    size_t need = 0;
+    int rc = gsa_forward_host_arena_bytes(p, slab_rows, &need);
+    if (rc) return rc;
+    if (!Q || !K || !V || !qI || !kI || !w || !g1_logits || !out) return GSA_ERR_INVALID_ARG;
+    if (!arena || !aligned16(arena) || arena_bytes < need) return GSA_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t q = (size_t)p->B * p->Lq * p->n_h * p->d_h * 2, kv = (size_t)p->B * p->Lk * p->n_kv * p->d_h * 2;
+    const size_t qi = (size_t)p->B * p->Lq * p->HI * p->dI * 2, ki = (size_t)p->B * p->Lk * p->dI * 2;
+    const size_t wb = (size_t)p->B * p->Lq * p->HI * 4, ktb = (size_t)p->B * p->Lq * 4;
+    char* a = (char*)arena;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { char* r = a + off; off += align_up(bytes, 256); return r; };
+    char *dQ = take(q), *dG1 = take(q), *dOut = take(q), *dK = take(kv), *dV = take(kv), *dG2 = take(kv);
+    char *dqI = take(qi), *dkI = take(ki), *dw = take(wb), *dbI = take(256), *dkt = take(ktb);
+    char* dws = a + off;
+    cudaError_t e;
+#define GSA_H2D(dst, src, n) if ((e = cudaMemcpyAsync(dst, src, n, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_rc(e)
+    GSA_H2D(dQ, Q, q); GSA_H2D(dK, K, kv); GSA_H2D(dV, V, kv); GSA_H2D(dqI, qI, qi); GSA_H2D(dkI, kI, ki);
+    GSA_H2D(dw, w, wb); GSA_H2D(dG1, g1_logits, q);
+    if (g2_logits) GSA_H2D(dG2, g2_logits, kv);
+    if (bI) GSA_H2D(dbI, bI, (size_t)p->HI * 4);
+#undef GSA_H2D
+    rc = gsa_forward(p, dQ, dK, dV, dqI, dkI, (const float*)dw, bI ? (const float*)dbI : nullptr, dG1,
+                     g2_logits ? dG2 : nullptr, dOut, nullptr, (int32_t*)dkt, nullptr, slab_rows, dws,
+                     arena_bytes - off, st);
+    if (rc) return rc;
+    if ((e = cudaMemcpyAsync(out, dOut, q, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_rc(e);
+    if (kt_out && (e = cudaMemcpyAsync(kt_out, dkt, ktb, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_rc(e);
+    if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_rc(e);
+    int32_t dev = 0;
+    return gsa_device_status(dws, stream, &dev);
+}
+
+int gsa_device_status(const void* ws, void* stream, int32_t* status_out) {
+    if (!ws) return GSA_ERR_WORKSPACE;
+    int32_t v = 0;
+    cudaError_t e = cudaMemcpyAsync(&v, ws, sizeof(v), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_rc(e);
+    if (status_out) *status_out = v;
+    return v == kDevOk ? GSA_OK : GSA_ERR_DEVICE_TIMEOUT;
+}
+
+int64_t gsa_launch_count(void) { return g_launches; }
+
+void gsa_debug_set_indexer_path(int32_t path) { g_indexer_path = path; }
+
+const char* gsa_status_string(int s) {
+    switch (s) {
+        case GSA_OK: return "ok";
+        case GSA_ERR_INVALID_ARG: return "invalid argument";
+        case GSA_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+        case GSA_ERR_WORKSPACE: return "workspace missing or too small";
+        case GSA_ERR_CUDA: return "CUDA error";
+        case GSA_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

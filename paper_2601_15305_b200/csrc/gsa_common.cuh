@@ -1,0 +1,100 @@
+// Shared declarations of the sm_100a GSA kernels: argument structs, small device helpers.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "gsa.h"
+
+namespace gsa {
+
+// A contiguous block of work: batch elements b0 .. b0+nb-1, query rows q_begin .. q_begin+R-1
+// of each.  Local row index lr = (b - b0) * R + (t - q_begin).
+struct RowRange {
+    int32_t b0, nb, q_begin, R;
+    __host__ __device__ int32_t rows() const { return nb * R; }
+};
+
+// Where the index sets of a RowRange live: row (b, t) starts at
+// idx + ((b - b_origin) * batch_rows + (t - t_origin)) * k_max, kt likewise without k_max.
+struct IdxLayout {
+    int32_t b_origin, t_origin, batch_rows;
+    __host__ __device__ int64_t row(int32_t b, int32_t t) const {
+        return (int64_t)(b - b_origin) * batch_rows + (t - t_origin);
+    }
+};
+
+constexpr int kStatusBytes = 256;   // head of every workspace: device status word + padding
+
+// device status word values
+enum : int32_t { kDevOk = 0, kDevTimeoutTma = 1, kDevTimeoutMma = 2, kDevTimeoutEpi = 3 };
+
+extern int64_t g_launches;          // host-side launch counter
+
+// ---- stage launchers (host) ----------------------------------------------------------------
+cudaError_t launch_indexer(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* qI,
+                           const __nv_bfloat16* kI, const float* w, const float* bI, float* scores,
+                           int64_t row_stride, int32_t* dev_status, cudaStream_t st);
+
+cudaError_t launch_select(const gsa_params_t& p, RowRange rr, const float* scores,
+                          int64_t row_stride, int32_t* idx, int32_t* kt, float* var,
+                          IdxLayout il, cudaStream_t st);
+
+cudaError_t launch_value_gate(const __nv_bfloat16* V, const __nv_bfloat16* g2, __nv_bfloat16* Vg,
+                              int64_t n_elems, cudaStream_t st);
+
+cudaError_t launch_sparse_attn(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* Q,
+                               const __nv_bfloat16* K, const __nv_bfloat16* V,
+                               const __nv_bfloat16* g1, const __nv_bfloat16* g2 /*nullable*/,
+                               const int32_t* idx, const int32_t* kt, IdxLayout il,
+                               __nv_bfloat16* out, cudaStream_t st);
+
+// ---- device helpers ------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ float fast_sigmoid(float x) {
+    // 1 / (1 + 2^(-x log2 e)); ex2.approx and rcp.approx are accurate to a few ulp
+    return __frcp_rn(1.0f + exp2f(-1.4426950408889634f * x));
+}
+
+__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gsrc) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(smem_dst), "l"(gsrc));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;\n" ::"n"(N));
+}
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3,
+                                            uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t& r0, uint32_t& r1, uint32_t& r2,
+                                                  uint32_t& r3, uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+
+// D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                               uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
+        "{%8,%9}, {%0,%1,%2,%3};\n"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+}  // namespace gsa

@@ -1,0 +1,146 @@
+"""Helpers shared by the GPU parity tests: device staging, per-stage calls through the C ABI,
+and the comparison rules (tolerances written where they are applied)."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2601_15305_b200 import binding as gsa
+from paper_2601_15305_b200.inputs import GsaConfig
+
+# Tolerances (stated by the benchmark spec):
+SCORE_REL_TOL = 1e-3     # indexer scores, relative
+SCORE_ABS_TOL = 5e-6     # what the end-to-end index rule needs from fp32 scores (half of 1e-5)
+OUT_MAX_ABS_TOL = 2e-2   # final bf16 outputs, max-abs
+# derived: outputs are O(1e-2) at the workloads' value scale, so max-abs alone is loose; bf16 rounding of
+# P and V' (2^-9 each) and of the output (2^-9) bound the error by ~1.2% of the row's largest magnitude.
+OUT_REL_TO_ROWMAX_TOL = 2.5e-2
+E2E_SCORE_GAP = 1e-5     # an index swap is tolerated only between candidates whose oracle scores are this close
+
+
+def oracle_params(cfg: GsaConfig, **kw) -> oracle.OracleParams:
+    """Oracle parameters with v_bar rounded to fp32, the precision the C ABI carries it in."""
+    kw.setdefault("v_bar", float(np.float32(cfg.v_bar)))
+    return oracle.OracleParams.from_config(cfg, **kw)
+
+
+def to_dev(x: dict) -> dict:
+    return {k: v.cuda() for k, v in x.items()}
+
+
+def row_stride(cfg: GsaConfig) -> int:
+    return (cfg.Lk + 31) // 32 * 32
+
+
+def run_scores(cfg, d, q_begin=0, q_end=0, bI=None, poison=True):
+    """gsa_indexer_scores for rows [q_begin, q_end) of every batch element -> [B, R, stride] fp32 (NaN-poisoned)."""
+    qe = q_end or cfg.Lq
+    R = qe - q_begin
+    st = row_stride(cfg)
+    sc = torch.full((cfg.B, R, st), float("nan"), device="cuda", dtype=torch.float32) if poison else \
+        torch.empty((cfg.B, R, st), device="cuda", dtype=torch.float32)
+    ws = torch.zeros(1024, dtype=torch.uint8, device="cuda")
+    p = gsa.make_params(cfg, q_begin=q_begin, q_end=qe)
+    gsa.gsa_indexer_scores(p, d["qI"], d["kI"], d["w"], bI, sc, st, ws)
+    assert gsa.gsa_device_status(ws) == 0
+    return sc
+
+
+def run_topk(cfg, scores, q_begin=0, q_end=0, k_mode=0, **over):
+    qe = q_end or cfg.Lq
+    R = qe - q_begin
+    p = gsa.make_params(cfg, q_begin=q_begin, q_end=qe, k_mode=k_mode, **over)
+    idx = torch.full((cfg.B, R, p.k_max), -7, device="cuda", dtype=torch.int32)
+    kt = torch.full((cfg.B, R), -7, device="cuda", dtype=torch.int32)
+    var = torch.empty((cfg.B, R), device="cuda", dtype=torch.float32)
+    gsa.gsa_adaptive_topk(p, scores, scores.shape[-1], idx, kt, var)
+    torch.cuda.synchronize()
+    return idx, kt, var
+
+
+def run_attn(cfg, d, idx, kt, q_begin=0, q_end=0, use_g2=True, ws_bytes=None, sm_scale=0.0, **over):
+    qe = q_end or cfg.Lq
+    p = gsa.make_params(cfg, q_begin=q_begin, q_end=qe, sm_scale=sm_scale, **over)
+    out = torch.full_like(d["Q"], float("nan"))
+    if ws_bytes is None:
+        ws_bytes = 256 + d["V"].numel() * 2
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda") if ws_bytes else None
+    gsa.gsa_sparse_gated_attn_fwd(p, d["Q"], d["K"], d["V"], d["g1"], d["g2"] if use_g2 else None, idx, kt, out, ws)
+    torch.cuda.synchronize()
+    return out
+
+
+def run_forward(cfg, d, slab_rows=0, bI=None, want_idx=True, k_mode=0, **over):
+    p = gsa.make_params(cfg, k_mode=k_mode, **over)
+    out = torch.full_like(d["Q"], float("nan"))
+    idx = torch.full((cfg.B, cfg.Lq, p.k_max), -7, device="cuda", dtype=torch.int32) if want_idx else None
+    kt = torch.full((cfg.B, cfg.Lq), -7, device="cuda", dtype=torch.int32)
+    var = torch.empty((cfg.B, cfg.Lq), device="cuda", dtype=torch.float32)
+    ws = torch.empty(gsa.gsa_workspace_bytes(p, slab_rows), dtype=torch.uint8, device="cuda")
+    gsa.gsa_forward(p, d["Q"], d["K"], d["V"], d["qI"], d["kI"], d["w"], bI, d["g1"], d["g2"], out, idx, kt, var,
+                    slab_rows, ws)
+    assert gsa.gsa_device_status(ws) == 0
+    return out, idx, kt, var
+
+
+def check_scores(got_rows: np.ndarray, want_rows: np.ndarray, n_vis):
+    """got/want: [n, >=Lk]; n_vis[i] visible keys of row i."""
+    for i, n in enumerate(n_vis):
+        g, w = got_rows[i, :n].astype(np.float64), want_rows[i, :n]
+        assert np.isfinite(g).all()
+        rel = np.abs(g - w) / np.abs(w)
+        assert rel.max() <= SCORE_REL_TOL, (i, rel.max())
+        assert np.abs(g - w).max() <= SCORE_ABS_TOL, (i, np.abs(g - w).max())
+
+
+def check_selection_exact(o: dict, idx: np.ndarray, kt: np.ndarray, oracle_select_again=None):
+    """Bit-exact index sets given the same fp32 scores.  If k_t differs, it may only be because
+    k_base*Var/v_bar sits within 1e-9 (relative) of an integer; sets are nested, so the GPU's set
+    must then be the oracle's top-k for the GPU's k (checked by the caller via oracle_select_again)."""
+    n = len(kt)
+    for i in range(n):
+        if kt[i] != o["keff"][i]:
+            r = o["r"][i]
+            assert abs(r - round(r)) <= 1e-9 * max(1.0, abs(r)), (i, kt[i], o["keff"][i], r)
+            assert oracle_select_again is not None
+            want = oracle_select_again(i, int(kt[i]))
+        else:
+            want = o["idx"][i]
+        k = int(kt[i])
+        assert (idx[i, :k] == want[:k]).all(), f"row {i}: index set differs"
+        assert (idx[i, k:] == -1).all(), f"row {i}: padding is not -1"
+
+
+def check_out(got: np.ndarray, want: np.ndarray):
+    """got: bf16->float [n, n_h, d_h]; want: oracle fp64."""
+    assert np.isfinite(got).all()
+    err = np.abs(got.astype(np.float64) - want)
+    assert err.max() <= OUT_MAX_ABS_TOL, err.max()
+    rowmax = np.abs(want).max(axis=-1, keepdims=True)
+    assert (err <= OUT_REL_TO_ROWMAX_TOL * rowmax + 1e-6).all(), (err / (rowmax + 1e-30)).max()
+
+
+def check_e2e_indices(o: dict, idx: np.ndarray, kt: np.ndarray, oracle_scores: np.ndarray, n_vis):
+    """End to end, an index may differ from the oracle's only where the two candidates' oracle scores
+    differ by less than 1e-5 (fp32 vs fp64 scoring)."""
+    mism = 0
+    for i, n in enumerate(n_vis):
+        kg, ko = int(kt[i]), int(o["keff"][i])
+        sg, so = set(idx[i, :kg].tolist()), set(o["idx"][i, :ko].tolist())
+        if kg != ko:
+            # budget flipped across an integer because the fp32 scores shift the variance slightly
+            r = o["r"][i]
+            assert abs(kg - ko) <= 1 and abs(r - round(r)) < 1e-2, (i, kg, ko, r)
+        only_g, only_o = sorted(sg - so), sorted(so - sg)
+        if not only_g and not only_o:
+            continue
+        mism += 1
+        sc = oracle_scores[i]
+        # every swapped pair must be a near-tie at the selection boundary
+        lo = min(sc[j] for j in (only_g + only_o))
+        hi = max(sc[j] for j in (only_g + only_o))
+        if kg == ko:
+            assert hi - lo < E2E_SCORE_GAP, (i, only_g, only_o, hi - lo)
+        assert all(0 <= j < n for j in sg)
+    return mism

@@ -1,0 +1,341 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 CPU oracle on the same
+seeded inputs.  Per stage (scores within 1e-3 relative; index sets bit-exact on equal fp32 scores;
+outputs within 2e-2 max-abs) and end to end."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2601_15305_b200 import binding as gsa
+from paper_2601_15305_b200.inputs import CONFIGS, make_inputs, sample_rows
+
+import gpu_util as U
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def tiny():
+    cfg = CONFIGS["tiny"]
+    x = make_inputs(cfg)
+    return cfg, x, U.to_dev(x)
+
+
+@pytest.fixture(scope="module")
+def l8k():
+    cfg = CONFIGS["l8k"]
+    x = make_inputs(cfg)
+    return cfg, x, U.to_dev(x)
+
+
+def _vis(cfg, rows):
+    return [cfg.Lk - cfg.Lq + int(t) + 1 for t in rows]
+
+
+# ------------------------------------------------------------------------------------------ stage 1
+@pytest.mark.parametrize("path", [0, 1])
+def test_indexer_tiny_all_rows(tiny, path):
+    cfg, x, d = tiny
+    gsa.gsa_debug_set_indexer_path(path)
+    try:
+        sc = U.run_scores(cfg, d)[0].cpu().numpy()
+    finally:
+        gsa.gsa_debug_set_indexer_path(0)
+    rows = np.arange(cfg.Lq)
+    want = oracle.scores(U.oracle_params(cfg), x["qI"], x["kI"], x["w"], None, rows)
+    U.check_scores(sc, want, _vis(cfg, rows))
+    # nothing is written past a row's visible keys (buffer was NaN-poisoned)
+    for t in (0, 100, 510):
+        assert np.isnan(sc[t, t + 1:cfg.Lk]).all()
+    # fp32 scores stay inside [0, sum_j w_j] (the paper's (0, H^I))
+    wsum = x["w"][0].sum(-1).numpy()
+    for t in rows:
+        assert (sc[t, :t + 1] >= 0).all() and (sc[t, :t + 1] <= wsum[t] * (1 + 1e-6)).all()
+
+
+@pytest.mark.parametrize("path", [0, 1])
+def test_indexer_bias_and_row_range(tiny, path):
+    cfg, x, d = tiny
+    bI = torch.tensor([0.5, -1.0, 2.0, 0.0], dtype=torch.float32)
+    gsa.gsa_debug_set_indexer_path(path)
+    try:
+        sc = U.run_scores(cfg, d, q_begin=37, q_end=301, bI=bI.cuda())[0].cpu().numpy()
+    finally:
+        gsa.gsa_debug_set_indexer_path(0)
+    rows = np.arange(37, 301)
+    want = oracle.scores(U.oracle_params(cfg), x["qI"], x["kI"], x["w"], bI, rows)
+    U.check_scores(sc, want, _vis(cfg, rows))
+
+
+@pytest.mark.parametrize("path", [0, 1])
+def test_indexer_l8k_sampled_rows(l8k, path):
+    cfg, x, d = l8k
+    gsa.gsa_debug_set_indexer_path(path)
+    try:
+        sc = U.run_scores(cfg, d)[0]
+    finally:
+        gsa.gsa_debug_set_indexer_path(0)
+    rows = sample_rows(cfg, 48).numpy()
+    got = sc[torch.from_numpy(rows).cuda()].cpu().numpy()
+    want = oracle.scores(U.oracle_params(cfg), x["qI"], x["kI"], x["w"], None, rows)
+    U.check_scores(got, want, _vis(cfg, rows))
+
+
+def test_indexer_ragged_batch_decode_shapes():
+    """Lq not a multiple of any tile, Lk > Lq (chunked prefill), B > 1."""
+    cfg = CONFIGS["l8k"].with_(name="ragged", B=2, Lq=203, Lk=459, seed=11)
+    x = make_inputs(cfg)
+    d = U.to_dev(x)
+    for path in (0, 1):
+        gsa.gsa_debug_set_indexer_path(path)
+        try:
+            sc = U.run_scores(cfg, d).cpu().numpy()
+        finally:
+            gsa.gsa_debug_set_indexer_path(0)
+        p = U.oracle_params(cfg)
+        for b in range(cfg.B):
+            rows = np.arange(cfg.Lq)
+            want = oracle.scores(p, x["qI"], x["kI"], x["w"], None, rows, np.full_like(rows, b))
+            U.check_scores(sc[b], want, _vis(cfg, rows))
+
+
+# ------------------------------------------------------------------------------------------ stage 2
+def _select_and_compare(cfg, sc_dev, rows=None, k_mode=0, **over):
+    """sc_dev: [B, Lq, stride] fp32 on the GPU; compares every (or the listed) row of batch 0."""
+    idx, kt, var = U.run_topk(cfg, sc_dev, k_mode=k_mode, **over)
+    rows = np.arange(cfg.Lq) if rows is None else np.asarray(rows)
+    sel = torch.from_numpy(rows).cuda()
+    sc_rows = sc_dev[0][sel].cpu().numpy()
+    p = U.oracle_params(cfg, k_mode=k_mode, **over)
+    o = oracle.select_f32(p, sc_rows, rows)
+
+    def again(i, k):
+        p2 = U.oracle_params(cfg, k_mode=2, **{**over, "k_base": k, "k_min": 1, "k_max": p.k_max})
+        return oracle.select_f32(p2, sc_rows[i:i + 1], rows[i:i + 1])["idx"][0]
+
+    U.check_selection_exact(o, idx[0][sel].cpu().numpy(), kt[0][sel].cpu().numpy(), again)
+    np.testing.assert_allclose(var[0][sel].cpu().numpy(), o["var"], rtol=2e-6, atol=1e-12)
+    return o, kt[0][sel].cpu().numpy()
+
+
+@pytest.mark.parametrize("k_mode", [0, 1, 2])
+def test_topk_bit_exact_tiny(tiny, k_mode):
+    cfg, x, d = tiny
+    sc = U.run_scores(cfg, d, poison=True)
+    o, kt = _select_and_compare(cfg, sc, k_mode=k_mode)
+    if k_mode == 0:
+        assert len(set(kt.tolist())) > 5          # budgets really vary
+    if k_mode == 2:
+        assert (kt == np.minimum(cfg.k_base, np.arange(cfg.Lq) + 1)).all()
+
+
+def test_topk_bit_exact_on_oracle_scores_with_ties():
+    """Scores quantised to a few levels: thousands of exact ties; lower position must win."""
+    cfg = CONFIGS["tiny"].with_(Lq=700, Lk=700, k_base=100, k_min=30, k_max=333)
+    g = torch.Generator().manual_seed(5)
+    lv = torch.randint(0, 7, (1, cfg.Lq, U.row_stride(cfg)), generator=g).float() * 0.125 + 0.5
+    lv[0, 500:520] = 1.25                         # constant rows: variance 0
+    sc = lv.cuda()
+    for k_mode in (0, 1, 2):
+        _select_and_compare(cfg, sc, k_mode=k_mode, v_bar=0.05)
+
+
+def test_topk_wide_dynamic_range_and_negatives():
+    """Keys spanning many binades (three radix rounds) and negative values."""
+    cfg = CONFIGS["tiny"].with_(Lq=1500, Lk=1500, k_base=200, k_min=10, k_max=1000)
+    g = torch.Generator().manual_seed(6)
+    e = torch.randint(-20, 3, (1, cfg.Lq, U.row_stride(cfg)), generator=g).float()
+    sc = (torch.rand(e.shape, generator=g) + 1.0) * torch.pow(2.0, e)
+    sc[0, 1000:1100] *= -1.0
+    sc[0, 1200:1300, ::3] *= -1.0
+    _select_and_compare(cfg, sc.cuda(), k_mode=2)
+    _select_and_compare(cfg, sc.cuda(), k_mode=0, v_bar=0.3)
+
+
+def test_topk_l8k_rows_cached_and_global_paths(l8k):
+    cfg, x, d = l8k
+    sc = U.run_scores(cfg, d)
+    rows = sample_rows(cfg, 64).numpy()
+    _select_and_compare(cfg, sc, rows=rows)
+
+
+def test_topk_long_rows_take_the_uncached_path():
+    """Rows longer than the shared-memory cache (n > ~46K) are re-read from global memory."""
+    cfg = CONFIGS["l8k"].with_(name="long", B=1, Lq=8, Lk=70000, seed=12)
+    x = make_inputs(cfg)
+    d = U.to_dev(x)
+    sc = U.run_scores(cfg, d)
+    _select_and_compare(cfg, sc)
+
+
+# ------------------------------------------------------------------------------------------ stage 3
+def _oracle_idx(cfg, x, rows, **kw):
+    p = U.oracle_params(cfg, **kw)
+    return p, oracle.forward(p, **x, rows_t=rows, want_scores=True)
+
+
+def test_attn_given_oracle_indices_tiny(tiny):
+    cfg, x, d = tiny
+    rows = np.arange(cfg.Lq)
+    p, o = _oracle_idx(cfg, x, rows)
+    idx = torch.from_numpy(o["idx"]).cuda()[None]
+    kt = torch.from_numpy(o["keff"]).cuda()[None]
+    for use_prepass in (True, False):
+        out = U.run_attn(cfg, d, idx, kt, ws_bytes=None if use_prepass else 0)
+        U.check_out(out[0].float().cpu().numpy(), o["out"])
+
+
+def test_attn_pregated_values_and_custom_scale(tiny):
+    cfg, x, d = tiny
+    rows = np.arange(0, cfg.Lq, 7)
+    p = U.oracle_params(cfg, sm_scale=0.2)
+    o = oracle.forward(p, **x, rows_t=rows)
+    # rows subset through q_begin/q_end is contiguous; use the full range and compare the subset
+    po, oa = _oracle_idx(cfg, x, np.arange(cfg.Lq))
+    idx = torch.from_numpy(oa["idx"]).cuda()[None]
+    kt = torch.from_numpy(oa["keff"]).cuda()[None]
+    out = U.run_attn(cfg, d, idx, kt, sm_scale=0.2)
+    U.check_out(out[0, rows].float().cpu().numpy(), o["out"])
+    # g2 = NULL means V is already gated: feed V' = V*sigmoid(g2) rounded to bf16
+    d2 = dict(d)
+    d2["V"] = (d["V"].float() * torch.sigmoid(d["g2"].float())).to(torch.bfloat16)
+    out2 = U.run_attn(cfg, d2, idx, kt, use_g2=False, sm_scale=0.2)
+    U.check_out(out2[0, rows].float().cpu().numpy(), o["out"])
+
+
+def test_attn_l8k_sampled_rows(l8k):
+    cfg, x, d = l8k
+    rows = sample_rows(cfg, 24).numpy()
+    p, o = _oracle_idx(cfg, x, rows)
+    q0, q1 = int(rows.min()), int(rows.max()) + 1
+    # place the oracle's index sets into a full [R, k_max] table (other rows: a valid dummy set)
+    R = q1 - q0
+    idx = torch.zeros((1, R, cfg.k_max), dtype=torch.int32)
+    kt = torch.ones((1, R), dtype=torch.int32)
+    idx[0, rows - q0] = torch.from_numpy(o["idx"])
+    kt[0, rows - q0] = torch.from_numpy(o["keff"])
+    out = U.run_attn(cfg, d, idx.cuda(), kt.cuda(), q_begin=q0, q_end=q1)
+    U.check_out(out[0, rows].float().cpu().numpy(), o["out"])
+    # rows outside [q_begin, q_end) are untouched (NaN-poisoned)
+    if q0 > 0:
+        assert torch.isnan(out[0, :q0].float()).all()
+
+
+def test_attn_saturated_gates_is_plain_attention(tiny):
+    """Gate logits +40: sigmoid is 1.0 in fp32 too, the layer is ungated sparse attention."""
+    cfg, x, d = tiny
+    x2 = dict(x)
+    x2["g1"] = torch.full_like(x["g1"], 40.0)
+    x2["g2"] = torch.full_like(x["g2"], 40.0)
+    rows = np.arange(cfg.Lq)
+    p, o = _oracle_idx(cfg, x2, rows)
+    d2 = U.to_dev(x2)
+    out = U.run_attn(cfg, d2, torch.from_numpy(o["idx"]).cuda()[None], torch.from_numpy(o["keff"]).cuda()[None])
+    U.check_out(out[0].float().cpu().numpy(), o["out"])
+    # and g1 = -40 closes the output gate
+    d2["g1"] = torch.full_like(d["g1"], -40.0)
+    out = U.run_attn(cfg, d2, torch.from_numpy(o["idx"]).cuda()[None], torch.from_numpy(o["keff"]).cuda()[None])
+    assert out.float().abs().max().item() < 1e-12
+
+
+# ------------------------------------------------------------------------------------------ end to end
+def _forward_and_compare(cfg, x, d, rows, slab_rows=0, **kw):
+    out, idx, kt, var = U.run_forward(cfg, d, slab_rows=slab_rows, **kw)
+    rows = np.asarray(rows)
+    sel = torch.from_numpy(rows).cuda()
+    p = U.oracle_params(cfg, **kw)
+    o = oracle.forward(p, **x, rows_t=rows, want_scores=True)
+    mism = U.check_e2e_indices(o, idx[0][sel].cpu().numpy(), kt[0][sel].cpu().numpy(), o["scores"], _vis(cfg, rows))
+    U.check_out(out[0][sel].float().cpu().numpy(), o["out"])
+    assert not torch.isnan(out.float()).any()
+    return mism, kt
+
+
+@pytest.mark.parametrize("slab_rows", [0, 32, 96])
+def test_forward_tiny_all_rows(tiny, slab_rows):
+    cfg, x, d = tiny
+    mism, kt = _forward_and_compare(cfg, x, d, np.arange(cfg.Lq), slab_rows=slab_rows)
+    assert mism <= 5
+
+
+def test_forward_l8k_sampled_rows(l8k):
+    cfg, x, d = l8k
+    mism, kt = _forward_and_compare(cfg, x, d, sample_rows(cfg, 40).numpy())
+    k = kt[0, cfg.k_max:].float()
+    assert k.min() >= cfg.k_min and k.max() <= cfg.k_max and k.mean() > 1200 and k.mean() < 3000
+
+
+def test_forward_large_budget_equals_dense_gated_attention():
+    """k_min >= L: S_t is everything visible; the output is dense gated attention (oracle's dense limit)."""
+    cfg = CONFIGS["tiny"].with_(Lq=200, Lk=200, k_base=256, k_min=256, k_max=256)
+    x = make_inputs(cfg)
+    d = U.to_dev(x)
+    out, idx, kt, var = U.run_forward(cfg, d)
+    assert (kt[0].cpu().numpy() == np.arange(1, 201)).all()
+    for t in (0, 1, 57, 199):
+        assert idx[0, t, :t + 1].tolist() == list(range(t + 1)) and (idx[0, t, t + 1:] == -1).all()
+    o = oracle.forward(U.oracle_params(cfg), **x, rows_t=np.arange(200))
+    U.check_out(out[0].float().cpu().numpy(), o["out"])
+
+
+def test_forward_batched_chunked_prefill():
+    """B = 3, Lk > Lq, ragged sizes, k_max not a multiple of the 16-key tile."""
+    cfg = CONFIGS["l8k"].with_(name="chunk", B=3, Lq=150, Lk=1111, k_base=300, k_min=50, k_max=777, seed=13,
+                               v_bar=2.0e-3)
+    x = make_inputs(cfg)
+    d = U.to_dev(x)
+    out, idx, kt, var = U.run_forward(cfg, d, slab_rows=64)
+    p = U.oracle_params(cfg)
+    for b in range(cfg.B):
+        rows = np.arange(0, cfg.Lq, 5)
+        o = oracle.forward(p, **x, rows_t=rows, rows_b=np.full_like(rows, b), want_scores=True)
+        U.check_e2e_indices(o, idx[b][rows].cpu().numpy(), kt[b][rows].cpu().numpy(), o["scores"], _vis(cfg, rows))
+        U.check_out(out[b][rows].float().cpu().numpy(), o["out"])
+
+
+def test_forward_small_decode_batch():
+    """Decode geometry (Lq = 1) with the value gate applied inside the gather."""
+    cfg = CONFIGS["decode"].with_(name="dec_small", B=5, Lk=9000, seed=14)
+    x = make_inputs(cfg)
+    d = U.to_dev(x)
+    out, idx, kt, var = U.run_forward(cfg, d)
+    p = U.oracle_params(cfg)
+    rows_b = np.arange(cfg.B)
+    o = oracle.forward(p, **x, rows_t=np.zeros(cfg.B, np.int32), rows_b=rows_b, want_scores=True)
+    U.check_e2e_indices(o, idx[:, 0].cpu().numpy(), kt[:, 0].cpu().numpy(), o["scores"], [cfg.Lk] * cfg.B)
+    U.check_out(out[:, 0].float().cpu().numpy(), o["out"])
+
+
+def test_forward_is_deterministic(tiny):
+    cfg, x, d = tiny
+    a = U.run_forward(cfg, d)
+    b = U.run_forward(cfg, d)
+    assert torch.equal(a[1], b[1]) and torch.equal(a[2], b[2])
+    assert torch.equal(a[0].view(torch.int16), b[0].view(torch.int16))
+
+
+def test_forward_host_buffers_match_device_call(tiny):
+    cfg, x, d = tiny
+    p = gsa.make_params(cfg)
+    out_dev, _, kt_dev, _ = U.run_forward(cfg, d)
+    pin = {k: v.pin_memory() for k, v in x.items()}
+    out_h = torch.empty_like(x["Q"]).pin_memory()
+    kt_h = torch.empty((cfg.B, cfg.Lq), dtype=torch.int32).pin_memory()
+    arena = torch.empty(gsa.gsa_forward_host_arena_bytes(p, 0), dtype=torch.uint8, device="cuda")
+    gsa.gsa_forward_host(p, pin["Q"], pin["K"], pin["V"], pin["qI"], pin["kI"], pin["w"], None, pin["g1"], pin["g2"],
+                         out_h, kt_h, 0, arena)
+    assert torch.equal(out_h.view(torch.int16), out_dev.cpu().view(torch.int16))
+    assert torch.equal(kt_h, kt_dev.cpu())
+
+
+def test_argument_errors_do_not_launch(tiny):
+    cfg, x, d = tiny
+    p = gsa.make_params(cfg)
+    n0 = gsa.gsa_launch_count()
+    out = torch.empty_like(d["Q"])
+    small_ws = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(gsa.GsaError, match="workspace"):
+        gsa.gsa_forward(p, d["Q"], d["K"], d["V"], d["qI"], d["kI"], d["w"], None, d["g1"], d["g2"], out, ws=small_ws)
+    with pytest.raises(gsa.GsaError, match="invalid"):
+        gsa.gsa_indexer_scores(p, d["qI"], d["kI"], d["w"], None, torch.empty(10, device="cuda"), 100, small_ws)
+    assert gsa.gsa_launch_count() == n0
