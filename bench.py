@@ -1,0 +1,304 @@
+#!/usr/bin/env python
+"""Benchmark of the GSA forward path: tokens/s of gsa_forward at L = 128K on one B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload l128k] [--impl reference]
+
+A step is one gsa_forward over the whole workload (value gate, indexer, budget, top-k,
+sparse attention, output gate).  Inputs are seeded synthetic tensors, resident in HBM before
+the timed region; `e2e` repeats the measurement through gsa_forward_host with pinned host
+buffers, so host<->device copies are inside its timed region.  N > 1 runs N independent
+replicas (the path has no exchange step) and reports the aggregate.
+`--impl reference` times the CPU oracle, as it stands, on a bounded sample of the same
+workload (rank 0 only).
+Prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2601_15305_b200.inputs import CONFIGS, make_inputs, sample_rows
+
+METRIC = "gsa_fwd_tokens_per_s"
+UNIT = "tokens/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons sampled every 200 ms while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows, self.proc, self.gpu = [], None, gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "200", "-i", str(self.gpu)], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        self.thread.join(timeout=2)
+        sm = [float(r[1]) for r in self.rows if len(r) >= 9 and r[1].replace(".", "").isdigit()]
+        mx = [float(r[2]) for r in self.rows if len(r) >= 9 and r[2].replace(".", "").isdigit()]
+        reasons = set()
+        for r in self.rows:
+            if len(r) >= 9:
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def aggregate_over_ranks(ms_local: float, units_local: float):
+    """max time over ranks, sum of units: the whole-job throughput of N independent replicas."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return ms_local, units_local
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([ms_local], dtype=torch.float64, device=dev)
+    u = torch.tensor([units_local], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+def attention_bytes(cfg, kt_sum: int) -> float:
+    """Algorithmic bytes of one sparse-attention launch: per selected (t, s) one K row and one V' row of
+    all KV heads (2 * n_kv * d_h * 2 B) and one 4-byte index; per token Q, g1 and out (3 * n_h * d_h * 2 B)."""
+    per_pair = 2 * cfg.n_kv * cfg.d_h * 2 + 4
+    per_tok = 3 * cfg.n_h * cfg.d_h * 2 + 4
+    return float(kt_sum) * per_pair + float(cfg.B * cfg.Lq) * per_tok
+
+
+def oracle_sample_rate(cfg, x, n_rows: int):
+    """tokens/s of the fp64 oracle on a stratified sample of query rows (mean row cost = mean over the sequence)."""
+    import oracle
+    p = oracle.OracleParams.from_config(cfg, v_bar=float(np.float32(cfg.v_bar)))
+    if cfg.decode:
+        rows_b = np.arange(min(cfg.B, n_rows), dtype=np.int32)
+        rows_t = np.zeros_like(rows_b)
+    else:
+        strata = np.linspace(0, cfg.Lq, n_rows + 1)
+        rows_t = ((strata[:-1] + strata[1:]) / 2).astype(np.int32)
+        rows_b = np.zeros_like(rows_t)
+    f32 = {k: oracle._f32(v) for k, v in x.items()}          # widening is not part of the timed work
+    t0 = time.perf_counter()
+    oracle.forward(p, **f32, rows_t=rows_t, rows_b=rows_b)
+    dt = time.perf_counter() - t0
+    return len(rows_t) / dt, dt, len(rows_t), oracle.num_threads()
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    x = make_inputs(cfg, slice(0, min(cfg.B, 4)) if cfg.decode else None)
+    cores = oracle.num_threads()
+    n_rows = 256
+    rates = []
+    for i in range(args.warmup + args.steps):
+        r, dt, n, cores = oracle_sample_rate(cfg.with_(B=x["Q"].shape[0]), x, n_rows)
+        if i >= args.warmup:
+            rates.append((r, dt))
+    value = float(np.mean([r for r, _ in rates]))
+    ms = float(np.mean([dt for _, dt in rates]) * 1e3)
+    sample = f"{n_rows} stratified query rows of {cfg.name} per step, full visible context each, fp64, OpenMP"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(cfg),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def workload_config(cfg):
+    return {"workload": f"{cfg.name}: GSA layer fwd, B={cfg.B}, Lq={cfg.Lq}, Lk={cfg.Lk}, causal, n_h={cfg.n_h}, "
+                        f"n_kv={cfg.n_kv}, d_h={cfg.d_h}, H^I={cfg.HI}, d^I={cfg.dI}, k_base={cfg.k_base}, "
+                        f"k in [{cfg.k_min},{cfg.k_max}], planted needles, seed {cfg.seed}",
+            "global_batch_tokens": cfg.B * cfg.Lq, "seq_len": cfg.Lk, "parallelism": "replicas",
+            "l2": "inputs (>= 1 GB) exceed the 126 MB L2; no flush between steps"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="l128k", choices=sorted(CONFIGS))
+    ap.add_argument("--impl", default="gsa_b200", choices=["gsa_b200", "reference"])
+    ap.add_argument("--slab-rows", type=int, default=0)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "gsa_b200" else args.warmup
+    cfg = CONFIGS[args.workload]
+
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    from paper_2601_15305_b200 import binding as gsa
+    gsa.lib()                                   # fails loudly if the CUDA library is missing
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device"
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    x = make_inputs(cfg)
+    d = {k: v.cuda() for k, v in x.items()}
+    p = gsa.make_params(cfg)
+    out = torch.empty_like(d["Q"])
+    kt = torch.empty((cfg.B, cfg.Lq), dtype=torch.int32, device="cuda")
+    ws = torch.empty(gsa.gsa_workspace_bytes(p, args.slab_rows), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step():
+        gsa.gsa_forward(p, d["Q"], d["K"], d["V"], d["qI"], d["kI"], d["w"], None, d["g1"], d["g2"], out, None, kt,
+                        None, args.slab_rows, ws, stream)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    assert gsa.gsa_device_status(ws) == 0
+    kt_sum = int(kt.sum().item())
+
+    # per-step stage events (recorded by the library on the launching stream)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    for tri in evs:
+        for e in tri:
+            e.record(stream)
+    t_beg, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    n0 = gsa.gsa_launch_count()
+    t_beg.record(stream)
+    for i in range(args.steps):
+        gsa.gsa_profile_set_events(*evs[i])
+        step()
+    t_end.record(stream)
+    barrier()
+    launches = gsa.gsa_launch_count() - n0
+    clocks = sampler.stop()
+    gsa.gsa_profile_set_events(None, None, None)
+    assert gsa.gsa_device_status(ws) == 0
+    ms_local = t_beg.elapsed_time(t_end)
+    ms_total, tokens_total = aggregate_over_ranks(ms_local, float(cfg.B * cfg.Lq * args.steps))
+    value = tokens_total / (ms_total * 1e-3)
+    sel_ms = float(np.mean([tri[0].elapsed_time(tri[1]) for tri in evs]))
+    attn_ms = float(np.mean([tri[1].elapsed_time(tri[2]) for tri in evs]))
+
+    peaks = measured_peaks()
+    ab = attention_bytes(cfg, kt_sum)
+    achieved = ab / (attn_ms * 1e-3) / 1e9
+    roofline = {"kernel": "gsa_sparse_attn_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                "peak_source": f"{peaks['source']} (MEASURED_PEAKS.json hbm_gbs)" if peaks["source"] == "measured"
+                else "fallback 6650 GB/s",
+                "algorithmic_bytes_per_launch": ab, "launch_ms": attn_ms,
+                "note": "frac may exceed 1 when the 126 MB L2 serves part of the gather"}
+    causal_pairs = cfg.B * sum(cfg.Lk - cfg.Lq + t + 1 for t in (0, cfg.Lq - 1)) * cfg.Lq / 2.0
+    stages = {"indexer_plus_topk_ms": sel_ms, "sparse_attn_ms": attn_ms,
+              "indexer_causal_tflop": 2.0 * cfg.HI * cfg.dI * causal_pairs / 1e12,
+              "mean_k_t": kt_sum / float(cfg.B * cfg.Lq)}
+
+    # ---- end to end through the host-buffer entry point ------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        pin = {k: v.pin_memory() for k, v in x.items()}
+        out_h = torch.empty_like(x["Q"]).pin_memory()
+        kt_h = torch.empty((cfg.B, cfg.Lq), dtype=torch.int32).pin_memory()
+        del ws
+        arena = torch.empty(gsa.gsa_forward_host_arena_bytes(p, args.slab_rows), dtype=torch.uint8, device="cuda")
+        h2d = sum(v.numel() * v.element_size() for v in pin.values())
+        d2h = out_h.numel() * 2 + kt_h.numel() * 4
+
+        def step_host():
+            gsa.gsa_forward_host(p, pin["Q"], pin["K"], pin["V"], pin["qI"], pin["kI"], pin["w"], None, pin["g1"],
+                                 pin["g2"], out_h, kt_h, args.slab_rows, arena, stream)
+
+        step_host()
+        barrier()
+        e_steps = max(1, min(args.steps, 3))
+        t0 = time.perf_counter()
+        for _ in range(e_steps):
+            step_host()                      # returns after the result is on the host
+        barrier()
+        e_ms, e_tok = aggregate_over_ranks((time.perf_counter() - t0) * 1e3, float(cfg.B * cfg.Lq * e_steps))
+        e2e = {"value": e_tok / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "steps": e_steps, "api": "gsa_forward_host (pinned host buffers)"}
+        assert torch.equal(out_h.view(torch.int16), out.cpu().view(torch.int16)), "host and device paths disagree"
+
+    # ---- the oracle on the host cores, bounded sample (rank 0, N = 1 only) ------------------
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        cores = oracle.num_threads()
+        n_rows = 256
+        r, dt, n, cores = oracle_sample_rate(cfg, x, n_rows)
+        cpu_baseline = {"value": r, "unit": UNIT, "cores": cores, "kind": "oracle",
+                        "sample": f"{n} stratified query rows of {cfg.name} (full visible context each), {dt:.1f} s"}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": workload_config(cfg), "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+                "roofline": roofline, "cpu_baseline": cpu_baseline, "stages": stages}
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -162,6 +162,14 @@ int64_t gsa_launch_count(void);
  */
 void gsa_debug_set_indexer_path(int32_t path);
 
+/*
+ * Profiling hook: three cudaEvent_t handles (or NULL to switch off) that every following
+ * gsa_forward records on its stream: at entry, after the last indexer/top-k slab (before the
+ * sparse-attention launch), and after the sparse-attention launch.  Process-wide; the caller
+ * owns the events and reads them after synchronising.
+ */
+void gsa_profile_set_events(void *ev_begin, void *ev_selected, void *ev_end);
+
 /* Static string for a gsa_status value. */
 const char *gsa_status_string(int status);
 

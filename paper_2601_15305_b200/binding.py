@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_PKG, "libgsa_b200.so")
 EXPORTS = (
     "gsa_workspace_bytes", "gsa_indexer_scores", "gsa_adaptive_topk", "gsa_sparse_gated_attn_fwd",
     "gsa_forward", "gsa_forward_host_arena_bytes", "gsa_forward_host", "gsa_device_status",
-    "gsa_launch_count", "gsa_debug_set_indexer_path", "gsa_status_string",
+    "gsa_launch_count", "gsa_debug_set_indexer_path", "gsa_profile_set_events", "gsa_status_string",
 )
 
 
@@ -157,3 +157,9 @@ def gsa_launch_count() -> int:
 
 def gsa_debug_set_indexer_path(path: int) -> None:
     lib().gsa_debug_set_indexer_path(ctypes.c_int32(path))
+
+
+def gsa_profile_set_events(ev_begin=None, ev_selected=None, ev_end=None) -> None:
+    """torch.cuda.Event objects (already recorded once, so their handles exist) or None."""
+    h = lambda e: ctypes.c_void_p(0 if e is None else e.cuda_event)
+    lib().gsa_profile_set_events(h(ev_begin), h(ev_selected), h(ev_end))

@@ -9,6 +9,7 @@ namespace gsa {
 
 int64_t g_launches = 0;
 static int32_t g_indexer_path = 0;
+static cudaEvent_t g_prof_ev[3] = {nullptr, nullptr, nullptr};
 
 cudaError_t launch_indexer_simple(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* qI,
                                   const __nv_bfloat16* kI, const float* w, const float* bI,
@@ -196,6 +197,7 @@ int gsa_forward(const gsa_params_t* p, const void* Q, const void* K, const void*
     int32_t* kt = kt_out ? kt_out : (int32_t*)(wsb + wp.kt_off);
     const IdxLayout il{0, 0, p->Lq};
 
+    if (g_prof_ev[0]) cudaEventRecord(g_prof_ev[0], st);
     // Eq. 9: value gate (independent of the indexer)
     const bf16* Vuse = (const bf16*)V;
     const bf16* g2use = (const bf16*)g2_logits;
@@ -230,9 +232,12 @@ int gsa_forward(const gsa_params_t* p, const void* Q, const void* K, const void*
     }
 
     // Eq. 11, 12, 10 over all rows
+    if (g_prof_ev[1]) cudaEventRecord(g_prof_ev[1], st);
     RowRange all{0, p->B, 0, p->Lq};
-    return cuda_rc(launch_sparse_attn(*p, all, (const bf16*)Q, (const bf16*)K, Vuse, (const bf16*)g1_logits,
-                                      g2use, idx, kt, il, (bf16*)out, st));
+    e = launch_sparse_attn(*p, all, (const bf16*)Q, (const bf16*)K, Vuse, (const bf16*)g1_logits, g2use, idx,
+                           kt, il, (bf16*)out, st);
+    if (g_prof_ev[2]) cudaEventRecord(g_prof_ev[2], st);
+    return cuda_rc(e);
 }
 
 int gsa_forward_host_arena_bytes(const gsa_params_t* p, int32_t slab_rows, size_t* bytes) {
@@ -303,6 +308,12 @@ int gsa_device_status(const void* ws, void* stream, int32_t* status_out) {
 int64_t gsa_launch_count(void) { return g_launches; }
 
 void gsa_debug_set_indexer_path(int32_t path) { g_indexer_path = path; }
+
+void gsa_profile_set_events(void* ev_begin, void* ev_selected, void* ev_end) {
+    g_prof_ev[0] = (cudaEvent_t)ev_begin;
+    g_prof_ev[1] = (cudaEvent_t)ev_selected;
+    g_prof_ev[2] = (cudaEvent_t)ev_end;
+}
 
 const char* gsa_status_string(int s) {
     switch (s) {
