@@ -1,9 +1,465 @@
-// placeholder until the tcgen05 kernel lands
+// Gated lightning indexer (Eq. 7) on the 5th-generation tensor cores.
+//
+//   D[s, (t, j)] = k^I[s, :] . q^I[t, j, :]         tcgen05.mma, bf16 x bf16 -> fp32 in TMEM
+//   I[t, s]      = sum_j w[t, j] * sigmoid(D[s, (t, j)] + b_j)      epilogue, in registers
+//
+// Orientation: keys are the M dimension (128 per tile = the 128 TMEM lanes), the N dimension is
+// (query, indexer head) flattened, 256 columns = 256/H^I queries.  A thread of the epilogue owns
+// one key: it reads that key's 256 accumulators, sums the H^I adjacent columns of each query
+// after the sigmoid, and consecutive lanes write consecutive s of a score row (128-byte stores).
+//
+// A CTA works on one query group and a run of key tiles at or below the diagonal (tiles above
+// it are never touched).  Warp roles: warp 0 feeds shared memory by TMA (k^I tiles through a
+// ring of stages, the q^I tile once), warp 1 issues the MMAs and owns the TMEM allocation,
+// warps 2..9 are the epilogue.  Two 256-column accumulators alternate, so the MMAs of tile i+1
+// overlap the epilogue of tile i; the epilogue (exp2 + reciprocal per sigmoid on the
+// special-function unit) is the longer of the two.
+//
+// Every mbarrier wait is bounded: when a wait runs out the CTA records it in the status word,
+// stops issuing work, drains what it has in flight and exits with its TMEM released.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
 #include "gsa_common.cuh"
+
 namespace gsa {
-bool indexer_tc_supported(const gsa_params_t&) { return false; }
-cudaError_t launch_indexer_tc(const gsa_params_t&, RowRange, const __nv_bfloat16*, const __nv_bfloat16*,
-                              const float*, const float*, float*, int64_t, int32_t*, cudaStream_t) {
-    return cudaErrorNotSupported;
+
+namespace {
+
+constexpr int kTileKeys = 128;
+constexpr int kNCols = 256;            // N of one MMA = (queries x heads) of a group
+constexpr int kStages = 6;
+constexpr int kThreads = 320;          // 10 warps
+constexpr int kEpiWarps = 8;
+constexpr uint32_t kSpinLimit = 1u << 24;       // polls
+constexpr long long kSpinCycles = 1ll << 31;     // ~1 s of SM clock: no wait may last longer
+
+struct TcArgs {
+    const float* w;
+    const float* bI;
+    float* scores;
+    int64_t row_stride;
+    int32_t* dev_status;
+    RowRange rr;
+    int32_t Lq, Lk;
+    int32_t groups_per_batch;
+    int32_t tiles_per_cta;
+};
+
+template <int DI>
+struct SmemPlan {
+    static constexpr int Q_BYTES = kNCols * DI * 2;
+    static constexpr int K_BYTES = kTileKeys * DI * 2;
+    static constexpr int OFF_Q = 0;
+    static constexpr int OFF_K = OFF_Q + Q_BYTES;
+    static constexpr int OFF_W = OFF_K + kStages * K_BYTES;
+    static constexpr int OFF_B = OFF_W + kNCols * 4;
+    static constexpr int OFF_BAR = OFF_B + 64;                    // 8-byte aligned
+    static constexpr int N_BARS = 2 * kStages + 1 + 4;
+    static constexpr int OFF_TMEM = OFF_BAR + N_BARS * 8;
+    static constexpr int OFF_ABORT = OFF_TMEM + 8;
+    static constexpr int TOTAL = OFF_ABORT + 8;
+    static constexpr int ALLOC = TOTAL + 1024;                    // slack to align the base to 1024
+};
+
+// ---- PTX wrappers ------------------------------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// bounded wait; returns false if it gave up (and raises the CTA's abort flag)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t_start = clock64();
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 63u) {
+            if (*abort_flag) return false;
+            if (clock64() - t_start > kSpinCycles) break;
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+// waits for the outstanding tcgen05.ld; the registers are listed as in/out operands so that no
+// use of them can be scheduled ahead of the wait
+__device__ __forceinline__ void tc_wait_ld(uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.wait::ld.sync.aligned;"
+        : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+          "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+          "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+          "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+        :
+        : "memory");
+}
+
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float rcp_approx(float x) {
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// sum_j w_j * sigmoid(x_j + b_j) over HI heads, with one reciprocal per group of up to four heads:
+//   w1/a1 + w2/a2 = (w1 a2 + w2 a1) / (a1 a2),   a_j = 1 + 2^(-(x_j + b_j) log2 e).
+// The exponent is clamped at 28 (sigmoid < 4e-9 there), so a product of four a_j stays below
+// 2^116 and cannot overflow.  nb[j] = -b_j log2 e.
+template <int HI>
+__device__ __forceinline__ float gated_head_sum(const uint32_t* x, const float* w, const float (&nb)[HI]) {
+    float a[HI];
+#pragma unroll
+    for (int j = 0; j < HI; ++j)
+        a[j] = 1.0f + ex2_approx(fminf(fmaf(__uint_as_float(x[j]), -1.4426950408889634f, nb[j]), 28.0f));
+    float acc = 0.f;
+    if constexpr (HI >= 4) {
+#pragma unroll
+        for (int g = 0; g < HI; g += 4) {
+            const float n01 = fmaf(w[g], a[g + 1], w[g + 1] * a[g]), d01 = a[g] * a[g + 1];
+            const float n23 = fmaf(w[g + 2], a[g + 3], w[g + 3] * a[g + 2]), d23 = a[g + 2] * a[g + 3];
+            const float num = fmaf(n01, d23, n23 * d01);
+            acc = fmaf(num, rcp_approx(d01 * d23), acc);
+        }
+    } else if constexpr (HI == 2) {
+        acc = fmaf(w[0], a[1], w[1] * a[0]) * rcp_approx(a[0] * a[1]);
+    } else {
+        acc = w[0] * rcp_approx(a[0]);
+    }
+    return acc;
+}
+
+// shared-memory matrix descriptor, K-major operand whose rows are one swizzle span wide
+// (128 B rows: 128-byte swizzle; 64 B rows: 64-byte swizzle); 8-row groups are contiguous.
+template <int ROW_BYTES>
+__device__ __forceinline__ uint64_t make_kmajor_desc(uint32_t smem_addr) {
+    constexpr uint64_t layout = ROW_BYTES == 128 ? 2ull : 4ull;       // SWIZZLE_128B : SWIZZLE_64B
+    constexpr uint64_t sbo = (8 * ROW_BYTES) >> 4;                     // bytes between 8-row groups, /16
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);                      // start address
+    d |= 1ull << 16;                                                   // leading byte offset (unused) = 1
+    d |= sbo << 32;                                                    // stride byte offset
+    d |= 1ull << 46;                                                   // descriptor version (sm_100)
+    d |= layout << 61;
+    return d;
+}
+
+// instruction descriptor: D fp32, A = B = bf16, both K-major, M = 128, N = 256
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kNCols >> 3) << 17) |
+                            ((uint32_t)(kTileKeys >> 4) << 24);
+
+template <int DI, int HI>
+__global__ void __launch_bounds__(kThreads, 1)
+gsa_indexer_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
+                      const TcArgs a) {
+    using P = SmemPlan<DI>;
+    constexpr int NQ = kNCols / HI;             // queries per group
+    constexpr int KSTEPS = DI / 16;
+    constexpr int ROW_BYTES = DI * 2;
+
+    // ---- which work is mine ------------------------------------------------------------------
+    const int g = (int)gridDim.y - 1 - (int)blockIdx.y;               // heavy (late) groups first
+    const int bl = g / a.groups_per_batch;
+    const int tr0 = (g % a.groups_per_batch) * NQ;
+    const int nq = min(NQ, a.rr.R - tr0);
+    const int b = a.rr.b0 + bl;
+    const int t0 = a.rr.q_begin + tr0;
+    const int off = a.Lk - a.Lq;
+    const int n_vis_last = off + t0 + nq;                             // visible keys of the group's last query
+    const int tiles_group = (n_vis_last + kTileKeys - 1) / kTileKeys;
+    const int tile0 = blockIdx.x * a.tiles_per_cta;
+    const int ntiles = min(a.tiles_per_cta, tiles_group - tile0);
+    if (ntiles <= 0) return;                                          // whole CTA, before any barrier
+    if (*reinterpret_cast<volatile int32_t*>(a.dev_status) != kDevOk) return;   // an earlier CTA gave up
+
+    extern __shared__ unsigned char dyn_smem_raw[];
+    const uint32_t raw_u32 = smem_u32(dyn_smem_raw);
+    const uint32_t pad = (1024u - (raw_u32 & 1023u)) & 1023u;
+    unsigned char* smem = dyn_smem_raw + pad;
+    const uint32_t sbase = raw_u32 + pad;
+
+    float* s_w = reinterpret_cast<float*>(smem + P::OFF_W);
+    float* s_b = reinterpret_cast<float*>(smem + P::OFF_B);
+    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + P::OFF_TMEM);
+    volatile int* s_abort = reinterpret_cast<volatile int*>(smem + P::OFF_ABORT);
+    const uint32_t bar0 = sbase + P::OFF_BAR;
+    auto bar_full = [&](int s) { return bar0 + 8u * s; };
+    auto bar_empty = [&](int s) { return bar0 + 8u * (kStages + s); };
+    const uint32_t bar_q = bar0 + 8u * (2 * kStages);
+    auto bar_tfull = [&](int i) { return bar0 + 8u * (2 * kStages + 1 + i); };
+    auto bar_tempty = [&](int i) { return bar0 + 8u * (2 * kStages + 3 + i); };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
+        mbar_init(bar_q, 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull(i), 1); mbar_init(bar_tempty(i), kEpiWarps); }
+        *s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(sbase + P::OFF_TMEM)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (warp >= 2) {
+        const int e = threadIdx.x - 64;                               // 0..255 = (query, head) column
+        const int qi = e / HI, j = e % HI;
+        s_w[e] = qi < nq ? a.w[((size_t)b * a.Lq + t0 + qi) * HI + j] : 0.f;
+        if (e < 8) s_b[e] = (a.bI && e < HI) ? a.bI[e] : 0.f;
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *s_tmem;
+
+    if (warp == 0) {
+        // ================= TMA producer =======================================================
+        if (lane == 0) {
+            mbar_expect_tx(bar_q, P::Q_BYTES);
+            tma_load_2d(sbase + P::OFF_Q, &tm_q, 0, (b * a.Lq + t0) * HI, bar_q);
+            int issued = 0;
+            for (int i = 0; i < ntiles; ++i) {
+                const int s = i % kStages;
+                if (!mbar_wait(bar_empty(s), ((i / kStages) & 1) ^ 1, s_abort)) break;
+                mbar_expect_tx(bar_full(s), P::K_BYTES);
+                tma_load_2d(sbase + P::OFF_K + s * P::K_BYTES, &tm_k, 0, b * a.Lk + (tile0 + i) * kTileKeys,
+                            bar_full(s));
+                issued = i + 1;
+            }
+            if (*s_abort) {
+                // drain: wait (bounded) for the copies still in flight before the CTA may exit
+                atomicExch(a.dev_status, kDevTimeoutTma);
+                for (int i = max(0, issued - kStages); i < issued; ++i) {
+                    const uint32_t bar = bar_full(i % kStages), par = (i / kStages) & 1;
+                    for (uint32_t it = 0; it < (1u << 20) && !mbar_try_wait(bar, par); ++it) {}
+                }
+                for (uint32_t it = 0; it < (1u << 20) && !mbar_try_wait(bar_q, 0); ++it) {}
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =========================================================
+        if (lane == 0) {
+            bool ok = mbar_wait(bar_q, 0, s_abort);
+            const uint64_t bdesc = make_kmajor_desc<ROW_BYTES>(sbase + P::OFF_Q);
+            for (int i = 0; ok && i < ntiles; ++i) {
+                const int s = i % kStages, buf = i & 1;
+                if (!mbar_wait(bar_tempty(buf), ((i >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
+                if (!mbar_wait(bar_full(s), (i / kStages) & 1, s_abort)) { ok = false; break; }
+                tc_fence_after();
+                const uint64_t adesc = make_kmajor_desc<ROW_BYTES>(sbase + P::OFF_K + s * P::K_BYTES);
+#pragma unroll
+                for (int k = 0; k < KSTEPS; ++k)           // 16 K-elements = 32 bytes = 2 descriptor units
+                    tc_mma_bf16(tmem_base + buf * kNCols, adesc + 2 * k, bdesc + 2 * k, kIdesc, k > 0);
+                tc_commit(bar_empty(s));                   // stage reusable once these MMAs have read it
+                tc_commit(bar_tfull(buf));                 // accumulator ready for the epilogue
+            }
+            if (!ok) atomicExch(a.dev_status, kDevTimeoutMma);
+        }
+    } else {
+        // ================= epilogue: sigmoid, head weights, head sum, store ===================
+        const int ew = warp - 2;
+        const int quad = warp & 3;                          // TMEM lanes this warp may touch: 32*quad ..
+        const int half = ew >> 2;                           // which 128 of the 256 columns
+        constexpr int QPC = 32 / HI;                        // queries per 32-column chunk
+        float bias[HI];
+#pragma unroll
+        for (int j = 0; j < HI; ++j) bias[j] = s_b[j] * -1.4426950408889634f;
+        for (int i = 0; i < ntiles; ++i) {
+            const int buf = i & 1;
+            if (!mbar_wait(bar_tfull(buf), (i >> 1) & 1, s_abort)) {
+                if (lane == 0) atomicExch(a.dev_status, kDevTimeoutEpi);
+                break;
+            }
+            tc_fence_after();
+            const int s = (tile0 + i) * kTileKeys + quad * 32 + lane;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * kNCols + half * 128;
+            // columns are read 32 at a time, the next chunk's load in flight behind the current
+            // chunk's arithmetic
+            float* const out_col = a.scores + ((int64_t)bl * a.rr.R + tr0) * a.row_stride + s;
+            auto do_chunk = [&](const uint32_t (&r)[32], int c) {
+                const int q_first = (half * 128 + c * 32) / HI;
+#pragma unroll
+                for (int qq = 0; qq < QPC; ++qq) {
+                    const int qi = q_first + qq;
+                    float wv[HI];
+                    if constexpr (HI >= 4) {
+#pragma unroll
+                        for (int j = 0; j < HI; j += 4) {
+                            const float4 v = *reinterpret_cast<const float4*>(s_w + qi * HI + j);
+                            wv[j] = v.x; wv[j + 1] = v.y; wv[j + 2] = v.z; wv[j + 3] = v.w;
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < HI; ++j) wv[j] = s_w[qi * HI + j];
+                    }
+                    const float acc = gated_head_sum<HI>(&r[qq * HI], wv, bias);
+                    if (qi < nq && s <= off + t0 + qi) out_col[(int64_t)qi * a.row_stride] = acc;
+                }
+            };
+            uint32_t ra[32], rb[32];
+            tc_ld32(taddr, ra);
+            tc_wait_ld(ra);
+            tc_ld32(taddr + 32, rb);
+            do_chunk(ra, 0);
+            tc_wait_ld(rb);
+            tc_ld32(taddr + 64, ra);
+            do_chunk(rb, 1);
+            tc_wait_ld(ra);
+            tc_ld32(taddr + 96, rb);
+            do_chunk(ra, 2);
+            tc_wait_ld(rb);
+            do_chunk(rb, 3);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_tempty(buf));
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+    }
+}
+
+PFN_cuTensorMapEncodeTiled_v12000 get_encode_fn() {
+    static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(p);
+    }
+    return fn;
+}
+
+// rows x DI bf16, row-major; box = box_rows x DI; swizzle = one row wide
+bool make_rows_tmap(CUtensorMap* tm, const void* base, uint64_t rows, int DI, uint32_t box_rows) {
+    auto fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)DI, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)DI * 2};
+    cuuint32_t box[2] = {(cuuint32_t)DI, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    const CUtensorMapSwizzle sw = DI == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int DI, int HI>
+cudaError_t launch_t(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* qI, const __nv_bfloat16* kI,
+                     const float* w, const float* bI, float* scores, int64_t row_stride, int32_t* dev_status,
+                     cudaStream_t st) {
+    using P = SmemPlan<DI>;
+    constexpr int NQ = kNCols / HI;
+    CUtensorMap tm_k, tm_q;
+    if (!make_rows_tmap(&tm_k, kI, (uint64_t)p.B * p.Lk, DI, kTileKeys)) return cudaErrorUnknown;
+    if (!make_rows_tmap(&tm_q, qI, (uint64_t)p.B * p.Lq * HI, DI, kNCols)) return cudaErrorUnknown;
+
+    TcArgs a;
+    a.w = w; a.bI = bI; a.scores = scores; a.row_stride = row_stride; a.dev_status = dev_status;
+    a.rr = rr; a.Lq = p.Lq; a.Lk = p.Lk;
+    a.groups_per_batch = (rr.R + NQ - 1) / NQ;
+    const int groups = rr.nb * a.groups_per_batch;
+    const int n_vis_max = p.Lk - p.Lq + rr.q_begin + rr.R;
+    const int tiles_max = (n_vis_max + kTileKeys - 1) / kTileKeys;
+    // enough CTAs to fill the GPU a few times over, but runs long enough to amortise the q^I load
+    int64_t total_tiles = (int64_t)groups * tiles_max;
+    int tpc = (int)(total_tiles / (148 * 4));
+    tpc = tpc < 4 ? 4 : (tpc > 64 ? 64 : tpc);
+    a.tiles_per_cta = tpc;
+    dim3 grid((tiles_max + tpc - 1) / tpc, groups);
+
+    // one CTA per SM: the kernel allocates all 512 TMEM columns, so a second resident CTA would
+    // only sit in tcgen05.alloc until the first one leaves
+    constexpr int kSmem = P::ALLOC > 120 * 1024 ? P::ALLOC : 120 * 1024;
+    auto kern = gsa_indexer_tc_kernel<DI, HI>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, kThreads, kSmem, st>>>(tm_k, tm_q, a);
+    ++g_launches;
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+bool indexer_tc_supported(const gsa_params_t& p) {
+    if (!(p.dI == 64 || p.dI == 32)) return false;
+    if (!(p.HI == 1 || p.HI == 2 || p.HI == 4 || p.HI == 8)) return false;
+    if ((int64_t)p.B * p.Lq * p.HI >= (1ll << 31) || (int64_t)p.B * p.Lk >= (1ll << 31)) return false;
+    return get_encode_fn() != nullptr;
+}
+
+cudaError_t launch_indexer_tc(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* qI,
+                              const __nv_bfloat16* kI, const float* w, const float* bI, float* scores,
+                              int64_t row_stride, int32_t* dev_status, cudaStream_t st) {
+    if (rr.rows() <= 0) return cudaSuccess;
+#define GSA_TC_CASE(DI_, HI_) \
+    if (p.dI == DI_ && p.HI == HI_) return launch_t<DI_, HI_>(p, rr, qI, kI, w, bI, scores, row_stride, dev_status, st)
+    GSA_TC_CASE(64, 8); GSA_TC_CASE(64, 4); GSA_TC_CASE(64, 2); GSA_TC_CASE(64, 1);
+    GSA_TC_CASE(32, 8); GSA_TC_CASE(32, 4); GSA_TC_CASE(32, 2); GSA_TC_CASE(32, 1);
+#undef GSA_TC_CASE
+    return cudaErrorInvalidValue;
+}
+
 }  // namespace gsa

@@ -1,18 +1,17 @@
 // Adaptive sparsity controller: per query row, the variance of the visible scores (Eq. 8),
 // the budget k_t, and the exact top-k_t positions (Eq. 4) by radix select.
 //
-// One CTA per row.  The fp32 row is staged in shared memory when it fits (one read of
-// global memory); longer rows are re-read from global memory, where the forward pass keeps
-// the current slab of rows L2-resident.  Passes over the row:
-//   A   fp64 sum / sum of squares (second pass for the centred sum when the row is staged),
-//       min and max of the order-preserving integer key
-//   B*  histogram of (key - lo) >> shift over the live key range [lo, hi], 4096 bins; the
-//       bin holding the k-th largest key becomes the next range.  At most three rounds
-//       (32 key bits / 12 bits per round); two when the row spans at most two binades.
-//   C   per-warp counts of keys above / equal to the threshold T over contiguous segments
-//   D   ordered emission: keys > T, and the first (k - #greater) keys == T by position,
-//       written in ascending position order.
-// Ties therefore go to the lower position, and the output is unique.
+// One CTA per row; two reads of the row (one when it fits in shared memory):
+//   0  a small contiguous-chunk sample of the row fixes the key range the histogram resolves
+//   1  full read: fp64 sum and sum of squares (a centred second pass when the row is staged in
+//      shared memory), and a 4096-bin histogram of the order-preserving integer key
+//      -> Var, k_t, the bin b holding the k_t-th largest key, the count above it
+//   2  full read: every position whose bin is >= b is appended, in position order, to a list in
+//      shared memory (k_t "sure" entries at most, plus the candidates of bin b)
+//   3  on chip: radix rounds over the candidates give the exact threshold key T and how many keys
+//      equal to T are taken; one ordered compaction of the list writes S_t ascending.
+// Equal keys go to the lower position, so the output is unique.  If the list would overflow
+// (degenerate rows: huge ties in bin b), the CTA falls back to radix rounds over the whole row.
 #include "gsa_common.cuh"
 
 namespace gsa {
@@ -24,6 +23,10 @@ constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kBinsLog2 = 12;
 constexpr int kBins = 1 << kBinsLog2;
 constexpr int kBinsPerThread = kBins / kSelThreads;   // 8
+constexpr int kListCap = 6144;                        // entries of the candidate list
+constexpr int kListPerThread = kListCap / kSelThreads;  // 12
+constexpr int kChunkPerThread = 8;                    // pass 2: consecutive elements per thread
+constexpr int kChunk = kSelThreads * kChunkPerThread;
 
 struct SelectArgs {
     const float* scores;
@@ -36,7 +39,6 @@ struct SelectArgs {
     int32_t Lq, Lk;
     int32_t k_base, k_min, k_max, k_mode;
     float v_bar;
-    int32_t cache_cap;    // floats of row cache in dynamic shared memory (0: none)
 };
 
 // monotone map fp32 -> uint32 (larger float <=> larger key); -0 is folded onto +0
@@ -47,11 +49,13 @@ __device__ __forceinline__ uint32_t order_key(float x) {
 
 struct SelShared {
     uint32_t hist[kBins];
+    uint32_t list_idx[kListCap];
+    uint32_t list_key[kListCap];
     double red_a[kSelWarps];
     double red_b[kSelWarps];
     uint32_t red_min[kSelWarps];
     uint32_t red_max[kSelWarps];
-    uint32_t warp_tot[kSelWarps];
+    uint32_t warp_tot[2][kSelWarps];
     uint32_t seg_gt[kSelWarps];
     uint32_t seg_eq[kSelWarps];
     uint32_t found_bin;
@@ -63,6 +67,109 @@ struct SelShared {
 template <bool CACHED>
 __device__ __forceinline__ float row_at(const float* __restrict__ grow, const float* srow, int i) {
     return CACHED ? srow[i] : __ldg(grow + i);
+}
+
+__device__ __forceinline__ void block_minmax(SelShared& sh, uint32_t& kmin, uint32_t& kmax) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        kmin = min(kmin, __shfl_xor_sync(0xFFFFFFFFu, kmin, o));
+        kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, o));
+    }
+    if (lane == 0) { sh.red_min[wid] = kmin; sh.red_max[wid] = kmax; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t mn = 0xFFFFFFFFu, mx = 0u;
+        for (int i = 0; i < kSelWarps; ++i) { mn = min(mn, sh.red_min[i]); mx = max(mx, sh.red_max[i]); }
+        sh.bc_min = mn; sh.bc_max = mx;
+    }
+    __syncthreads();
+    kmin = sh.bc_min; kmax = sh.bc_max;
+    __syncthreads();
+}
+
+// After a histogram has been filled: the bin holding the `want`-th largest entry (1 = largest) and
+// the number of entries in higher bins.  All threads get the result.
+__device__ __forceinline__ void find_bin(SelShared& sh, uint32_t want, uint32_t& bin, uint32_t& above) {
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    uint32_t mine = 0;
+#pragma unroll
+    for (int j = 0; j < kBinsPerThread; ++j) mine += sh.hist[tid * kBinsPerThread + j];
+    uint32_t suf = mine;                    // inclusive suffix over higher lanes
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_down_sync(0xFFFFFFFFu, suf, o);
+        if (lane + o < 32) suf += v;
+    }
+    if (lane == 0) sh.warp_tot[0][wid] = suf;
+    __syncthreads();
+    uint32_t above_warp = 0;
+    for (int i = wid + 1; i < kSelWarps; ++i) above_warp += sh.warp_tot[0][i];
+    const uint32_t above_mine = above_warp + suf - mine;   // entries in bins above my 8 bins
+    if (above_mine < want && want <= above_mine + mine) {
+        uint32_t acc = above_mine;
+        for (int j = kBinsPerThread - 1; j >= 0; --j) {
+            const uint32_t c = sh.hist[tid * kBinsPerThread + j];
+            if (want <= acc + c) { sh.found_bin = tid * kBinsPerThread + j; sh.found_above = acc; break; }
+            acc += c;
+        }
+    }
+    __syncthreads();
+    bin = sh.found_bin;
+    above = sh.found_above;
+    __syncthreads();
+}
+
+// Radix rounds over `count` keys fetched by `key_of(i)`: narrows [lo, hi] onto the want-th largest
+// key.  Returns T = that key, need_eq = how many keys == T belong to the top set.
+template <class KeyOf>
+__device__ __forceinline__ void radix_rounds(SelShared& sh, int count, KeyOf key_of, uint32_t lo, uint32_t hi,
+                                             uint32_t want, uint32_t& T, uint32_t& need_eq) {
+    const int tid = threadIdx.x;
+    while (true) {
+        const uint32_t span = hi - lo;          // inclusive range has span + 1 keys
+        int shift = 0;
+        while (shift < 32 && (span >> shift) >= (uint32_t)kBins) ++shift;
+        for (int i = tid; i < kBins; i += kSelThreads) sh.hist[i] = 0u;
+        __syncthreads();
+        for (int i = tid; i < count; i += kSelThreads) {
+            const uint32_t key = key_of(i);
+            if (key >= lo && key <= hi) atomicAdd(&sh.hist[(key - lo) >> shift], 1u);
+        }
+        __syncthreads();
+        uint32_t fb, fa;
+        find_bin(sh, want, fb, fa);
+        want -= fa;
+        const uint32_t nlo = lo + (fb << shift);
+        const uint32_t nhi = shift == 0 ? nlo : min(hi, nlo + ((1u << shift) - 1u));
+        lo = nlo; hi = nhi;
+        if (shift == 0) break;
+    }
+    T = lo;
+    need_eq = want;
+}
+
+// block-wide exclusive scan of one value per thread; returns the exclusive prefix and the total.
+// `slot` alternates 0/1 between consecutive calls so one barrier per call suffices.
+__device__ __forceinline__ uint32_t block_excl_scan(SelShared& sh, uint32_t v, int slot, uint32_t& total) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    uint32_t inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+        if (lane >= o) inc += u;
+    }
+    if (lane == 31) sh.warp_tot[slot][wid] = inc;
+    __syncthreads();
+    uint32_t before = 0, tot = 0;
+#pragma unroll
+    for (int i = 0; i < kSelWarps; ++i) {
+        const uint32_t t = sh.warp_tot[slot][i];
+        before += i < wid ? t : 0u;
+        tot += t;
+    }
+    total = tot;
+    return before + inc - v;
 }
 
 template <bool CACHED>
@@ -80,36 +187,76 @@ __global__ void __launch_bounds__(kSelThreads) gsa_select_kernel(const SelectArg
     const int64_t orow = a.il.row(b, t);
     int32_t* __restrict__ out_idx = a.idx + orow * a.k_max;
 
-    // ---- pass A: stage the row, fp64 moments, key range -------------------------------------
+    // ---- pass 0: key range from a sample of 32-element chunks -------------------------------
+    uint32_t smin = 0xFFFFFFFFu, smax = 0u;
+    {
+        const int chunks = (n + 31) >> 5;
+        const int step = max(1, chunks >> 7);                 // about 128..255 chunks
+        for (int c = wid * step; c < chunks; c += kSelWarps * step) {
+            const int i = (c << 5) + lane;
+            if (i < n) {
+                const uint32_t k = order_key(__ldg(grow + i));
+                smin = min(smin, k);
+                smax = max(smax, k);
+            }
+        }
+        block_minmax(sh, smin, smax);
+    }
+    // histogram range: the sampled range widened below by a quarter and above by once its span;
+    // bin 0 collects keys below it, bin kBins-1 keys above it.
+    uint32_t h_lo, h_hi;
+    int h_shift = 0;
+    {
+        const uint32_t span = smax - smin;
+        h_lo = smin - min(smin, span >> 2);
+        h_hi = smax + min(0xFFFFFFFFu - smax, span);
+        const uint32_t hspan = h_hi - h_lo;
+        while (h_shift < 32 && (hspan >> h_shift) >= (uint32_t)(kBins - 2)) ++h_shift;
+    }
+    auto bin_of = [&](uint32_t key) -> uint32_t {
+        return key < h_lo ? 0u : (key > h_hi ? (uint32_t)(kBins - 1) : 1u + ((key - h_lo) >> h_shift));
+    };
+
+    // ---- pass 1: fp64 moments + histogram (and staging) -------------------------------------
+    for (int i = tid; i < kBins; i += kSelThreads) sh.hist[i] = 0u;
+    __syncthreads();
     double s1 = 0.0, s2 = 0.0;
-    uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
-    for (int i = tid; i < n; i += kSelThreads) {
-        const float x = __ldg(grow + i);
-        if (CACHED) srow[i] = x;
-        const double xd = (double)x;
-        s1 += xd;
-        if (!CACHED) s2 += xd * xd;
-        const uint32_t k = order_key(x);
-        kmin = min(kmin, k);
-        kmax = max(kmax, k);
+    {
+        const int n4 = n >> 2;
+        const float4* __restrict__ g4 = reinterpret_cast<const float4*>(grow);
+        for (int i = tid; i < n4; i += kSelThreads) {
+            const float4 v = __ldg(g4 + i);
+            if (CACHED) reinterpret_cast<float4*>(srow)[i] = v;
+            const float xs[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const double xd = (double)xs[e];
+                s1 += xd;
+                if (!CACHED) s2 = fma(xd, xd, s2);
+                atomicAdd(&sh.hist[bin_of(order_key(xs[e]))], 1u);
+            }
+        }
+        const int i = (n4 << 2) + tid;
+        if (i < n) {
+            const float x = __ldg(grow + i);
+            if (CACHED) srow[i] = x;
+            const double xd = (double)x;
+            s1 += xd;
+            if (!CACHED) s2 = fma(xd, xd, s2);
+            atomicAdd(&sh.hist[bin_of(order_key(x))], 1u);
+        }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         s1 += __shfl_xor_sync(0xFFFFFFFFu, s1, o);
         s2 += __shfl_xor_sync(0xFFFFFFFFu, s2, o);
-        kmin = min(kmin, __shfl_xor_sync(0xFFFFFFFFu, kmin, o));
-        kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, o));
     }
-    if (lane == 0) { sh.red_a[wid] = s1; sh.red_b[wid] = s2; sh.red_min[wid] = kmin; sh.red_max[wid] = kmax; }
+    if (lane == 0) { sh.red_a[wid] = s1; sh.red_b[wid] = s2; }
     __syncthreads();
     if (tid == 0) {
         double ta = 0.0, tb = 0.0;
-        uint32_t mn = 0xFFFFFFFFu, mx = 0u;
-        for (int i = 0; i < kSelWarps; ++i) {
-            ta += sh.red_a[i]; tb += sh.red_b[i];
-            mn = min(mn, sh.red_min[i]); mx = max(mx, sh.red_max[i]);
-        }
-        sh.bc_a = ta; sh.bc_b = tb; sh.bc_min = mn; sh.bc_max = mx;
+        for (int i = 0; i < kSelWarps; ++i) { ta += sh.red_a[i]; tb += sh.red_b[i]; }
+        sh.bc_a = ta; sh.bc_b = tb;
     }
     __syncthreads();
     const double mean = sh.bc_a / (double)n;
@@ -118,7 +265,7 @@ __global__ void __launch_bounds__(kSelThreads) gsa_select_kernel(const SelectArg
         double c2 = 0.0;
         for (int i = tid; i < n; i += kSelThreads) {
             const double dlt = (double)srow[i] - mean;
-            c2 += dlt * dlt;
+            c2 = fma(dlt, dlt, c2);
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) c2 += __shfl_xor_sync(0xFFFFFFFFu, c2, o);
@@ -154,90 +301,132 @@ __global__ void __launch_bounds__(kSelThreads) gsa_select_kernel(const SelectArg
         return;
     }
 
-    // ---- passes B: narrow [lo, hi] onto the k-th largest key ---------------------------------
-    uint32_t lo = sh.bc_min, hi = sh.bc_max;
-    uint32_t want = (uint32_t)k;                // rank (1 = largest) wanted inside [lo, hi]
-    uint32_t n_above = 0;                       // keys > hi
-    while (true) {
-        const uint32_t span = hi - lo;          // inclusive range has span + 1 keys
-        int shift = 0;
-        while (shift < 32 && (span >> shift) >= (uint32_t)kBins) ++shift;
-        for (int i = tid; i < kBins; i += kSelThreads) sh.hist[i] = 0u;
-        __syncthreads();
-        for (int i = tid; i < n; i += kSelThreads) {
-            const uint32_t key = order_key(row_at<CACHED>(grow, srow, i));
-            if (key >= lo && key <= hi) atomicAdd(&sh.hist[(key - lo) >> shift], 1u);
-        }
-        __syncthreads();
-        // thread `tid` owns bins [8 tid, 8 tid + 8); suffix sums from the top bin down
-        uint32_t mine = 0;
-#pragma unroll
-        for (int j = 0; j < kBinsPerThread; ++j) mine += sh.hist[tid * kBinsPerThread + j];
-        uint32_t suf = mine;                    // inclusive suffix over higher lanes
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t v = __shfl_down_sync(0xFFFFFFFFu, suf, o);
-            if (lane + o < 32) suf += v;
-        }
-        if (lane == 0) sh.warp_tot[wid] = suf;
-        __syncthreads();
-        uint32_t above_warp = 0;
-        for (int i = wid + 1; i < kSelWarps; ++i) above_warp += sh.warp_tot[i];
-        const uint32_t above_mine = above_warp + suf - mine;   // keys in bins above my 8 bins
-        if (above_mine < want && want <= above_mine + mine) {
-            uint32_t acc = above_mine;
-            for (int j = kBinsPerThread - 1; j >= 0; --j) {
-                const uint32_t c = sh.hist[tid * kBinsPerThread + j];
-                if (want <= acc + c) { sh.found_bin = tid * kBinsPerThread + j; sh.found_above = acc; break; }
-                acc += c;
-            }
-        }
-        __syncthreads();
-        const uint32_t fb = sh.found_bin, fa = sh.found_above;
-        n_above += fa;
-        want -= fa;
-        const uint32_t nlo = lo + (fb << shift);
-        const uint32_t nhi = shift == 0 ? nlo : min(hi, nlo + ((1u << shift) - 1u));
-        lo = nlo; hi = nhi;
-        if (shift == 0) break;
-        __syncthreads();                         // found_* are rewritten next round
-    }
-    const uint32_t T = lo;                       // the k-th largest key
-    const uint32_t need_eq = want;               // how many keys == T are taken (lowest positions)
-
-    // ---- pass C: per-warp segment counts ----------------------------------------------------
-    const int seg = ((n + kSelWarps - 1) / kSelWarps + 31) & ~31;
-    const int seg_lo = wid * seg, seg_hi = min(n, seg_lo + seg);
-    uint32_t cg = 0, ce = 0;
-    for (int i = seg_lo + lane; i < seg_hi; i += 32) {
-        const uint32_t key = order_key(row_at<CACHED>(grow, srow, i));
-        cg += key > T;
-        ce += key == T;
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        cg += __shfl_xor_sync(0xFFFFFFFFu, cg, o);
-        ce += __shfl_xor_sync(0xFFFFFFFFu, ce, o);
-    }
-    if (lane == 0) { sh.seg_gt[wid] = cg; sh.seg_eq[wid] = ce; }
+    // ---- the bin of the k-th largest key ----------------------------------------------------
+    uint32_t b1, n_above;
+    find_bin(sh, (uint32_t)k, b1, n_above);
+    const uint32_t c1 = sh.hist[b1];
     __syncthreads();
-    uint32_t run_gt = 0, run_eq = 0;
-    for (int i = 0; i < wid; ++i) { run_gt += sh.seg_gt[i]; run_eq += sh.seg_eq[i]; }
 
-    // ---- pass D: ordered emission -----------------------------------------------------------
-    const uint32_t lt_mask = (1u << lane) - 1u;
-    for (int base = seg_lo; base < seg_hi; base += 32) {
-        const int i = base + lane;
-        uint32_t key = 0;
-        const bool in = i < seg_hi;
-        if (in) key = order_key(row_at<CACHED>(grow, srow, i));
-        const bool gt = in && key > T, eq = in && key == T;
-        const uint32_t bg = __ballot_sync(0xFFFFFFFFu, gt), be = __ballot_sync(0xFFFFFFFFu, eq);
-        const uint32_t g_before = run_gt + __popc(bg & lt_mask);
-        const uint32_t e_before = run_eq + __popc(be & lt_mask);
-        if (gt || (eq && e_before < need_eq)) out_idx[g_before + min(e_before, need_eq)] = i;
-        run_gt += __popc(bg);
-        run_eq += __popc(be);
+    uint32_t T, need_eq;
+    if (n_above + c1 <= (uint32_t)kListCap) {
+        // ---- pass 2: ordered list of every position with bin >= b1 --------------------------
+        uint32_t base = 0;
+        int slot = 0;
+        for (int c0 = 0; c0 < n; c0 += kChunk, slot ^= 1) {
+            const int i0 = c0 + tid * kChunkPerThread;
+            uint32_t keys[kChunkPerThread];
+            uint32_t flags = 0;
+            if (i0 + kChunkPerThread <= n) {
+                float xs[kChunkPerThread];
+                if (CACHED) {
+                    const float4 v0 = *reinterpret_cast<const float4*>(srow + i0);
+                    const float4 v1 = *reinterpret_cast<const float4*>(srow + i0 + 4);
+                    xs[0] = v0.x; xs[1] = v0.y; xs[2] = v0.z; xs[3] = v0.w;
+                    xs[4] = v1.x; xs[5] = v1.y; xs[6] = v1.z; xs[7] = v1.w;
+                } else {
+                    const float4 v0 = __ldg(reinterpret_cast<const float4*>(grow + i0));
+                    const float4 v1 = __ldg(reinterpret_cast<const float4*>(grow + i0 + 4));
+                    xs[0] = v0.x; xs[1] = v0.y; xs[2] = v0.z; xs[3] = v0.w;
+                    xs[4] = v1.x; xs[5] = v1.y; xs[6] = v1.z; xs[7] = v1.w;
+                }
+#pragma unroll
+                for (int e = 0; e < kChunkPerThread; ++e) {
+                    keys[e] = order_key(xs[e]);
+                    flags |= (bin_of(keys[e]) >= b1 ? 1u : 0u) << e;
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < kChunkPerThread; ++e) {
+                    keys[e] = 0u;
+                    if (i0 + e < n) {
+                        keys[e] = order_key(row_at<CACHED>(grow, srow, i0 + e));
+                        flags |= (bin_of(keys[e]) >= b1 ? 1u : 0u) << e;
+                    }
+                }
+            }
+            uint32_t total;
+            uint32_t pos = base + block_excl_scan(sh, __popc(flags), slot, total);
+#pragma unroll
+            for (int e = 0; e < kChunkPerThread; ++e)
+                if (flags & (1u << e)) {
+                    sh.list_idx[pos] = (uint32_t)(i0 + e);
+                    sh.list_key[pos] = keys[e];
+                    ++pos;
+                }
+            base += total;
+        }
+        __syncthreads();
+        const int m = (int)base;                               // == n_above + c1
+
+        // ---- exact threshold among the candidates of bin b1 ---------------------------------
+        uint32_t cmin = 0xFFFFFFFFu, cmax = 0u;
+        for (int i = tid; i < m; i += kSelThreads) {
+            const uint32_t key = sh.list_key[i];
+            if (bin_of(key) == b1) { cmin = min(cmin, key); cmax = max(cmax, key); }
+        }
+        block_minmax(sh, cmin, cmax);
+        radix_rounds(sh, m, [&](int i) { return sh.list_key[i]; }, cmin, cmax, (uint32_t)k - n_above, T, need_eq);
+
+        // ---- ordered compaction of the list into S_t ----------------------------------------
+        uint32_t gt = 0, eq = 0;
+        const int j0 = tid * kListPerThread;
+#pragma unroll
+        for (int e = 0; e < kListPerThread; ++e)
+            if (j0 + e < m) {
+                const uint32_t key = sh.list_key[j0 + e];
+                gt += key > T;
+                eq += key == T;
+            }
+        uint32_t total;
+        const uint32_t packed = block_excl_scan(sh, (eq << 16) | gt, 0, total);
+        uint32_t g_before = packed & 0xFFFFu, e_before = packed >> 16;
+#pragma unroll
+        for (int e = 0; e < kListPerThread; ++e)
+            if (j0 + e < m) {
+                const uint32_t key = sh.list_key[j0 + e];
+                if (key > T) {
+                    out_idx[g_before + min(e_before, need_eq)] = (int32_t)sh.list_idx[j0 + e];
+                    ++g_before;
+                } else if (key == T) {
+                    if (e_before < need_eq) out_idx[g_before + e_before] = (int32_t)sh.list_idx[j0 + e];
+                    ++e_before;
+                }
+            }
+    } else {
+        // ---- fallback: radix rounds over the whole row, then ordered emission ----------------
+        radix_rounds(sh, n, [&](int i) { return order_key(row_at<CACHED>(grow, srow, i)); }, 0u, 0xFFFFFFFFu,
+                     (uint32_t)k, T, need_eq);
+        const int seg = ((n + kSelWarps - 1) / kSelWarps + 31) & ~31;
+        const int seg_lo = min(n, wid * seg), seg_hi = min(n, seg_lo + seg);
+        uint32_t cg = 0, ce = 0;
+        for (int i = seg_lo + lane; i < seg_hi; i += 32) {
+            const uint32_t key = order_key(row_at<CACHED>(grow, srow, i));
+            cg += key > T;
+            ce += key == T;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            cg += __shfl_xor_sync(0xFFFFFFFFu, cg, o);
+            ce += __shfl_xor_sync(0xFFFFFFFFu, ce, o);
+        }
+        if (lane == 0) { sh.seg_gt[wid] = cg; sh.seg_eq[wid] = ce; }
+        __syncthreads();
+        uint32_t run_gt = 0, run_eq = 0;
+        for (int i = 0; i < wid; ++i) { run_gt += sh.seg_gt[i]; run_eq += sh.seg_eq[i]; }
+        const uint32_t lt_mask = (1u << lane) - 1u;
+        for (int base = seg_lo; base < seg_hi; base += 32) {
+            const int i = base + lane;
+            uint32_t key = 0;
+            const bool in = i < seg_hi;
+            if (in) key = order_key(row_at<CACHED>(grow, srow, i));
+            const bool gt = in && key > T, eq = in && key == T;
+            const uint32_t bg = __ballot_sync(0xFFFFFFFFu, gt), be = __ballot_sync(0xFFFFFFFFu, eq);
+            const uint32_t g_before = run_gt + __popc(bg & lt_mask);
+            const uint32_t e_before = run_eq + __popc(be & lt_mask);
+            if (gt || (eq && e_before < need_eq)) out_idx[g_before + min(e_before, need_eq)] = i;
+            run_gt += __popc(bg);
+            run_eq += __popc(be);
+        }
     }
     for (int i = k + tid; i < a.k_max; i += kSelThreads) out_idx[i] = -1;
 }
@@ -256,22 +445,18 @@ cudaError_t launch_select(const gsa_params_t& p, RowRange rr, const float* score
     const int n_max = p.Lk - p.Lq + (rr.q_begin + rr.R - 1) + 1;
     const size_t fixed = ((sizeof(SelShared) + 15) / 16) * 16;
     constexpr size_t kMaxSmem = 200 * 1024;
-    const size_t want = fixed + (size_t)n_max * sizeof(float);
+    const size_t cached = fixed + (((size_t)n_max + 3) / 4 * 4) * sizeof(float);
     cudaError_t e;
-    if (want <= kMaxSmem) {
-        a.cache_cap = n_max;
-        static bool attr_done = false;
-        if (!attr_done) {
-            e = cudaFuncSetAttribute(gsa_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)kMaxSmem);
-            if (e != cudaSuccess) return e;
-            attr_done = true;
-        }
-        gsa_select_kernel<true><<<rr.rows(), kSelThreads, want, st>>>(a);
-    } else {
-        a.cache_cap = 0;
-        gsa_select_kernel<false><<<rr.rows(), kSelThreads, fixed, st>>>(a);
+    static bool attr_done = false;
+    if (!attr_done) {
+        e = cudaFuncSetAttribute(gsa_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(gsa_select_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fixed);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
     }
+    if (cached <= kMaxSmem) gsa_select_kernel<true><<<rr.rows(), kSelThreads, cached, st>>>(a);
+    else gsa_select_kernel<false><<<rr.rows(), kSelThreads, fixed, st>>>(a);
     ++g_launches;
     return cudaGetLastError();
 }
