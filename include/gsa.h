@@ -70,7 +70,7 @@ typedef struct gsa_params {
 /*
  * Bytes of device workspace gsa_forward (and the per-stage calls) need for `p`.
  * `slab_rows` is the number of query rows whose fp32 score rows gsa_forward keeps
- * resident at a time (0 = library default, chosen so the slab stays near the L2 size).
+ * resident at a time (0 = library default: about 1 GiB of score rows, at least 32 rows).
  * Host call; writes *bytes.
  */
 int gsa_workspace_bytes(const gsa_params_t *p, int32_t slab_rows, size_t *bytes);

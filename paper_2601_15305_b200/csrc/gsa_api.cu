@@ -72,7 +72,9 @@ WsPlan plan_ws(const gsa_params_t& p, int32_t slab_rows) {
     w.row_stride = (int64_t)align_up((size_t)p.Lk, 32);
     const int64_t rows_total = (int64_t)p.B * p.Lq;
     if (slab_rows <= 0) {
-        const int64_t target = 64ll << 20;
+        // measured on B200 at L = 128K: per-slab launch and tail costs outweigh L2 residency of the
+        // slab, so the default is large (about 1 GiB of score rows)
+        const int64_t target = 1ll << 30;
         int64_t r = target / (w.row_stride * 4);
         r = r / 32 * 32;
         slab_rows = (int32_t)(r < 32 ? 32 : r);
