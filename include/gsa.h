@@ -43,7 +43,9 @@ typedef enum {
     GSA_ERR_UNSUPPORTED_SHAPE = -2,/* a shape outside the list above                         */
     GSA_ERR_WORKSPACE = -3,        /* workspace missing or smaller than gsa_workspace_bytes  */
     GSA_ERR_CUDA = -4,             /* a CUDA runtime / driver call failed                    */
-    GSA_ERR_DEVICE_TIMEOUT = -5    /* a bounded device-side wait expired (see device status) */
+    GSA_ERR_DEVICE_TIMEOUT = -5,   /* a bounded device-side wait expired (see device status) */
+    GSA_ERR_STATIC_SCRATCH = -6    /* problem larger than the built-in scratch array of the
+                                      allocation-free entry point                            */
 } gsa_status;
 
 /* Hyper-parameters (Table 1 of the paper) plus the call's geometry. */
@@ -119,6 +121,32 @@ int gsa_sparse_gated_attn_fwd(const gsa_params_t *p, const void *Q, const void *
                               const void *g1_logits, const void *g2_logits, const int32_t *idx,
                               const int32_t *kt, void *out, void *ws, size_t ws_bytes,
                               void *stream);
+
+/*
+ * gsa_sparse_gated_attn_fwd for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a deployment variant of the call above, same arithmetic, same kernels.)
+ *
+ * Who needs it: code that runs inside a fixed, pre-reserved memory budget, in a latency-critical
+ * or callback context, or under a host allocator that must not be entered from the GPU-driving
+ * thread cannot call cudaMalloc (it may block, synchronise the device, or fail) and may have no
+ * spare buffer to pass as workspace.  Here the scratch the call needs -- the gated values
+ * V' = bf16(V * sigmoid(g2)) of Eq. 9 -- lives in an array of GSA_STATIC_SCRATCH_BYTES that is part
+ * of the library image; every GPU that loads the library holds that array until the process exits.
+ * The call and everything below it allocate nothing.
+ *
+ *   Arguments as gsa_sparse_gated_attn_fwd, without ws; g2_logits must not be NULL.
+ *   Limit: B * Lk * n_kv * d_h * 2 <= GSA_STATIC_SCRATCH_BYTES (8192 cache tokens at n_kv = 8,
+ *   d_h = 128); larger problems return GSA_ERR_STATIC_SCRATCH and launch nothing.
+ *   The first call on each device looks up the array's device address (one runtime query, made with
+ *   that device current); make that first call outside of any stream capture.
+ *   All calls on one GPU share the one array: calls that may overlap on the GPU (different streams,
+ *   different host threads) race on it -- serialise them.  Each call rewrites every element it
+ *   later reads, so no contents carry over from one call to the next.
+ */
+#define GSA_STATIC_SCRATCH_BYTES (16u << 20)
+int gsa_sparse_gated_attn_fwd_static(const gsa_params_t *p, const void *Q, const void *K, const void *V,
+                                     const void *g1_logits, const void *g2_logits, const int32_t *idx,
+                                     const int32_t *kt, void *out, void *stream);
 
 /*
  * The whole forward path (pipeline of Sec. 3.2): G2, indexer, budget, top-k, sparse

@@ -20,7 +20,10 @@ EXPORTS = (
     "gsa_workspace_bytes", "gsa_indexer_scores", "gsa_adaptive_topk", "gsa_sparse_gated_attn_fwd",
     "gsa_forward", "gsa_forward_host_arena_bytes", "gsa_forward_host", "gsa_device_status",
     "gsa_launch_count", "gsa_debug_set_indexer_path", "gsa_profile_set_events", "gsa_status_string",
+    "gsa_sparse_gated_attn_fwd_static",
 )
+
+STATIC_SCRATCH_BYTES = 16 << 20     # GSA_STATIC_SCRATCH_BYTES of include/gsa.h
 
 
 class GsaError(RuntimeError):
@@ -115,6 +118,16 @@ def gsa_sparse_gated_attn_fwd(p, Q, K, V, g1, g2, idx, kt, out, ws=None, stream=
                                            _dp(g2, BF16), _dp(idx, I32), _dp(kt, I32), _dp(out, BF16), _dp(ws),
                                            ctypes.c_size_t(0 if ws is None else ws.numel() * ws.element_size()),
                                            _stream(stream)), "gsa_sparse_gated_attn_fwd")
+
+
+def gsa_sparse_gated_attn_fwd_static(p, Q, K, V, g1, g2, idx, kt, out, stream=None) -> None:
+    """Sparse gated attention with the library's built-in scratch array: nothing is allocated, so it
+    suits callers that cannot call cudaMalloc or hand over a workspace.  Problems whose gated values
+    exceed STATIC_SCRATCH_BYTES are refused; calls on one GPU must not overlap (one shared array)."""
+    _check(lib().gsa_sparse_gated_attn_fwd_static(ctypes.byref(p), _dp(Q, BF16), _dp(K, BF16), _dp(V, BF16),
+                                                  _dp(g1, BF16), _dp(g2, BF16), _dp(idx, I32), _dp(kt, I32),
+                                                  _dp(out, BF16), _stream(stream)),
+           "gsa_sparse_gated_attn_fwd_static")
 
 
 def gsa_forward(p, Q, K, V, qI, kI, w, bI, g1, g2, out, idx_out=None, kt_out=None, var_out=None, slab_rows: int = 0,

@@ -325,6 +325,7 @@ const char* gsa_status_string(int s) {
         case GSA_ERR_WORKSPACE: return "workspace missing or too small";
         case GSA_ERR_CUDA: return "CUDA error";
         case GSA_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+        case GSA_ERR_STATIC_SCRATCH: return "problem exceeds the built-in scratch array (GSA_STATIC_SCRATCH_BYTES)";
     }
     return "unknown status";
 }
