@@ -116,7 +116,13 @@ int gsa_adaptive_topk(const gsa_params_t *p, const float *scores, int64_t row_st
  *   g2_logits may be NULL: V is then taken as already gated.
  *   idx [B, R, k_max], kt [B, R] as written by gsa_adaptive_topk (R = q_end - q_begin)
  *   out [B, Lq, n_h, d_h] bf16 (rows outside q_begin..q_end untouched)
+ *   ws  workspace of at least gsa_attn_workspace_bytes(p, 0) bytes (status word, the fp32
+ *       online-softmax state that is carried between key ranges or merged across parallel
+ *       segments).  With gsa_attn_workspace_bytes(p, 1) bytes there is room for the gated values as
+ *       well and G2 runs as one streaming pre-pass when that is cheaper than gating the gathered
+ *       rows; otherwise the g2 rows are gathered with K and V.
  */
+int gsa_attn_workspace_bytes(const gsa_params_t *p, int32_t with_value_gate_prepass, size_t *bytes);
 int gsa_sparse_gated_attn_fwd(const gsa_params_t *p, const void *Q, const void *K, const void *V,
                               const void *g1_logits, const void *g2_logits, const int32_t *idx,
                               const int32_t *kt, void *out, void *ws, size_t ws_bytes,
@@ -130,20 +136,21 @@ int gsa_sparse_gated_attn_fwd(const gsa_params_t *p, const void *Q, const void *
  * or callback context, or under a host allocator that must not be entered from the GPU-driving
  * thread cannot call cudaMalloc (it may block, synchronise the device, or fail) and may have no
  * spare buffer to pass as workspace.  Here the scratch the call needs -- the gated values
- * V' = bf16(V * sigmoid(g2)) of Eq. 9 -- lives in an array of GSA_STATIC_SCRATCH_BYTES that is part
- * of the library image; every GPU that loads the library holds that array until the process exits.
+ * V' = bf16(V * sigmoid(g2)) of Eq. 9 and the attention kernels' fp32 softmax state -- lives in an
+ * array of GSA_STATIC_SCRATCH_BYTES that is part of the library image; every GPU that loads the library holds that array until the process exits.
  * The call and everything below it allocate nothing.
  *
  *   Arguments as gsa_sparse_gated_attn_fwd, without ws; g2_logits must not be NULL.
- *   Limit: B * Lk * n_kv * d_h * 2 <= GSA_STATIC_SCRATCH_BYTES (8192 cache tokens at n_kv = 8,
- *   d_h = 128); larger problems return GSA_ERR_STATIC_SCRATCH and launch nothing.
+ *   Limit: B * Lk * n_kv * d_h * 2 + (gsa_attn_workspace_bytes(p, 0) - 256) <= GSA_STATIC_SCRATCH_BYTES
+ *   (for example 8192 cache tokens and 1024 query tokens at n_kv = 8, n_h = 16, d_h = 128); larger
+ *   problems return GSA_ERR_STATIC_SCRATCH and launch nothing.
  *   The first call on each device looks up the array's device address (one runtime query, made with
  *   that device current); make that first call outside of any stream capture.
  *   All calls on one GPU share the one array: calls that may overlap on the GPU (different streams,
  *   different host threads) race on it -- serialise them.  Each call rewrites every element it
  *   later reads, so no contents carry over from one call to the next.
  */
-#define GSA_STATIC_SCRATCH_BYTES (16u << 20)
+#define GSA_STATIC_SCRATCH_BYTES (32u << 20)
 int gsa_sparse_gated_attn_fwd_static(const gsa_params_t *p, const void *Q, const void *K, const void *V,
                                      const void *g1_logits, const void *g2_logits, const int32_t *idx,
                                      const int32_t *kt, void *out, void *stream);
@@ -177,7 +184,8 @@ int gsa_forward_host(const gsa_params_t *p, const void *Q, const void *K, const 
 /*
  * Waits for `stream`, reads the device status word at the start of `ws` into
  * *status_out (host) and returns GSA_OK / GSA_ERR_DEVICE_TIMEOUT accordingly.
- * The word is cleared by every call that takes `ws`.
+ * The word is cleared by every call that takes `ws`.  ws == NULL reads the status word of
+ * gsa_sparse_gated_attn_fwd_static (it lives in the library's built-in array on the current device).
  */
 int gsa_device_status(const void *ws, void *stream, int32_t *status_out);
 
@@ -189,6 +197,13 @@ int64_t gsa_launch_count(void);
  * 1 = plain CUDA-core indexer.  Process-wide; not meant for production use.
  */
 void gsa_debug_set_indexer_path(int32_t path);
+
+/*
+ * Tuning knob: keys per key range of the sparse-attention gather (default 16384: the K and V' rows of
+ * a range then occupy 64 MB of the 126 MB L2 at n_kv * d_h = 1024).  Process-wide; the workspace size
+ * depends on it, so set it before gsa_workspace_bytes.
+ */
+void gsa_debug_set_attn_range_keys(int32_t keys);
 
 /*
  * Profiling hook: three cudaEvent_t handles (or NULL to switch off) that every following

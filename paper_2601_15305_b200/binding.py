@@ -20,10 +20,10 @@ EXPORTS = (
     "gsa_workspace_bytes", "gsa_indexer_scores", "gsa_adaptive_topk", "gsa_sparse_gated_attn_fwd",
     "gsa_forward", "gsa_forward_host_arena_bytes", "gsa_forward_host", "gsa_device_status",
     "gsa_launch_count", "gsa_debug_set_indexer_path", "gsa_profile_set_events", "gsa_status_string",
-    "gsa_sparse_gated_attn_fwd_static",
+    "gsa_sparse_gated_attn_fwd_static", "gsa_attn_workspace_bytes", "gsa_debug_set_attn_range_keys",
 )
 
-STATIC_SCRATCH_BYTES = 16 << 20     # GSA_STATIC_SCRATCH_BYTES of include/gsa.h
+STATIC_SCRATCH_BYTES = 32 << 20     # GSA_STATIC_SCRATCH_BYTES of include/gsa.h
 
 
 class GsaError(RuntimeError):
@@ -99,6 +99,17 @@ def gsa_workspace_bytes(p: gsa_params_t, slab_rows: int = 0) -> int:
     return n.value
 
 
+def gsa_attn_workspace_bytes(p: gsa_params_t, with_value_gate_prepass: bool = True) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().gsa_attn_workspace_bytes(ctypes.byref(p), ctypes.c_int32(1 if with_value_gate_prepass else 0),
+                                          ctypes.byref(n)), "gsa_attn_workspace_bytes")
+    return n.value
+
+
+def gsa_debug_set_attn_range_keys(keys: int) -> None:
+    lib().gsa_debug_set_attn_range_keys(ctypes.c_int32(keys))
+
+
 def gsa_indexer_scores(p, qI, kI, w, bI, scores, row_stride: int, ws, stream=None) -> None:
     _check(lib().gsa_indexer_scores(ctypes.byref(p), _dp(qI, BF16), _dp(kI, BF16), _dp(w, F32), _dp(bI, F32),
                                     _dp(scores, F32), ctypes.c_int64(row_stride), _dp(ws),
@@ -157,6 +168,8 @@ def gsa_forward_host(p, Q, K, V, qI, kI, w, bI, g1, g2, out, kt_out, slab_rows: 
 
 
 def gsa_device_status(ws, stream=None) -> int:
+    """Waits for the stream and returns the device status word (0 = ok) of `ws`; ws=None reads the
+    one of gsa_sparse_gated_attn_fwd_static."""
     v = ctypes.c_int32(0)
     rc = lib().gsa_device_status(_dp(ws), _stream(stream), ctypes.byref(v))
     if rc not in (0, -5):

@@ -64,7 +64,7 @@ struct WsPlan {
     int64_t row_stride;
     int32_t slab_rows;
     bool prepass;                  // Eq. 9 as a pre-pass (prefill) or inside the gather (decode)
-    size_t slab_off, vg_off, idx_off, kt_off, total;
+    size_t slab_off, vg_off, idx_off, kt_off, attn_off, total;
 };
 
 WsPlan plan_ws(const gsa_params_t& p, int32_t slab_rows) {
@@ -89,6 +89,7 @@ WsPlan plan_ws(const gsa_params_t& p, int32_t slab_rows) {
     w.vg_off = off;   off += w.prepass ? align_up((size_t)p.B * p.Lk * p.n_kv * p.d_h * 2, 256) : 0;
     w.idx_off = off;  off += align_up((size_t)rows_total * p.k_max * 4, 256);
     w.kt_off = off;   off += align_up((size_t)rows_total * 4, 256);
+    w.attn_off = off; off += align_up(attn_scratch_bytes(p), 256);
     w.total = off;
     return w;
 }
@@ -146,6 +147,21 @@ int gsa_adaptive_topk(const gsa_params_t* p, const float* scores, int64_t row_st
     return cuda_rc(launch_select(*p, rr, scores, row_stride, idx, kt, var, il, (cudaStream_t)stream));
 }
 
+// workspace of the per-stage attention call: [status][attention scratch][V' (optional)]
+static size_t attn_ws_bytes(const gsa_params_t& p, bool with_prepass) {
+    size_t n = kStatusBytes + align_up(attn_scratch_bytes(p), 256);
+    if (with_prepass) n += align_up((size_t)p.B * p.Lk * p.n_kv * p.d_h * 2, 256);
+    return n;
+}
+
+int gsa_attn_workspace_bytes(const gsa_params_t* p, int32_t with_value_gate_prepass, size_t* bytes) {
+    int rc = check_params(p);
+    if (rc) return rc;
+    if (!bytes) return GSA_ERR_INVALID_ARG;
+    *bytes = attn_ws_bytes(*p, with_value_gate_prepass != 0);
+    return GSA_OK;
+}
+
 int gsa_sparse_gated_attn_fwd(const gsa_params_t* p, const void* Q, const void* K, const void* V,
                               const void* g1_logits, const void* g2_logits, const int32_t* idx,
                               const int32_t* kt, void* out, void* ws, size_t ws_bytes, void* stream) {
@@ -157,16 +173,20 @@ int gsa_sparse_gated_attn_fwd(const gsa_params_t* p, const void* Q, const void* 
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(g1_logits) || !aligned16(out) ||
         !aligned16(idx) || (g2_logits && !aligned16(g2_logits)))
         return GSA_ERR_INVALID_ARG;
+    if (!ws || !aligned16(ws) || ws_bytes < attn_ws_bytes(*p, false)) return GSA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e0 = cudaMemsetAsync(ws, 0, kStatusBytes, st);
+    if (e0 != cudaSuccess) return cuda_rc(e0);
     IdxLayout il{0, rr.q_begin, rr.R};
+    char* wsb = (char*)ws;
+    void* scratch = wsb + kStatusBytes;
     const bf16* Vuse = (const bf16*)V;
     const bf16* g2use = (const bf16*)g2_logits;
     if (g2_logits) {
         const WsPlan wp = plan_ws(*p, 0);
-        // pre-pass when it pays and the caller gave room for V'; otherwise gate inside the gather
-        const size_t vg_bytes = (size_t)p->B * p->Lk * p->n_kv * p->d_h * 2;
-        if (wp.prepass && ws && aligned16(ws) && ws_bytes >= (size_t)kStatusBytes + vg_bytes) {
-            bf16* Vg = (bf16*)((char*)ws + kStatusBytes);
+        // pre-pass when it pays and the caller gave room for V'; otherwise gate the gathered rows
+        if (wp.prepass && ws_bytes >= attn_ws_bytes(*p, true)) {
+            bf16* Vg = (bf16*)(wsb + attn_ws_bytes(*p, false));
             cudaError_t e = launch_value_gate((const bf16*)V, (const bf16*)g2_logits, Vg,
                                               (int64_t)p->B * p->Lk * p->n_kv * p->d_h, st);
             if (e != cudaSuccess) return cuda_rc(e);
@@ -175,7 +195,7 @@ int gsa_sparse_gated_attn_fwd(const gsa_params_t* p, const void* Q, const void* 
         }
     }
     return cuda_rc(launch_sparse_attn(*p, rr, (const bf16*)Q, (const bf16*)K, Vuse, (const bf16*)g1_logits,
-                                      g2use, idx, kt, il, (bf16*)out, st));
+                                      g2use, idx, kt, il, (bf16*)out, scratch, st));
 }
 
 int gsa_forward(const gsa_params_t* p, const void* Q, const void* K, const void* V, const void* qI,
@@ -237,7 +257,7 @@ int gsa_forward(const gsa_params_t* p, const void* Q, const void* K, const void*
     if (g_prof_ev[1]) cudaEventRecord(g_prof_ev[1], st);
     RowRange all{0, p->B, 0, p->Lq};
     e = launch_sparse_attn(*p, all, (const bf16*)Q, (const bf16*)K, Vuse, (const bf16*)g1_logits, g2use, idx,
-                           kt, il, (bf16*)out, st);
+                           kt, il, (bf16*)out, wsb + wp.attn_off, st);
     if (g_prof_ev[2]) cudaEventRecord(g_prof_ev[2], st);
     return cuda_rc(e);
 }
@@ -298,7 +318,13 @@ int gsa_forward_host(const gsa_params_t* p, const void* Q, const void* K, const 
 }
 
 int gsa_device_status(const void* ws, void* stream, int32_t* status_out) {
-    if (!ws) return GSA_ERR_WORKSPACE;
+    if (!ws) {
+        // the allocation-free entry point keeps its status word in the library's built-in array
+        void* builtin = nullptr;
+        cudaError_t e = static_scratch_address(&builtin);
+        if (e != cudaSuccess) return cuda_rc(e);
+        ws = builtin;
+    }
     int32_t v = 0;
     cudaError_t e = cudaMemcpyAsync(&v, ws, sizeof(v), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
@@ -310,6 +336,8 @@ int gsa_device_status(const void* ws, void* stream, int32_t* status_out) {
 int64_t gsa_launch_count(void) { return g_launches; }
 
 void gsa_debug_set_indexer_path(int32_t path) { g_indexer_path = path; }
+
+void gsa_debug_set_attn_range_keys(int32_t keys) { set_attn_range_keys(keys); }
 
 void gsa_profile_set_events(void* ev_begin, void* ev_selected, void* ev_end) {
     g_prof_ev[0] = (cudaEvent_t)ev_begin;

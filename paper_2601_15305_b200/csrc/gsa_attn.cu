@@ -1,15 +1,37 @@
-// Sparse gated attention (Eq. 9, 11, 12, 10): one warp per (query, KV head).
+// Sparse gated attention (Eq. 9, 11, 12, 10).
 //
-// The warp gathers the selected keys' K and V' rows of its KV head (d_h bf16 = 16-byte chunks,
-// cp.async, L2-only) into a private multi-stage ring in shared memory, 16 keys per stage, and
-// runs an online-softmax loop on bf16 tensor-core MMAs (m16n8k16, fp32 accumulate):
-//     S[head, key]  = Q[head, :] . K[key, :]        rows = the G query heads of the KV group
-//     O[head, :]   += P[head, key] * V'[key, :]
-// The eight warps of a CTA cover the eight KV heads of one query, so together they fetch each
-// selected token's whole 2 KB K row and 2 KB V' row exactly once.  G2 is either applied by a
-// streaming pre-pass (V' = bf16(V * sigmoid(g2)), prefill) or inside the gather (decode, where
-// gating the whole cache would cost more than the attention); G1 is applied to the fp32
-// accumulator before the single rounding to bf16.
+// Work item = (query token, KV head, segment of the token's index set S_t); one warp per item,
+// 16 warps per CTA, items dealt to warps round-robin so that the warps of a CTA work on the same
+// two tokens.  A warp walks its segment 16 selected keys at a time:
+//
+//   K   the 16 keys' d_h-wide slices are read with 16-byte loads straight into the registers that
+//       the tensor-core MMA takes as its A operand (keys are M).  The contraction index of Q.K is
+//       d, and a sum does not care about the order of its terms, so each thread simply uses the 8
+//       consecutive d it loaded as "its" k-indices and reads Q with the same permutation: no
+//       shared memory, no shuffles.                          S^T[key, head] = K[key,:] . Q[head,:]
+//   softmax  online, per head = per column of S^T: max/sum across the 8 lanes that hold a column.
+//   P^T -> B operand: the bf16 pairs of S^T's fragment are an 8x8 matrix; one movmatrix
+//       transposes it into the B-fragment layout.
+//   V'  the 16 keys' slices arrive by 16-byte async copies in a private two-stage buffer in
+//       shared memory and are read transposed (ldmatrix.trans) as the A operand of
+//                                                          O^T[d, head] += V'^T[d, key] P^T[key, head]
+//       With heads on the N side one MMA covers all G <= 8 query heads of the KV group, so the
+//       whole tile costs d_h/16 + d_h/16 MMAs of m16n8k16.
+//   The next tile's K loads, V' copies and indices are in flight while the current tile is
+//   computed.  16 warps x (4 KB in registers + 4 KB in shared memory) per SM keep the L2 busy.
+//
+// The gather dominates: every selected (token, key) pair moves one K row and one V' row of all KV
+// heads (4 KB at the 1.7B shape).  Random 2 KB rows come at ~8 TB/s out of HBM but at 11-13 TB/s
+// out of the 126 MB L2, so for long contexts the key axis is cut into ranges whose K and V' rows
+// fit in L2 and the kernel is launched once per range, over every query's sub-list in that range
+// (index sets are ascending, so a sub-list is contiguous).  The online-softmax state (m, l, O) of a
+// (token, head) is carried from range to range in fp32 in the workspace.  For decode-sized calls
+// (few tokens) the same state slots hold the partial results of segments that run in parallel.
+// A last small kernel merges the slots, normalises, applies G1 and rounds to bf16 once.
+//
+// G2 is either applied by a streaming pre-pass (V' = bf16(V * sigmoid(g2)), prefill) or in
+// registers on the gathered rows (decode, where gating the whole cache would cost more than the
+// attention): V and g2 slices are then loaded to registers, gated, and stored to the shared tile.
 #include "gsa_common.cuh"
 
 namespace gsa {
@@ -17,202 +39,383 @@ namespace gsa {
 namespace {
 
 constexpr int kTileKeys = 16;
+constexpr int kWarpsPrefill = 16;          // warps per CTA, V' pre-gated
+constexpr int kWarpsFused = 8;             // warps per CTA when V and g2 pass through registers
+constexpr int kRangeKeysDefault = 16384;   // keys per L2 range: K + V' rows of 16K tokens = 64 MB at the 1.7B shape
+constexpr int kMaxRanges = 48;
+constexpr int kPartKeys = 256;             // decode: keys per parallel segment
+constexpr int kMaxParts = 8;
 
 struct AttnArgs {
     const __nv_bfloat16* Q;
     const __nv_bfloat16* K;
     const __nv_bfloat16* V;
-    const __nv_bfloat16* g1;
     const __nv_bfloat16* g2;
     const int32_t* idx;
     const int32_t* kt;
-    __nv_bfloat16* out;
+    const int32_t* cuts;      // range mode: [idx rows][n_cuts] positions in the index row where each range starts
+    float* state;             // [slots][idx rows][n_kv][G*(d_h+2)] fp32
     RowRange rr;
     IdxLayout il;
+    int64_t idx_rows;         // rows of the idx / kt / state tables
     int32_t Lq, Lk, n_h, n_kv, k_max;
-    int32_t q_per_cta;
-    float scale_log2;     // sm_scale * log2(e)
+    int32_t mode;             // 0: one key range per launch (range index `range`), 1: parallel parts
+    int32_t range, n_cuts;
+    float scale_log2;         // sm_scale * log2(e)
 };
 
-template <int DH, int G, bool FUSE_G2, int STAGES>
-__global__ void __launch_bounds__(256) gsa_sparse_attn_kernel(const AttnArgs a) {
-    constexpr int ROW_BYTES = DH * 2;
-    constexpr int CHUNKS = ROW_BYTES / 16;                  // 16-byte chunks per row: 8 or 16
-    constexpr int TENSORS = FUSE_G2 ? 3 : 2;
-    constexpr int TILE_BYTES = kTileKeys * ROW_BYTES;       // one tensor, one stage
-    constexpr int STAGE_BYTES = TENSORS * TILE_BYTES;
-    constexpr int KSTEPS = DH / 16;                         // QK^T k-steps
-    constexpr int NT_O = DH / 8;                            // output n-tiles
-    constexpr int ROWS_PER_IT = 32 / CHUNKS;                // key rows one warp-wide cp.async covers
-    constexpr int ITS = kTileKeys / ROWS_PER_IT;
+struct RowId { int32_t b, t; int64_t irow; };
+
+__device__ __forceinline__ RowId row_of(const RowRange& rr, const IdxLayout& il, int lr) {
+    RowId r;
+    r.b = rr.b0 + lr / rr.R;
+    r.t = rr.q_begin + lr % rr.R;
+    r.irow = il.row(r.b, r.t);
+    return r;
+}
+
+__device__ __forceinline__ uint4 ldg_stream(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+// 32 bytes per thread: a warp-wide load covers whole 128-byte lines of 8 rows
+__device__ __forceinline__ void ldg_stream32(const void* p, uint4& lo, uint4& hi) {
+    asm volatile("ld.global.nc.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(lo.x), "=r"(lo.y), "=r"(lo.z), "=r"(lo.w), "=r"(hi.x), "=r"(hi.y), "=r"(hi.z), "=r"(hi.w)
+                 : "l"(p));
+}
+__device__ __forceinline__ float ex2_fast(float x) {          // 2^x, one special-function instruction; 2^-inf = 0
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
+__device__ __forceinline__ int parts_of(int k_eff) {
+    const int p = (k_eff + kPartKeys - 1) / kPartKeys;
+    return p < 1 ? 1 : (p > kMaxParts ? kMaxParts : p);
+}
+
+template <int DH, int G, bool FUSE_G2>
+__global__ void __launch_bounds__((FUSE_G2 ? kWarpsFused : kWarpsPrefill) * 32, 1)
+gsa_sparse_attn_kernel(const AttnArgs a) {
+    constexpr int kWarpsPerCta = FUSE_G2 ? kWarpsFused : kWarpsPrefill;
+    constexpr int HEAD_BYTES = DH * 2;
+    constexpr int NC = DH / 32;                         // 32-d chunks of a head row (one uint4 per thread each)
+    constexpr int MT = DH / 16;                         // output m-tiles
+    constexpr int VSTRIDE = HEAD_BYTES + 16;            // padded row of the staged V' tile
+    constexpr int VTILE = kTileKeys * VSTRIDE;
+    constexpr int VSTAGES = FUSE_G2 ? 1 : 2;
+    constexpr int CHUNKS = HEAD_BYTES / 16;             // 16-byte chunks per head row
+    constexpr int KPI = 32 / CHUNKS;                    // keys one warp-wide 16-byte copy covers
+    constexpr int ITS = kTileKeys / KPI;
+    constexpr int STATE_F = G * (DH + 2);               // floats of one (row, KV head) state
 
     extern __shared__ __align__(128) unsigned char smem[];
-    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    const int slot = wid / a.n_kv, g = wid % a.n_kv;
-    const int lr = blockIdx.x * a.q_per_cta + slot;
-    if (slot >= a.q_per_cta || lr >= a.rr.rows()) return;   // warp-uniform; no CTA barriers below
-    const int b = a.rr.b0 + lr / a.rr.R;
-    const int t = a.rr.q_begin + lr % a.rr.R;
-    const int64_t irow = a.il.row(b, t);
-    const int32_t* __restrict__ idx_row = a.idx + irow * a.k_max;
-    const int k_eff = a.kt[irow];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int gid = lane >> 2, tig = lane & 3;
+    unsigned char* my_smem = smem + (size_t)warp * VSTAGES * VTILE;
+    const uint32_t my_s32 = smem_u32(my_smem);
+    const int n_kv = a.n_kv;
+    const int vkey = lane / CHUNKS, vch = lane % CHUNKS;
+    const bool real_head = gid < G;                     // this thread's column of Q^T is a real head
+    const bool real_cols = 2 * tig < G;                 // this thread's output columns hold real heads
 
-    unsigned char* my_smem = smem + (size_t)wid * STAGES * STAGE_BYTES;
-    const uint32_t my_smem_u32 = smem_u32(my_smem);
+    const int rows = a.rr.rows();
+    const int64_t n_items = (int64_t)rows * n_kv * (a.mode == 1 ? kMaxParts : 1);
+    const int64_t warps_total = (int64_t)gridDim.x * kWarpsPerCta;
 
-    const int qrow = lane >> 2, qcol = (lane & 3) * 2;
-    const bool real_row = qrow < G;
-    const int h = g * G + (real_row ? qrow : 0);
-    const size_t q_off = (((size_t)b * a.Lq + t) * a.n_h + h) * DH;
-
-    // Q as the A operand: rows = heads of the group (rows >= G are zero padding)
-    uint32_t qa[KSTEPS][2];
-#pragma unroll
-    for (int ks = 0; ks < KSTEPS; ++ks) {
-        qa[ks][0] = real_row ? *reinterpret_cast<const uint32_t*>(a.Q + q_off + ks * 16 + qcol) : 0u;
-        qa[ks][1] = real_row ? *reinterpret_cast<const uint32_t*>(a.Q + q_off + ks * 16 + 8 + qcol) : 0u;
-    }
-
-    const size_t kv_batch = (size_t)b * a.Lk;
-    const int my_chunk = lane % CHUNKS, my_sub = lane / CHUNKS;
-
-    auto issue_tile = [&](int tile) {
-        const int stage = tile % STAGES;
-        const int j0 = tile * kTileKeys;
-        int pos_l = 0;
-        if (lane < kTileKeys) {
-            const int j = j0 + lane;
-            pos_l = idx_row[j < k_eff ? j : 0];           // padding keys re-read a valid row; P = 0 there
+    for (int64_t item = (int64_t)blockIdx.x * kWarpsPerCta + warp; item < n_items; item += warps_total) {
+        const int g = (int)(item % n_kv);
+        int64_t rest = item / n_kv;
+        int part = 0;
+        if (a.mode == 1) { part = (int)(rest % kMaxParts); rest /= kMaxParts; }
+        const RowId r = row_of(a.rr, a.il, (int)rest);
+        const int k_eff = min(a.kt[r.irow], a.k_max);
+        int lo, hi, slot = 0;
+        if (a.mode == 0) {
+            lo = 0;
+            hi = k_eff;
+            if (a.n_cuts > 1) {
+                const int32_t* c = a.cuts + r.irow * a.n_cuts + a.range;
+                lo = c[0];
+                if (a.range + 1 < a.n_cuts) hi = c[1];
+            }
+        } else {
+            const int np = parts_of(k_eff);
+            if (part >= np) continue;
+            const int per = ((k_eff + np - 1) / np + kTileKeys - 1) / kTileKeys * kTileKeys;
+            lo = part * per;
+            hi = min(k_eff, lo + per);
+            slot = part;
         }
-        const uint32_t sbase = my_smem_u32 + stage * STAGE_BYTES;
+        const int count = hi - lo;
+        if (count <= 0 && !(a.mode == 1)) continue;
+        const int32_t* __restrict__ idx_seg = a.idx + r.irow * a.k_max + lo;
+        const int ntiles = (count + kTileKeys - 1) / kTileKeys;
+        float* __restrict__ st = a.state + (((int64_t)slot * a.idx_rows + r.irow) * n_kv + g) * STATE_F;
+
+        // ---- Q^T as the B operand, in the permuted-d order the K loads use ----------------------
+        uint4 qb[NC];     // piece c = bytes [(c/2)*128 + tig*32 + (c%2)*16, +16) of the head row
+        {
+            const int h = g * G + (real_head ? gid : 0);
+            const __nv_bfloat16* qp = a.Q + (((size_t)r.b * a.Lq + r.t) * a.n_h + h) * DH + tig * 16;
 #pragma unroll
-        for (int it = 0; it < ITS; ++it) {
-            const int r = it * ROWS_PER_IT + my_sub;
-            const int pos = __shfl_sync(0xFFFFFFFFu, pos_l, r);
-            const size_t goff = ((kv_batch + pos) * a.n_kv + g) * DH + my_chunk * 8;
-            const uint32_t soff = r * ROW_BYTES + ((my_chunk ^ (r & 7)) << 4);
-            cp_async16(sbase + soff, a.K + goff);
-            cp_async16(sbase + TILE_BYTES + soff, a.V + goff);
-            if (FUSE_G2) cp_async16(sbase + 2 * TILE_BYTES + soff, a.g2 + goff);
+            for (int c = 0; c < NC; ++c)
+                qb[c] = real_head ? *reinterpret_cast<const uint4*>(qp + (c >> 1) * 64 + (c & 1) * 8)
+                                  : make_uint4(0u, 0u, 0u, 0u);
         }
-    };
 
-    float o_acc[NT_O][4];
+        // ---- state: O^T[d, head] fragments, running max and sum per head ----------------------
+        float o[MT][4];
+        float m_run[2], l_run[2];
+        const bool carry_in = a.mode == 0 && lo > 0;
+        if (carry_in && real_cols) {
 #pragma unroll
-    for (int i = 0; i < NT_O; ++i) { o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f; }
-    float m_run = -INFINITY, l_run = 0.f;
-
-    const int ntiles = (k_eff + kTileKeys - 1) / kTileKeys;
+            for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-    for (int s = 0; s < STAGES - 1; ++s) {
-        if (s < ntiles) issue_tile(s);
-        cp_async_commit();
-    }
-
-    for (int tile = 0; tile < ntiles; ++tile) {
-        if (tile + STAGES - 1 < ntiles) issue_tile(tile + STAGES - 1);
-        cp_async_commit();
-        cp_async_wait<STAGES - 1>();
-        __syncwarp();
-        const uint32_t sbase = my_smem_u32 + (tile % STAGES) * STAGE_BYTES;
-
-        if (FUSE_G2) {       // Eq. 9 in place: V tile <- bf16(V * sigmoid(g2))
-            unsigned char* sv = my_smem + (tile % STAGES) * STAGE_BYTES + TILE_BYTES;
-            unsigned char* sg = sv + TILE_BYTES;
-#pragma unroll
-            for (int c = lane; c < kTileKeys * CHUNKS; c += 32) {
-                uint4 vv = *reinterpret_cast<uint4*>(sv + c * 16);
-                const uint4 gg = *reinterpret_cast<const uint4*>(sg + c * 16);
-                __nv_bfloat162* v2 = reinterpret_cast<__nv_bfloat162*>(&vv);
-                const __nv_bfloat162* g2v = reinterpret_cast<const __nv_bfloat162*>(&gg);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const float2 vf = __bfloat1622float2(v2[e]), gf = __bfloat1622float2(g2v[e]);
-                    v2[e] = __floats2bfloat162_rn(vf.x * fast_sigmoid(gf.x), vf.y * fast_sigmoid(gf.y));
+                for (int hf = 0; hf < 2; ++hf) {
+                    const int d = mt * 16 + hf * 8 + gid;
+                    if (G >= 2) {
+                        const float2 v = *reinterpret_cast<const float2*>(st + d * G + 2 * tig);
+                        o[mt][hf * 2] = v.x; o[mt][hf * 2 + 1] = v.y;
+                    } else {
+                        o[mt][hf * 2] = st[d]; o[mt][hf * 2 + 1] = 0.f;
+                    }
                 }
-                *reinterpret_cast<uint4*>(sv + c * 16) = vv;
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const bool ok = 2 * tig + e < G;
+                m_run[e] = ok ? st[G * DH + 2 * tig + e] : -INFINITY;
+                // every lane of a column accumulates its own share of l; the carried sum goes to one of them
+                l_run[e] = (ok && gid == 0) ? st[G * DH + G + 2 * tig + e] : 0.f;
             }
+        } else {
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) { o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f; }
+            m_run[0] = m_run[1] = -INFINITY;
+            l_run[0] = l_run[1] = 0.f;
+        }
+
+        // per-item address bases: a gathered row's address is base + position * row_bytes
+        const uint32_t row_bytes = (uint32_t)n_kv * HEAD_BYTES;
+        const size_t head0 = ((size_t)r.b * a.Lk * n_kv + g) * HEAD_BYTES;
+        const unsigned char* kbase = reinterpret_cast<const unsigned char*>(a.K) + head0 + tig * 32;
+        const unsigned char* vbase = reinterpret_cast<const unsigned char*>(a.V) + head0 + vch * 16;
+        const unsigned char* gbase = reinterpret_cast<const unsigned char*>(a.g2) + head0 + vch * 16;
+        const uint32_t vdst = my_s32 + vkey * VSTRIDE + vch * 16;
+        const int32_t pad_pos = count > 0 ? idx_seg[0] : 0;          // tail keys re-read a valid row (P = 0 there)
+        const int32_t max_pos = a.Lk - 1;
+        auto load_pos = [&](int tile) -> int32_t {
+            const int j = tile * kTileKeys + (lane & 15);
+            const int32_t p = j < count ? idx_seg[j] : pad_pos;
+            return min(max(p, 0), max_pos);                          // a corrupt index must not leave the tensor
+        };
+        uint4 kb[2 * NC];                                            // K tile = A operand fragments
+        auto issue_k = [&](int32_t pos16) {
+            const uint32_t p0 = __shfl_sync(0xFFFFFFFFu, pos16, gid), p1 = __shfl_sync(0xFFFFFFFFu, pos16, gid + 8);
+            const unsigned char* k0 = kbase + (uint64_t)p0 * row_bytes;
+            const unsigned char* k1 = kbase + (uint64_t)p1 * row_bytes;
+#pragma unroll
+            for (int c = 0; c < NC; c += 2) {
+                ldg_stream32(k0 + (c >> 1) * 128, kb[c], kb[c + 1]);
+                ldg_stream32(k1 + (c >> 1) * 128, kb[NC + c], kb[NC + c + 1]);
+            }
+        };
+        uint4 vreg[FUSE_G2 ? ITS : 1], greg[FUSE_G2 ? ITS : 1];
+        auto issue_v = [&](int32_t pos16, int stage) {
+#pragma unroll
+            for (int i = 0; i < ITS; ++i) {
+                const uint32_t p = __shfl_sync(0xFFFFFFFFu, pos16, i * KPI + vkey);
+                const uint64_t goff = (uint64_t)p * row_bytes;
+                if (FUSE_G2) {
+                    vreg[i] = ldg_stream(vbase + goff);
+                    greg[i] = ldg_stream(gbase + goff);
+                } else {
+                    cp_async16(vdst + stage * VTILE + i * KPI * VSTRIDE, vbase + goff);
+                }
+            }
+        };
+
+        int32_t pos_nxt = load_pos(1);
+        {
+            const int32_t pos0 = load_pos(0);
+            issue_v(pos0, 0);
+            cp_async_commit();
+            issue_k(pos0);
+        }
+
+        for (int tile = 0; tile < ntiles; ++tile) {
+            const int stage = FUSE_G2 ? 0 : (tile & 1);
+            const bool more = tile + 1 < ntiles;
+            if (FUSE_G2) {
+                // Eq. 9 in registers, then the gated tile goes to shared memory for the transposed read
+#pragma unroll
+                for (int i = 0; i < ITS; ++i) {
+                    uint4 vv = vreg[i];
+                    const uint4 gg = greg[i];
+                    __nv_bfloat162* v2 = reinterpret_cast<__nv_bfloat162*>(&vv);
+                    const __nv_bfloat162* g2v = reinterpret_cast<const __nv_bfloat162*>(&gg);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 vf = __bfloat1622float2(v2[e]), gf = __bfloat1622float2(g2v[e]);
+                        v2[e] = __floats2bfloat162_rn(vf.x * fast_sigmoid(gf.x), vf.y * fast_sigmoid(gf.y));
+                    }
+                    *reinterpret_cast<uint4*>(my_smem + (i * KPI + vkey) * VSTRIDE + vch * 16) = vv;
+                }
+                if (more) issue_v(pos_nxt, 0);
+            } else {
+                if (more) issue_v(pos_nxt, stage ^ 1);
+                cp_async_commit();
+            }
+
+            // ---- S^T = K Q^T : rows = 16 keys, columns = heads --------------------------------
+            float s[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int c = 0; c < NC; ++c) {
+                mma_bf16_16816(s, kb[c].x, kb[NC + c].x, kb[c].y, kb[NC + c].y, qb[c].x, qb[c].y);
+                mma_bf16_16816(s, kb[c].z, kb[NC + c].z, kb[c].w, kb[NC + c].w, qb[c].z, qb[c].w);
+            }
+            if (more) issue_k(pos_nxt);
+            pos_nxt = load_pos(tile + 2);
+
+            // ---- online softmax per head (column) ------------------------------------------------
+            const int j0 = tile * kTileKeys + gid;
+            const bool v0 = j0 < count, v1 = j0 + 8 < count;
+            float p[4];
+            float alpha[2];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const float s0 = v0 ? s[e] * a.scale_log2 : -INFINITY;
+                const float s1 = v1 ? s[2 + e] * a.scale_log2 : -INFINITY;
+                float mx = fmaxf(s0, s1);
+                mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 4));
+                mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 8));
+                mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 16));
+                const float m_new = fmaxf(m_run[e], mx);              // finite: key 0 of every tile is valid
+                alpha[e] = ex2_fast(m_run[e] - m_new);
+                m_run[e] = m_new;
+                p[e] = ex2_fast(s0 - m_new);
+                p[2 + e] = ex2_fast(s1 - m_new);
+                l_run[e] = fmaf(l_run[e], alpha[e], p[e] + p[2 + e]);
+            }
+            // the running maximum settles after a few tiles; rescale only when it moved
+            if (__any_sync(0xFFFFFFFFu, alpha[0] != 1.f || alpha[1] != 1.f)) {
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                    o[mt][0] *= alpha[0]; o[mt][1] *= alpha[1]; o[mt][2] *= alpha[0]; o[mt][3] *= alpha[1];
+                }
+            }
+            // P^T[key, head] as the B operand: transpose the two 8x8 bf16 blocks of the fragment
+            const uint32_t pb0 = movmatrix_trans(pack_bf16(p[0], p[1]));     // keys 0..7
+            const uint32_t pb1 = movmatrix_trans(pack_bf16(p[2], p[3]));     // keys 8..15
+
+            // ---- O^T += V'^T P^T -------------------------------------------------------------------
+            if (!FUSE_G2) cp_async_wait<1>();
             __syncwarp();
+            {
+                const int mi = lane >> 3;
+                const uint32_t vaddr = my_s32 + stage * VTILE + ((lane & 7) + (mi >> 1) * 8) * VSTRIDE + (mi & 1) * 16;
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                    uint32_t a0, a1, a2, a3;
+                    ldmatrix_x4_trans(a0, a1, a2, a3, vaddr + mt * 32);
+                    mma_bf16_16816(o[mt], a0, a1, a2, a3, pb0, pb1);
+                }
+            }
+            __syncwarp();                                             // the stage is rewritten two tiles on
         }
+        if (!FUSE_G2) cp_async_wait<0>();
 
-        // ---- S = Q K^T over the 16 keys of the tile (two n-tiles of 8 keys) -----------------
-        float s_acc[2][4];
+        // ---- write the state slot ---------------------------------------------------------------
 #pragma unroll
-        for (int nt = 0; nt < 2; ++nt) {
-            s_acc[nt][0] = s_acc[nt][1] = s_acc[nt][2] = s_acc[nt][3] = 0.f;
-            const int key = nt * 8 + (lane & 7);
+        for (int e = 0; e < 2; ++e) {
+            l_run[e] += __shfl_xor_sync(0xFFFFFFFFu, l_run[e], 4);
+            l_run[e] += __shfl_xor_sync(0xFFFFFFFFu, l_run[e], 8);
+            l_run[e] += __shfl_xor_sync(0xFFFFFFFFu, l_run[e], 16);
+        }
+        if (real_cols) {
 #pragma unroll
-            for (int kk = 0; kk < KSTEPS / 2; ++kk) {
-                const int chunk = kk * 4 + (lane >> 3);
-                uint32_t b0, b1, b2, b3;
-                ldmatrix_x4(b0, b1, b2, b3, sbase + key * ROW_BYTES + ((chunk ^ (key & 7)) << 4));
-                mma_bf16_16816(s_acc[nt], qa[2 * kk][0], 0u, qa[2 * kk][1], 0u, b0, b1);
-                mma_bf16_16816(s_acc[nt], qa[2 * kk + 1][0], 0u, qa[2 * kk + 1][1], 0u, b2, b3);
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    const int d = mt * 16 + hf * 8 + gid;
+                    if (G >= 2) *reinterpret_cast<float2*>(st + d * G + 2 * tig) = make_float2(o[mt][hf * 2], o[mt][hf * 2 + 1]);
+                    else st[d] = o[mt][hf * 2];
+                }
+            if (gid == 0) {
+#pragma unroll
+                for (int e = 0; e < 2; ++e)
+                    if (2 * tig + e < G) { st[G * DH + 2 * tig + e] = m_run[e]; st[G * DH + G + 2 * tig + e] = l_run[e]; }
             }
         }
-
-        // ---- online softmax on row lane/4 ---------------------------------------------------
-        const int j0 = tile * kTileKeys;
-        float p[2][2];
-        float tmax = -INFINITY;
-#pragma unroll
-        for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const int j = j0 + nt * 8 + qcol + e;
-                const float sv = j < k_eff ? s_acc[nt][e] * a.scale_log2 : -INFINITY;
-                p[nt][e] = sv;
-                tmax = fmaxf(tmax, sv);
-            }
-        tmax = fmaxf(tmax, __shfl_xor_sync(0xFFFFFFFFu, tmax, 1));
-        tmax = fmaxf(tmax, __shfl_xor_sync(0xFFFFFFFFu, tmax, 2));
-        const float m_new = fmaxf(m_run, tmax);              // finite: every tile has a valid key
-        const float alpha = exp2f(m_run - m_new);
-        m_run = m_new;
-        float psum = 0.f;
-#pragma unroll
-        for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                p[nt][e] = exp2f(p[nt][e] - m_new);
-                psum += p[nt][e];
-            }
-        l_run = l_run * alpha + psum;
-#pragma unroll
-        for (int i = 0; i < NT_O; ++i) { o_acc[i][0] *= alpha; o_acc[i][1] *= alpha; }
-
-        // ---- O += P V' ----------------------------------------------------------------------
-        const uint32_t pa0 = pack_bf16(p[0][0], p[0][1]);     // keys 0..7 of the tile
-        const uint32_t pa2 = pack_bf16(p[1][0], p[1][1]);     // keys 8..15
-        const uint32_t vbase = sbase + TILE_BYTES;
-        const int vkey = (lane & 7) + ((lane >> 3) & 1) * 8;
-#pragma unroll
-        for (int np = 0; np < NT_O / 2; ++np) {
-            const int chunk = np * 2 + (lane >> 4);
-            uint32_t b0, b1, b2, b3;
-            ldmatrix_x4_trans(b0, b1, b2, b3, vbase + vkey * ROW_BYTES + ((chunk ^ (vkey & 7)) << 4));
-            mma_bf16_16816(o_acc[2 * np], pa0, 0u, pa2, 0u, b0, b1);
-            mma_bf16_16816(o_acc[2 * np + 1], pa0, 0u, pa2, 0u, b2, b3);
-        }
-        __syncwarp();                                         // stage is refilled next iteration
     }
-    cp_async_wait<0>();
+}
 
-    // ---- normalise, G1, store ---------------------------------------------------------------
-    l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 1);
-    l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 2);
-    if (real_row) {
-        const float inv = l_run > 0.f ? 1.0f / l_run : 0.f;
-        const __nv_bfloat16* g1p = a.g1 + q_off;
-        __nv_bfloat16* op = a.out + q_off;
+// cuts[row][c] = number of selected positions of the row below c * range_keys (c = 0 .. n_cuts-1)
+__global__ void __launch_bounds__(256) gsa_range_cuts_kernel(const int32_t* __restrict__ idx, const int32_t* __restrict__ kt,
+                                                             int32_t* __restrict__ cuts, RowRange rr, IdxLayout il,
+                                                             int k_max, int n_cuts, int range_keys) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (int64_t)rr.rows() * n_cuts) return;
+    const int c = (int)(i % n_cuts);
+    const RowId r = row_of(rr, il, (int)(i / n_cuts));
+    const int32_t* __restrict__ row = idx + r.irow * k_max;
+    const int k_eff = min(kt[r.irow], k_max);
+    const int bound = c * range_keys;
+    int lo = 0, hi = k_eff;                      // first position with row[pos] >= bound
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (row[mid] < bound) lo = mid + 1; else hi = mid;
+    }
+    cuts[r.irow * n_cuts + c] = lo;
+}
+
+// merge the state slots of a (row, head): out = (sum_p 2^(m_p - M) O_p) / (sum_p 2^(m_p - M) l_p) * sigmoid(g1)
+template <int DH, int G>
+__global__ void __launch_bounds__(256) gsa_attn_finalize_kernel(const float* __restrict__ state, const int32_t* __restrict__ kt,
+                                                                const __nv_bfloat16* __restrict__ g1, __nv_bfloat16* __restrict__ out,
+                                                                RowRange rr, IdxLayout il, int64_t idx_rows, int Lq, int n_h,
+                                                                int n_kv, int k_max, int mode) {
+    constexpr int STATE_F = G * (DH + 2);
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t total = (int64_t)rr.rows() * n_kv * DH;
+    if (i >= total) return;
+    const int d = (int)(i % DH);
+    const int g = (int)((i / DH) % n_kv);
+    const RowId r = row_of(rr, il, (int)(i / ((int64_t)DH * n_kv)));
+    const int k_eff = min(kt[r.irow], k_max);
+    const int np = mode == 1 ? parts_of(k_eff) : 1;
+    float acc[G], mx[G], den[G];
 #pragma unroll
-        for (int i = 0; i < NT_O; ++i) {
-            const int d = i * 8 + qcol;
-            const float2 gl = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(g1p + d));
-            const float o0 = o_acc[i][0] * inv * fast_sigmoid(gl.x);
-            const float o1 = o_acc[i][1] * inv * fast_sigmoid(gl.y);
-            *reinterpret_cast<__nv_bfloat162*>(op + d) = __floats2bfloat162_rn(o0, o1);
+    for (int e = 0; e < G; ++e) { acc[e] = 0.f; den[e] = 0.f; mx[e] = -INFINITY; }
+    if (k_eff > 0) {
+        for (int p = 0; p < np; ++p) {
+            const float* st = state + (((int64_t)p * idx_rows + r.irow) * n_kv + g) * STATE_F;
+#pragma unroll
+            for (int e = 0; e < G; ++e) mx[e] = fmaxf(mx[e], st[G * DH + e]);
         }
+        for (int p = 0; p < np; ++p) {
+            const float* st = state + (((int64_t)p * idx_rows + r.irow) * n_kv + g) * STATE_F;
+#pragma unroll
+            for (int e = 0; e < G; ++e) {
+                const float m = st[G * DH + e];
+                const float sc = m == -INFINITY ? 0.f : exp2f(m - mx[e]);
+                acc[e] = fmaf(sc, st[d * G + e], acc[e]);
+                den[e] = fmaf(sc, st[G * DH + G + e], den[e]);
+            }
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < G; ++e) {
+        const size_t at = (((size_t)r.b * Lq + r.t) * n_h + g * G + e) * DH + d;
+        const float v = den[e] > 0.f ? acc[e] / den[e] * fast_sigmoid(__bfloat162float(g1[at])) : 0.f;
+        out[at] = __float2bfloat16_rn(v);
     }
 }
 
@@ -235,35 +438,113 @@ __global__ void __launch_bounds__(256) gsa_value_gate_kernel(const uint4* __rest
     }
 }
 
+int sm_count() {
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = 148;
+    }
+    return n;
+}
+
+int g_range_keys = kRangeKeysDefault;
+
+struct AttnPlan {
+    int mode;            // 0 ranges, 1 parts
+    int n_ranges;        // mode 0
+    int slots;
+    size_t state_bytes, cuts_bytes;
+};
+
+AttnPlan plan_attn(const gsa_params_t& p) {
+    AttnPlan pl;
+    const int64_t idx_rows = (int64_t)p.B * p.Lq;
+    const int G = p.n_h / p.n_kv;
+    const size_t row_state = (size_t)p.n_kv * G * (p.d_h + 2) * 4;
+    // few rows: split every index set into parallel parts; otherwise one launch per L2-sized key range
+    pl.mode = idx_rows * p.n_kv < 2 * (int64_t)sm_count() * kWarpsPrefill ? 1 : 0;
+    int nr = (p.Lk + g_range_keys - 1) / g_range_keys;
+    if (nr > kMaxRanges) nr = kMaxRanges;
+    pl.n_ranges = pl.mode == 0 ? nr : 1;
+    pl.slots = pl.mode == 1 ? kMaxParts : 1;
+    pl.state_bytes = (size_t)pl.slots * idx_rows * row_state;
+    pl.cuts_bytes = pl.mode == 0 && pl.n_ranges > 1 ? (size_t)idx_rows * pl.n_ranges * 4 : 0;
+    return pl;
+}
+
 template <int DH, int G, bool FUSE_G2>
-cudaError_t launch_attn_t(const AttnArgs& a0, int n_kv, cudaStream_t st) {
-    constexpr int STAGES = FUSE_G2 ? 2 : 3;
-    constexpr int PER_WARP = STAGES * (FUSE_G2 ? 3 : 2) * kTileKeys * DH * 2;
-    AttnArgs a = a0;
-    a.q_per_cta = 8 / n_kv > 0 ? 8 / n_kv : 1;
-    const int warps = a.q_per_cta * n_kv;
-    const size_t smem = (size_t)warps * PER_WARP;
-    auto kern = gsa_sparse_attn_kernel<DH, G, FUSE_G2, STAGES>;
+cudaError_t launch_attn_t(AttnArgs a, const gsa_params_t& p, const AttnPlan& pl, const __nv_bfloat16* g1,
+                          __nv_bfloat16* out, int32_t* cuts, cudaStream_t st) {
+    constexpr int VSTAGES = FUSE_G2 ? 1 : 2;
+    constexpr int kWarpsPerCta = FUSE_G2 ? kWarpsFused : kWarpsPrefill;
+    constexpr size_t smem = (size_t)kWarpsPerCta * VSTAGES * kTileKeys * (DH * 2 + 16);
+    auto kern = gsa_sparse_attn_kernel<DH, G, FUSE_G2>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    const int ctas = (a.rr.rows() + a.q_per_cta - 1) / a.q_per_cta;
-    kern<<<ctas, warps * 32, smem, st>>>(a);
+    int per_sm = 1;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kWarpsPerCta * 32, smem);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) per_sm = 1;
+    const int64_t cap = (int64_t)sm_count() * per_sm;
+    const RowRange rr_all = a.rr;
+    const int q_end = rr_all.q_begin + rr_all.R;
+    const int off = p.Lk - p.Lq;
+
+    if (pl.mode == 0 && pl.n_ranges > 1) {
+        const int64_t n = (int64_t)rr_all.rows() * pl.n_ranges;
+        gsa_range_cuts_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(a.idx, a.kt, cuts, rr_all, a.il, a.k_max,
+                                                                          pl.n_ranges, g_range_keys);
+        ++g_launches;
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
+    a.cuts = cuts;
+    a.n_cuts = pl.n_ranges;
+    a.mode = pl.mode;
+    for (int rg = 0; rg < pl.n_ranges; ++rg) {
+        AttnArgs ar = a;
+        ar.range = rg;
+        if (pl.mode == 0) {
+            // queries that cannot see the range's first key have nothing in it
+            const int t_min = rg * g_range_keys - off;
+            if (t_min >= q_end) break;
+            if (t_min > rr_all.q_begin) { ar.rr.q_begin = t_min; ar.rr.R = q_end - t_min; }
+        }
+        const int64_t items = (int64_t)ar.rr.rows() * a.n_kv * (pl.mode == 1 ? kMaxParts : 1);
+        const int64_t want = (items + kWarpsPerCta - 1) / kWarpsPerCta;
+        const int ctas = (int)(want < cap ? want : cap);
+        kern<<<ctas, kWarpsPerCta * 32, smem, st>>>(ar);
+        ++g_launches;
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
+    const int64_t total = (int64_t)rr_all.rows() * a.n_kv * DH;
+    gsa_attn_finalize_kernel<DH, G><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(
+        a.state, a.kt, g1, out, rr_all, a.il, a.idx_rows, p.Lq, p.n_h, p.n_kv, p.k_max, pl.mode);
     ++g_launches;
     return cudaGetLastError();
 }
 
 template <int DH, bool FUSE_G2>
-cudaError_t launch_attn_g(const AttnArgs& a, int G, int n_kv, cudaStream_t st) {
+cudaError_t launch_attn_g(const AttnArgs& a, const gsa_params_t& p, const AttnPlan& pl, const __nv_bfloat16* g1,
+                          __nv_bfloat16* out, int32_t* cuts, int G, cudaStream_t st) {
     switch (G) {
-        case 1: return launch_attn_t<DH, 1, FUSE_G2>(a, n_kv, st);
-        case 2: return launch_attn_t<DH, 2, FUSE_G2>(a, n_kv, st);
-        case 4: return launch_attn_t<DH, 4, FUSE_G2>(a, n_kv, st);
-        case 8: return launch_attn_t<DH, 8, FUSE_G2>(a, n_kv, st);
+        case 1: return launch_attn_t<DH, 1, FUSE_G2>(a, p, pl, g1, out, cuts, st);
+        case 2: return launch_attn_t<DH, 2, FUSE_G2>(a, p, pl, g1, out, cuts, st);
+        case 4: return launch_attn_t<DH, 4, FUSE_G2>(a, p, pl, g1, out, cuts, st);
+        case 8: return launch_attn_t<DH, 8, FUSE_G2>(a, p, pl, g1, out, cuts, st);
     }
     return cudaErrorInvalidValue;
 }
 
 }  // namespace
+
+size_t attn_scratch_bytes(const gsa_params_t& p) {
+    const AttnPlan pl = plan_attn(p);
+    return (pl.state_bytes + 255) / 256 * 256 + (pl.cuts_bytes + 255) / 256 * 256;
+}
+
+void set_attn_range_keys(int keys) { g_range_keys = keys >= 1024 ? keys : kRangeKeysDefault; }
 
 cudaError_t launch_value_gate(const __nv_bfloat16* V, const __nv_bfloat16* g2, __nv_bfloat16* Vg,
                               int64_t n_elems, cudaStream_t st) {
@@ -280,17 +561,25 @@ cudaError_t launch_value_gate(const __nv_bfloat16* V, const __nv_bfloat16* g2, _
 cudaError_t launch_sparse_attn(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* Q,
                                const __nv_bfloat16* K, const __nv_bfloat16* V,
                                const __nv_bfloat16* g1, const __nv_bfloat16* g2, const int32_t* idx,
-                               const int32_t* kt, IdxLayout il, __nv_bfloat16* out, cudaStream_t st) {
+                               const int32_t* kt, IdxLayout il, __nv_bfloat16* out, void* scratch,
+                               cudaStream_t st) {
     if (rr.rows() <= 0) return cudaSuccess;
+    const AttnPlan pl = plan_attn(p);
     AttnArgs a;
-    a.Q = Q; a.K = K; a.V = V; a.g1 = g1; a.g2 = g2; a.idx = idx; a.kt = kt; a.out = out;
-    a.rr = rr; a.il = il; a.Lq = p.Lq; a.Lk = p.Lk; a.n_h = p.n_h; a.n_kv = p.n_kv; a.k_max = p.k_max;
-    a.q_per_cta = 1;
+    a.Q = Q; a.K = K; a.V = V; a.g2 = g2; a.idx = idx; a.kt = kt;
+    a.state = reinterpret_cast<float*>(scratch);
+    int32_t* cuts = reinterpret_cast<int32_t*>((char*)scratch + (pl.state_bytes + 255) / 256 * 256);
+    a.cuts = cuts;
+    a.rr = rr; a.il = il; a.idx_rows = (int64_t)p.B * p.Lq;
+    a.Lq = p.Lq; a.Lk = p.Lk; a.n_h = p.n_h; a.n_kv = p.n_kv; a.k_max = p.k_max;
+    a.mode = pl.mode; a.range = 0; a.n_cuts = pl.n_ranges;
     const float sc = p.sm_scale > 0.f ? p.sm_scale : 1.0f / sqrtf((float)p.d_h);
     a.scale_log2 = sc * 1.4426950408889634f;
     const int G = p.n_h / p.n_kv;
-    if (p.d_h == 128) return g2 ? launch_attn_g<128, true>(a, G, p.n_kv, st) : launch_attn_g<128, false>(a, G, p.n_kv, st);
-    if (p.d_h == 64) return g2 ? launch_attn_g<64, true>(a, G, p.n_kv, st) : launch_attn_g<64, false>(a, G, p.n_kv, st);
+    if (p.d_h == 128)
+        return g2 ? launch_attn_g<128, true>(a, p, pl, g1, out, cuts, G, st) : launch_attn_g<128, false>(a, p, pl, g1, out, cuts, G, st);
+    if (p.d_h == 64)
+        return g2 ? launch_attn_g<64, true>(a, p, pl, g1, out, cuts, G, st) : launch_attn_g<64, false>(a, p, pl, g1, out, cuts, G, st);
     return cudaErrorInvalidValue;
 }
 

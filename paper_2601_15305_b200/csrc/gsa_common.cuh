@@ -28,7 +28,8 @@ struct IdxLayout {
 constexpr int kStatusBytes = 256;   // head of every workspace: device status word + padding
 
 // device status word values
-enum : int32_t { kDevOk = 0, kDevTimeoutTma = 1, kDevTimeoutMma = 2, kDevTimeoutEpi = 3 };
+enum : int32_t { kDevOk = 0, kDevTimeoutTma = 1, kDevTimeoutMma = 2, kDevTimeoutEpi = 3,
+                 kDevTimeoutGather = 4, kDevTimeoutAttn = 5 };
 
 extern int64_t g_launches;          // host-side launch counter
 
@@ -48,7 +49,16 @@ cudaError_t launch_sparse_attn(const gsa_params_t& p, RowRange rr, const __nv_bf
                                const __nv_bfloat16* K, const __nv_bfloat16* V,
                                const __nv_bfloat16* g1, const __nv_bfloat16* g2 /*nullable*/,
                                const int32_t* idx, const int32_t* kt, IdxLayout il,
-                               __nv_bfloat16* out, cudaStream_t st);
+                               __nv_bfloat16* out, void* scratch, cudaStream_t st);
+
+// bytes of device scratch launch_sparse_attn needs for `p` (softmax state slots, range cuts)
+size_t attn_scratch_bytes(const gsa_params_t& p);
+// keys per L2-resident key range of the sparse-attention gather (tuning knob)
+void set_attn_range_keys(int keys);
+
+// device address, on the current device, of the library's built-in scratch array (status word at
+// its start, then the gated values of the allocation-free entry point)
+cudaError_t static_scratch_address(void** ptr);
 
 // ---- device helpers ------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -90,6 +100,53 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
         "{%8,%9}, {%0,%1,%2,%3};\n"
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// ---- mbarrier (shared-memory barrier objects completed by arrivals and by async-copy bytes) --
+constexpr uint32_t kSpinLimit = 1u << 24;        // polls
+constexpr long long kSpinCycles = 1ll << 31;     // ~1 s of SM clock: no wait may last longer
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// bounded wait; returns false if it gave up (and raises the CTA's abort flag)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t_start = clock64();
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 63u) {
+            if (*abort_flag) return false;
+            if (clock64() - t_start > kSpinCycles) break;
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+// one contiguous run global -> shared by the bulk-copy engine; both addresses 16-byte aligned,
+// bytes a multiple of 16; completion is counted on `bar`
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t smem_dst, const void* gsrc, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_dst), "l"(gsrc), "r"(bytes), "r"(bar)
+                 : "memory");
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {

@@ -18,7 +18,8 @@ namespace {
 constexpr size_t kStaticVgBytes = GSA_STATIC_SCRATCH_BYTES;
 
 // Every GPU that loads the library holds this array until the process exits.
-static __device__ __align__(256) unsigned char g_static_scratch[kStaticVgBytes];
+// Layout: a 256-byte head holding the device status word, the attention scratch, the gated values.
+static __device__ __align__(256) unsigned char g_static_scratch[kStatusBytes + kStaticVgBytes];
 
 constexpr int kMaxDevices = 64;
 std::mutex g_setup_mutex;
@@ -45,6 +46,9 @@ cudaError_t scratch_on_current_device(void** ptr) {
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace
+
+cudaError_t static_scratch_address(void** ptr) { return scratch_on_current_device(ptr); }
+
 }  // namespace gsa
 
 using namespace gsa;
@@ -64,11 +68,13 @@ extern "C" int gsa_sparse_gated_attn_fwd_static(const gsa_params_t* p, const voi
         return GSA_ERR_INVALID_ARG;
 
     const size_t vg_bytes = (size_t)p->B * p->Lk * p->n_kv * p->d_h * 2;
-    if (vg_bytes > kStaticVgBytes) {
+    const size_t attn_bytes = (attn_scratch_bytes(*p) + 255) / 256 * 256;
+    if (vg_bytes + attn_bytes > kStaticVgBytes) {
         fprintf(stderr,
-                "gsa_sparse_gated_attn_fwd_static: B*Lk*n_kv*d_h*2 = %zu bytes of gated values exceed the "
-                "built-in scratch array of %zu bytes; use gsa_sparse_gated_attn_fwd with a workspace\n",
-                vg_bytes, kStaticVgBytes);
+                "gsa_sparse_gated_attn_fwd_static: %zu bytes of gated values (B*Lk*n_kv*d_h*2) plus %zu bytes of "
+                "attention scratch exceed the built-in scratch array of %zu bytes; use "
+                "gsa_sparse_gated_attn_fwd with a workspace\n",
+                vg_bytes, attn_bytes, kStaticVgBytes);
         return GSA_ERR_STATIC_SCRATCH;
     }
 
@@ -79,16 +85,21 @@ extern "C" int gsa_sparse_gated_attn_fwd_static(const gsa_params_t* p, const voi
         return GSA_ERR_CUDA;
     }
     cudaStream_t st = (cudaStream_t)stream;
-    __nv_bfloat16* Vg = (__nv_bfloat16*)scratch;
-    // the pre-pass overwrites every element the attention kernel will read, so nothing of an
-    // earlier call's contents survives into this one
-    e = launch_value_gate((const __nv_bfloat16*)V, (const __nv_bfloat16*)g2_logits, Vg,
+    void* attn_scratch = (char*)scratch + kStatusBytes;
+    __nv_bfloat16* Vg = (__nv_bfloat16*)((char*)scratch + kStatusBytes + attn_bytes);
+    // The array keeps what the previous call left in it.  The status word must start at zero and is
+    // cleared here; the pre-pass overwrites every gated value the attention kernel will read, and the
+    // attention kernels write every state slot before they read it.
+    e = cudaMemsetAsync(scratch, 0, kStatusBytes, st);
+    if (e == cudaSuccess)
+        e = launch_value_gate((const __nv_bfloat16*)V, (const __nv_bfloat16*)g2_logits, Vg,
                           (int64_t)p->B * p->Lk * p->n_kv * p->d_h, st);
     if (e == cudaSuccess) {
         RowRange rr{0, p->B, p->q_begin, qe - p->q_begin};
         IdxLayout il{0, rr.q_begin, rr.R};
         e = launch_sparse_attn(*p, rr, (const __nv_bfloat16*)Q, (const __nv_bfloat16*)K, Vg,
-                               (const __nv_bfloat16*)g1_logits, nullptr, idx, kt, il, (__nv_bfloat16*)out, st);
+                               (const __nv_bfloat16*)g1_logits, nullptr, idx, kt, il, (__nv_bfloat16*)out,
+                               attn_scratch, st);
     }
     if (e != cudaSuccess) {
         fprintf(stderr, "gsa: CUDA error: %s\n", cudaGetErrorString(e));

@@ -59,15 +59,15 @@ def run_topk(cfg, scores, q_begin=0, q_end=0, k_mode=0, **over):
     return idx, kt, var
 
 
-def run_attn(cfg, d, idx, kt, q_begin=0, q_end=0, use_g2=True, ws_bytes=None, sm_scale=0.0, **over):
+def run_attn(cfg, d, idx, kt, q_begin=0, q_end=0, use_g2=True, prepass=True, sm_scale=0.0, **over):
     qe = q_end or cfg.Lq
     p = gsa.make_params(cfg, q_begin=q_begin, q_end=qe, sm_scale=sm_scale, **over)
     out = torch.full_like(d["Q"], float("nan"))
-    if ws_bytes is None:
-        ws_bytes = 256 + d["V"].numel() * 2
-    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda") if ws_bytes else None
+    # without room for V' in the workspace, G2 is applied on the gathered rows
+    ws = torch.empty(gsa.gsa_attn_workspace_bytes(p, prepass), dtype=torch.uint8, device="cuda")
+    ws.fill_(0xFF)        # the kernels must not rely on a cleared workspace (0xFF..: NaN as fp32)
     gsa.gsa_sparse_gated_attn_fwd(p, d["Q"], d["K"], d["V"], d["g1"], d["g2"] if use_g2 else None, idx, kt, out, ws)
-    torch.cuda.synchronize()
+    assert gsa.gsa_device_status(ws) == 0
     return out
 
 

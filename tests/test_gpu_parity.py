@@ -181,7 +181,7 @@ def test_attn_given_oracle_indices_tiny(tiny):
     idx = torch.from_numpy(o["idx"]).cuda()[None]
     kt = torch.from_numpy(o["keff"]).cuda()[None]
     for use_prepass in (True, False):
-        out = U.run_attn(cfg, d, idx, kt, ws_bytes=None if use_prepass else 0)
+        out = U.run_attn(cfg, d, idx, kt, prepass=use_prepass)
         U.check_out(out[0].float().cpu().numpy(), o["out"])
 
 

@@ -43,7 +43,7 @@ def _both_paths(cfg, seed):
     want = U.run_attn(cfg, d, idx, kt)                       # regular entry point, caller's workspace
     got = torch.full_like(d["Q"], float("nan"))
     gsa.gsa_sparse_gated_attn_fwd_static(p, d["Q"], d["K"], d["V"], d["g1"], d["g2"], idx, kt, got)
-    torch.cuda.synchronize()
+    assert gsa.gsa_device_status(None) == 0          # the status word of the built-in array
     return got.float().cpu().numpy(), want.float().cpu().numpy()
 
 
@@ -60,8 +60,8 @@ def test_static_scratch_matches_regular_entry_point_twice():
 
 
 def test_static_scratch_rejects_oversized_problem():
-    # one token more than fits: 8193 tokens * 8 KV heads * 128 * 2 bytes > 16 MiB
-    cfg = CONFIGS["l8k"].with_(name="toolarge", B=1, Lq=1, Lk=8193)
+    # one token more than could ever fit: 16385 tokens * 8 KV heads * 128 * 2 bytes > 32 MiB
+    cfg = CONFIGS["l8k"].with_(name="toolarge", B=1, Lq=1, Lk=16385)
     assert cfg.B * cfg.Lk * cfg.n_kv * cfg.d_h * 2 > gsa.STATIC_SCRATCH_BYTES
     p = gsa.make_params(cfg)
     z = lambda *s, dt=torch.bfloat16: torch.zeros(*s, dtype=dt, device="cuda")
