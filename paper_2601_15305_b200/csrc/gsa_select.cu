@@ -1,17 +1,19 @@
 // Adaptive sparsity controller: per query row, the variance of the visible scores (Eq. 8),
-// the budget k_t, and the exact top-k_t positions (Eq. 4) by radix select.
+// the budget k_t, and the exact top-k_t positions (Eq. 4).
 //
-// One CTA per row; two reads of the row (one when it fits in shared memory):
-//   0  a small contiguous-chunk sample of the row fixes the key range the histogram resolves
-//   1  full read: fp64 sum and sum of squares (a centred second pass when the row is staged in
-//      shared memory), and a 4096-bin histogram of the order-preserving integer key
-//      -> Var, k_t, the bin b holding the k_t-th largest key, the count above it
-//   2  full read: every position whose bin is >= b is appended, in position order, to a list in
-//      shared memory (k_t "sure" entries at most, plus the candidates of bin b)
-//   3  on chip: radix rounds over the candidates give the exact threshold key T and how many keys
-//      equal to T are taken; one ordered compaction of the list writes S_t ascending.
-// Equal keys go to the lower position, so the output is unique.  If the list would overflow
-// (degenerate rows: huge ties in bin b), the CTA falls back to radix rounds over the whole row.
+// One CTA per row, one full read of the row:
+//   0  a sample of the row (256 chunks of 32 consecutive scores, evenly spread) is histogrammed;
+//      it gives a threshold key tau that about 1.3 * min(k_max, n) scores of the row should reach
+//      (k_t itself is not known yet: it depends on the variance of the whole row)
+//   1  full read: fp64 sum and sum of squares of every score; every position whose key reaches tau
+//      is appended, in position order, to a candidate list in shared memory (a few percent of the row)
+//      -> Var, k_t
+//   2  on chip: radix rounds over the candidates give the exact threshold key T of the k_t-th largest
+//      score and how many keys equal to T are taken; one ordered compaction of the list writes S_t
+//      ascending.
+// Equal keys go to the lower position, so the output is unique.  If the list overflows or comes out
+// shorter than k_t (the sample misjudged the row: huge ties, scores sorted by position, ...) the CTA
+// falls back to radix rounds over the whole row in global memory: slower, same result.
 #include "gsa_common.cuh"
 
 namespace gsa {
@@ -23,10 +25,12 @@ constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kBinsLog2 = 12;
 constexpr int kBins = 1 << kBinsLog2;
 constexpr int kBinsPerThread = kBins / kSelThreads;   // 8
-constexpr int kListCap = 6144;                        // entries of the candidate list
-constexpr int kListPerThread = kListCap / kSelThreads;  // 12
-constexpr int kChunkPerThread = 8;                    // pass 2: consecutive elements per thread
+constexpr int kListCap = 8192;                        // entries of the candidate list
+constexpr int kListPerThread = kListCap / kSelThreads;  // 16
+constexpr int kChunkPerThread = 16;                   // consecutive elements per thread and chunk
 constexpr int kChunk = kSelThreads * kChunkPerThread;
+constexpr int kSampleChunks = 256;                    // sample = 256 chunks of 32 scores
+constexpr int kSamplePerThread = kSampleChunks * 32 / kSelThreads;   // 16
 
 struct SelectArgs {
     const float* scores;
@@ -43,8 +47,8 @@ struct SelectArgs {
 
 // monotone map fp32 -> uint32 (larger float <=> larger key); -0 is folded onto +0
 __device__ __forceinline__ uint32_t order_key(float x) {
-    uint32_t b = __float_as_uint(x + 0.0f);
-    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+    const uint32_t b = __float_as_uint(x + 0.0f);
+    return b ^ ((uint32_t)((int32_t)b >> 31) | 0x80000000u);     // negative: all bits flip; else: sign bit set
 }
 
 struct SelShared {
@@ -60,14 +64,11 @@ struct SelShared {
     uint32_t seg_eq[kSelWarps];
     uint32_t found_bin;
     uint32_t found_above;
+    uint32_t overflow;
     double bc_a, bc_b;
     uint32_t bc_min, bc_max;
 };
 
-template <bool CACHED>
-__device__ __forceinline__ float row_at(const float* __restrict__ grow, const float* srow, int i) {
-    return CACHED ? srow[i] : __ldg(grow + i);
-}
 
 __device__ __forceinline__ void block_minmax(SelShared& sh, uint32_t& kmin, uint32_t& kmax) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -172,11 +173,9 @@ __device__ __forceinline__ uint32_t block_excl_scan(SelShared& sh, uint32_t v, i
     return before + inc - v;
 }
 
-template <bool CACHED>
-__global__ void __launch_bounds__(kSelThreads) gsa_select_kernel(const SelectArgs a) {
+__global__ void __launch_bounds__(kSelThreads, 2) gsa_select_kernel(const SelectArgs a) {
     extern __shared__ __align__(16) unsigned char dyn_smem[];
     SelShared& sh = *reinterpret_cast<SelShared*>(dyn_smem);
-    float* srow = reinterpret_cast<float*>(dyn_smem + ((sizeof(SelShared) + 15) / 16) * 16);
 
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int lr = blockIdx.x;
@@ -187,63 +186,93 @@ __global__ void __launch_bounds__(kSelThreads) gsa_select_kernel(const SelectArg
     const int64_t orow = a.il.row(b, t);
     int32_t* __restrict__ out_idx = a.idx + orow * a.k_max;
 
-    // ---- pass 0: key range from a sample of 32-element chunks -------------------------------
-    uint32_t smin = 0xFFFFFFFFu, smax = 0u;
-    {
-        const int chunks = (n + 31) >> 5;
-        const int step = max(1, chunks >> 7);                 // about 128..255 chunks
-        for (int c = wid * step; c < chunks; c += kSelWarps * step) {
-            const int i = (c << 5) + lane;
-            if (i < n) {
-                const uint32_t k = order_key(__ldg(grow + i));
-                smin = min(smin, k);
-                smax = max(smax, k);
-            }
+    if (tid == 0) sh.overflow = 0u;
+
+    // ---- pass 0: candidate threshold from a sample ------------------------------------------
+    uint32_t tau = 0u;                                        // every key reaches 0: short rows keep everything
+    if (n > kListCap) {
+        const int chunks = n >> 5;                            // full chunks of 32
+        // sample chunk j of 256 sits at floor(j * chunks / 256): evenly spread over the row
+        uint32_t skey[kSamplePerThread];
+        uint32_t smin = 0xFFFFFFFFu, smax = 0u;
+#pragma unroll
+        for (int e = 0; e < kSamplePerThread; ++e) {
+            const int j = wid + e * kSelWarps;
+            const int c = (int)(((int64_t)j * chunks) >> 8);
+            skey[e] = order_key(__ldg(grow + (c << 5) + lane));
+            smin = min(smin, skey[e]);
+            smax = max(smax, skey[e]);
         }
         block_minmax(sh, smin, smax);
-    }
-    // histogram range: the sampled range widened below by a quarter and above by once its span;
-    // bin 0 collects keys below it, bin kBins-1 keys above it.
-    uint32_t h_lo, h_hi;
-    int h_shift = 0;
-    {
-        const uint32_t span = smax - smin;
-        h_lo = smin - min(smin, span >> 2);
-        h_hi = smax + min(0xFFFFFFFFu - smax, span);
-        const uint32_t hspan = h_hi - h_lo;
-        while (h_shift < 32 && (hspan >> h_shift) >= (uint32_t)(kBins - 2)) ++h_shift;
-    }
-    auto bin_of = [&](uint32_t key) -> uint32_t {
-        return key < h_lo ? 0u : (key > h_hi ? (uint32_t)(kBins - 1) : 1u + ((key - h_lo) >> h_shift));
-    };
-
-    // ---- pass 1: fp64 moments + histogram (and staging) -------------------------------------
-    for (int i = tid; i < kBins; i += kSelThreads) sh.hist[i] = 0u;
-    __syncthreads();
-    double s1 = 0.0, s2 = 0.0;
-    {
-        const int n4 = n >> 2;
-        const float4* __restrict__ g4 = reinterpret_cast<const float4*>(grow);
-        for (int i = tid; i < n4; i += kSelThreads) {
-            const float4 v = __ldg(g4 + i);
-            if (CACHED) reinterpret_cast<float4*>(srow)[i] = v;
-            const float xs[4] = {v.x, v.y, v.z, v.w};
+        int shift = 0;
+        while (shift < 32 && ((smax - smin) >> shift) >= (uint32_t)kBins) ++shift;
+        for (int i = tid; i < kBins; i += kSelThreads) sh.hist[i] = 0u;
+        __syncthreads();
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const double xd = (double)xs[e];
-                s1 += xd;
-                if (!CACHED) s2 = fma(xd, xd, s2);
-                atomicAdd(&sh.hist[bin_of(order_key(xs[e]))], 1u);
+        for (int e = 0; e < kSamplePerThread; ++e) atomicAdd(&sh.hist[(skey[e] - smin) >> shift], 1u);
+        __syncthreads();
+        // the sample rank that corresponds to 1.3 * min(k_max, n) + 64 scores of the whole row
+        const int k_cap = a.k_max < n ? a.k_max : n;
+        const double frac = (1.3 * (double)k_cap + 64.0) / (double)n;
+        uint32_t want = (uint32_t)ceil(frac * (double)(kSampleChunks * 32));
+        want = max(1u, min(want, (uint32_t)(kSampleChunks * 32)));
+        uint32_t fb, fa;
+        find_bin(sh, want, fb, fa);
+        tau = smin + (fb << shift);                           // lower edge of that bin
+    }
+    __syncthreads();
+
+    // ---- pass 1: fp64 moments of every score; ordered list of the candidates ----------------
+    double s1 = 0.0, s2 = 0.0;
+    uint32_t base = 0;
+    {
+        int slot = 0;
+        for (int c0 = 0; c0 < n; c0 += kChunk, slot ^= 1) {
+            const int i0 = c0 + tid * kChunkPerThread;
+            uint32_t keys[kChunkPerThread];
+            uint32_t flags = 0;
+            if (i0 + kChunkPerThread <= n) {
+#pragma unroll
+                for (int v = 0; v < kChunkPerThread / 4; ++v) {
+                    const float4 x4 = __ldg(reinterpret_cast<const float4*>(grow + i0) + v);
+                    const float xs[4] = {x4.x, x4.y, x4.z, x4.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const double xd = (double)xs[e];
+                        s1 += xd;
+                        s2 = fma(xd, xd, s2);
+                        keys[v * 4 + e] = order_key(xs[e]);
+                        flags |= (keys[v * 4 + e] >= tau ? 1u : 0u) << (v * 4 + e);
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < kChunkPerThread; ++e) {
+                    keys[e] = 0u;
+                    if (i0 + e < n) {
+                        const float x = __ldg(grow + i0 + e);
+                        const double xd = (double)x;
+                        s1 += xd;
+                        s2 = fma(xd, xd, s2);
+                        keys[e] = order_key(x);
+                        flags |= (keys[e] >= tau ? 1u : 0u) << e;
+                    }
+                }
             }
-        }
-        const int i = (n4 << 2) + tid;
-        if (i < n) {
-            const float x = __ldg(grow + i);
-            if (CACHED) srow[i] = x;
-            const double xd = (double)x;
-            s1 += xd;
-            if (!CACHED) s2 = fma(xd, xd, s2);
-            atomicAdd(&sh.hist[bin_of(order_key(x))], 1u);
+            uint32_t total;
+            uint32_t pos = base + block_excl_scan(sh, __popc(flags), slot, total);
+            if (base + total <= (uint32_t)kListCap) {
+#pragma unroll
+                for (int e = 0; e < kChunkPerThread; ++e)
+                    if (flags & (1u << e)) {
+                        sh.list_idx[pos] = (uint32_t)(i0 + e);
+                        sh.list_key[pos] = keys[e];
+                        ++pos;
+                    }
+            } else if (tid == 0) {
+                sh.overflow = 1u;                             // block-uniform condition
+            }
+            base += total;
         }
     }
 #pragma unroll
@@ -260,25 +289,9 @@ __global__ void __launch_bounds__(kSelThreads) gsa_select_kernel(const SelectArg
     }
     __syncthreads();
     const double mean = sh.bc_a / (double)n;
-    double var;
-    if (CACHED) {
-        double c2 = 0.0;
-        for (int i = tid; i < n; i += kSelThreads) {
-            const double dlt = (double)srow[i] - mean;
-            c2 = fma(dlt, dlt, c2);
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) c2 += __shfl_xor_sync(0xFFFFFFFFu, c2, o);
-        __syncthreads();                       // red_a was read by thread 0 above
-        if (lane == 0) sh.red_a[wid] = c2;
-        __syncthreads();
-        double tc = 0.0;
-        for (int i = 0; i < kSelWarps; ++i) tc += sh.red_a[i];
-        var = tc / (double)n;
-    } else {
-        var = sh.bc_b / (double)n - mean * mean;
-        if (var < 0.0) var = 0.0;
-    }
+    double var = sh.bc_b / (double)n - mean * mean;
+    if (var < 0.0) var = 0.0;
+    const bool overflow = sh.overflow != 0u;
 
     // ---- Eq. 8 ------------------------------------------------------------------------------
     double r;
@@ -301,71 +314,17 @@ __global__ void __launch_bounds__(kSelThreads) gsa_select_kernel(const SelectArg
         return;
     }
 
-    // ---- the bin of the k-th largest key ----------------------------------------------------
-    uint32_t b1, n_above;
-    find_bin(sh, (uint32_t)k, b1, n_above);
-    const uint32_t c1 = sh.hist[b1];
-    __syncthreads();
-
+    const int m = (int)base;                    // candidates found (all of them listed unless overflow)
     uint32_t T, need_eq;
-    if (n_above + c1 <= (uint32_t)kListCap) {
-        // ---- pass 2: ordered list of every position with bin >= b1 --------------------------
-        uint32_t base = 0;
-        int slot = 0;
-        for (int c0 = 0; c0 < n; c0 += kChunk, slot ^= 1) {
-            const int i0 = c0 + tid * kChunkPerThread;
-            uint32_t keys[kChunkPerThread];
-            uint32_t flags = 0;
-            if (i0 + kChunkPerThread <= n) {
-                float xs[kChunkPerThread];
-                if (CACHED) {
-                    const float4 v0 = *reinterpret_cast<const float4*>(srow + i0);
-                    const float4 v1 = *reinterpret_cast<const float4*>(srow + i0 + 4);
-                    xs[0] = v0.x; xs[1] = v0.y; xs[2] = v0.z; xs[3] = v0.w;
-                    xs[4] = v1.x; xs[5] = v1.y; xs[6] = v1.z; xs[7] = v1.w;
-                } else {
-                    const float4 v0 = __ldg(reinterpret_cast<const float4*>(grow + i0));
-                    const float4 v1 = __ldg(reinterpret_cast<const float4*>(grow + i0 + 4));
-                    xs[0] = v0.x; xs[1] = v0.y; xs[2] = v0.z; xs[3] = v0.w;
-                    xs[4] = v1.x; xs[5] = v1.y; xs[6] = v1.z; xs[7] = v1.w;
-                }
-#pragma unroll
-                for (int e = 0; e < kChunkPerThread; ++e) {
-                    keys[e] = order_key(xs[e]);
-                    flags |= (bin_of(keys[e]) >= b1 ? 1u : 0u) << e;
-                }
-            } else {
-#pragma unroll
-                for (int e = 0; e < kChunkPerThread; ++e) {
-                    keys[e] = 0u;
-                    if (i0 + e < n) {
-                        keys[e] = order_key(row_at<CACHED>(grow, srow, i0 + e));
-                        flags |= (bin_of(keys[e]) >= b1 ? 1u : 0u) << e;
-                    }
-                }
-            }
-            uint32_t total;
-            uint32_t pos = base + block_excl_scan(sh, __popc(flags), slot, total);
-#pragma unroll
-            for (int e = 0; e < kChunkPerThread; ++e)
-                if (flags & (1u << e)) {
-                    sh.list_idx[pos] = (uint32_t)(i0 + e);
-                    sh.list_key[pos] = keys[e];
-                    ++pos;
-                }
-            base += total;
-        }
-        __syncthreads();
-        const int m = (int)base;                               // == n_above + c1
-
-        // ---- exact threshold among the candidates of bin b1 ---------------------------------
+    if (!overflow && m >= k) {
+        // ---- exact threshold among the candidates ---------------------------------------------
         uint32_t cmin = 0xFFFFFFFFu, cmax = 0u;
         for (int i = tid; i < m; i += kSelThreads) {
             const uint32_t key = sh.list_key[i];
-            if (bin_of(key) == b1) { cmin = min(cmin, key); cmax = max(cmax, key); }
+            cmin = min(cmin, key); cmax = max(cmax, key);
         }
         block_minmax(sh, cmin, cmax);
-        radix_rounds(sh, m, [&](int i) { return sh.list_key[i]; }, cmin, cmax, (uint32_t)k - n_above, T, need_eq);
+        radix_rounds(sh, m, [&](int i) { return sh.list_key[i]; }, cmin, cmax, (uint32_t)k, T, need_eq);
 
         // ---- ordered compaction of the list into S_t ----------------------------------------
         uint32_t gt = 0, eq = 0;
@@ -394,13 +353,13 @@ __global__ void __launch_bounds__(kSelThreads) gsa_select_kernel(const SelectArg
             }
     } else {
         // ---- fallback: radix rounds over the whole row, then ordered emission ----------------
-        radix_rounds(sh, n, [&](int i) { return order_key(row_at<CACHED>(grow, srow, i)); }, 0u, 0xFFFFFFFFu,
+        radix_rounds(sh, n, [&](int i) { return order_key(__ldg(grow + i)); }, 0u, 0xFFFFFFFFu,
                      (uint32_t)k, T, need_eq);
         const int seg = ((n + kSelWarps - 1) / kSelWarps + 31) & ~31;
         const int seg_lo = min(n, wid * seg), seg_hi = min(n, seg_lo + seg);
         uint32_t cg = 0, ce = 0;
         for (int i = seg_lo + lane; i < seg_hi; i += 32) {
-            const uint32_t key = order_key(row_at<CACHED>(grow, srow, i));
+            const uint32_t key = order_key(__ldg(grow + i));
             cg += key > T;
             ce += key == T;
         }
@@ -414,11 +373,11 @@ __global__ void __launch_bounds__(kSelThreads) gsa_select_kernel(const SelectArg
         uint32_t run_gt = 0, run_eq = 0;
         for (int i = 0; i < wid; ++i) { run_gt += sh.seg_gt[i]; run_eq += sh.seg_eq[i]; }
         const uint32_t lt_mask = (1u << lane) - 1u;
-        for (int base = seg_lo; base < seg_hi; base += 32) {
-            const int i = base + lane;
+        for (int base2 = seg_lo; base2 < seg_hi; base2 += 32) {
+            const int i = base2 + lane;
             uint32_t key = 0;
             const bool in = i < seg_hi;
-            if (in) key = order_key(row_at<CACHED>(grow, srow, i));
+            if (in) key = order_key(__ldg(grow + i));
             const bool gt = in && key > T, eq = in && key == T;
             const uint32_t bg = __ballot_sync(0xFFFFFFFFu, gt), be = __ballot_sync(0xFFFFFFFFu, eq);
             const uint32_t g_before = run_gt + __popc(bg & lt_mask);
@@ -442,21 +401,14 @@ cudaError_t launch_select(const gsa_params_t& p, RowRange rr, const float* score
     a.rr = rr; a.il = il; a.Lq = p.Lq; a.Lk = p.Lk;
     a.k_base = p.k_base; a.k_min = p.k_min; a.k_max = p.k_max; a.k_mode = p.k_mode; a.v_bar = p.v_bar;
 
-    const int n_max = p.Lk - p.Lq + (rr.q_begin + rr.R - 1) + 1;
-    const size_t fixed = ((sizeof(SelShared) + 15) / 16) * 16;
-    constexpr size_t kMaxSmem = 200 * 1024;
-    const size_t cached = fixed + (((size_t)n_max + 3) / 4 * 4) * sizeof(float);
-    cudaError_t e;
+    const size_t smem = ((sizeof(SelShared) + 15) / 16) * 16;
     static bool attr_done = false;
     if (!attr_done) {
-        e = cudaFuncSetAttribute(gsa_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(gsa_select_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fixed);
+        cudaError_t e = cudaFuncSetAttribute(gsa_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    if (cached <= kMaxSmem) gsa_select_kernel<true><<<rr.rows(), kSelThreads, cached, st>>>(a);
-    else gsa_select_kernel<false><<<rr.rows(), kSelThreads, fixed, st>>>(a);
+    gsa_select_kernel<<<rr.rows(), kSelThreads, smem, st>>>(a);
     ++g_launches;
     return cudaGetLastError();
 }
