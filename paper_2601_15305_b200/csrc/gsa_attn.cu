@@ -378,19 +378,18 @@ __global__ void __launch_bounds__(256) gsa_range_cuts_kernel(const int32_t* __re
 
 // merge the state slots of a (row, head): out = (sum_p 2^(m_p - M) O_p) / (sum_p 2^(m_p - M) l_p) * sigmoid(g1)
 template <int DH, int G>
-__global__ void __launch_bounds__(256) gsa_attn_finalize_kernel(const float* __restrict__ state, const int32_t* __restrict__ kt,
+__global__ void __launch_bounds__(1024) gsa_attn_finalize_kernel(const float* __restrict__ state, const int32_t* __restrict__ kt,
                                                                 const __nv_bfloat16* __restrict__ g1, __nv_bfloat16* __restrict__ out,
                                                                 RowRange rr, IdxLayout il, int64_t idx_rows, int Lq, int n_h,
                                                                 int n_kv, int k_max, int mode) {
     constexpr int STATE_F = G * (DH + 2);
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const int64_t total = (int64_t)rr.rows() * n_kv * DH;
-    if (i >= total) return;
-    const int d = (int)(i % DH);
-    const int g = (int)((i / DH) % n_kv);
-    const RowId r = row_of(rr, il, (int)(i / ((int64_t)DH * n_kv)));
+    // one CTA per query row; thread = (KV head, d), all G heads of the group
+    const RowId r = row_of(rr, il, (int)blockIdx.x);
     const int k_eff = min(kt[r.irow], k_max);
     const int np = mode == 1 ? parts_of(k_eff) : 1;
+    for (int i = threadIdx.x; i < n_kv * DH; i += blockDim.x) {
+    const int d = i % DH;
+    const int g = i / DH;
     float acc[G], mx[G], den[G];
 #pragma unroll
     for (int e = 0; e < G; ++e) { acc[e] = 0.f; den[e] = 0.f; mx[e] = -INFINITY; }
@@ -416,6 +415,7 @@ __global__ void __launch_bounds__(256) gsa_attn_finalize_kernel(const float* __r
         const size_t at = (((size_t)r.b * Lq + r.t) * n_h + g * G + e) * DH + d;
         const float v = den[e] > 0.f ? acc[e] / den[e] * fast_sigmoid(__bfloat162float(g1[at])) : 0.f;
         out[at] = __float2bfloat16_rn(v);
+    }
     }
 }
 
@@ -518,8 +518,8 @@ cudaError_t launch_attn_t(AttnArgs a, const gsa_params_t& p, const AttnPlan& pl,
         ++g_launches;
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
-    const int64_t total = (int64_t)rr_all.rows() * a.n_kv * DH;
-    gsa_attn_finalize_kernel<DH, G><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(
+    const int fin_threads = a.n_kv * DH < 1024 ? a.n_kv * DH : 1024;
+    gsa_attn_finalize_kernel<DH, G><<<(unsigned)rr_all.rows(), fin_threads, 0, st>>>(
         a.state, a.kt, g1, out, rr_all, a.il, a.idx_rows, p.Lq, p.n_h, p.n_kv, p.k_max, pl.mode);
     ++g_launches;
     return cudaGetLastError();

@@ -339,3 +339,71 @@ def test_argument_errors_do_not_launch(tiny):
     with pytest.raises(gsa.GsaError, match="invalid"):
         gsa.gsa_indexer_scores(p, d["qI"], d["kI"], d["w"], None, torch.empty(10, device="cuda"), 100, small_ws)
     assert gsa.gsa_launch_count() == n0
+
+
+# ------------------------------------------------------------------------------------------ full sizes
+# The workloads of the benchmark at their full sizes, in the launch configuration bench.py times
+# (default slab, default key ranges), checked on sampled rows the oracle computes one by one.
+@pytest.fixture(scope="module")
+def l128k():
+    cfg = CONFIGS["l128k"]
+    x = make_inputs(cfg)
+    return cfg, x, U.to_dev(x)
+
+
+def test_forward_l32k_sampled_rows_budgets_span_the_clamp_range():
+    cfg = CONFIGS["l32k"]
+    x = make_inputs(cfg)
+    d = U.to_dev(x)
+    mism, kt = _forward_and_compare(cfg, x, d, sample_rows(cfg, 24).numpy())
+    k = kt[0, cfg.k_max:].cpu().numpy()
+    assert k.min() == cfg.k_min and k.max() == cfg.k_max          # heterogeneous variance: both clamps are hit
+    assert ((k > cfg.k_min) & (k < cfg.k_max)).mean() > 0.3
+
+
+def test_stages_l128k_sampled_rows(l128k):
+    """Stage by stage at L = 131072: scores of a block of late rows, bit-exact selection on those fp32 scores."""
+    cfg, x, d = l128k
+    for q0 in (70000, cfg.Lq - 48):
+        q1 = q0 + 48
+        sc = U.run_scores(cfg, d, q_begin=q0, q_end=q1)
+        rows = np.array([q0, q0 + 17, q1 - 1])
+        got = sc[0][torch.from_numpy(rows - q0).cuda()].cpu().numpy()
+        want = oracle.scores(U.oracle_params(cfg), x["qI"], x["kI"], x["w"], None, rows)
+        U.check_scores(got, want, _vis(cfg, rows))
+        idx, kt, var = U.run_topk(cfg, sc, q_begin=q0, q_end=q1)
+        o = oracle.select_f32(U.oracle_params(cfg), got, rows)
+        sel = torch.from_numpy(rows - q0).cuda()
+        U.check_selection_exact(o, idx[0][sel].cpu().numpy(), kt[0][sel].cpu().numpy(), None)
+
+
+def test_forward_l128k_sampled_rows(l128k):
+    cfg, x, d = l128k
+    mism, kt = _forward_and_compare(cfg, x, d, sample_rows(cfg, 16).numpy())
+    k = kt[0, cfg.k_max:].float()
+    assert k.min() >= cfg.k_min and k.max() <= cfg.k_max and 1500 < k.mean() < 3000
+
+
+def test_forward_decode_full_size():
+    """B = 32 single-token queries over 131072-token caches; sequences are generated and uploaded one
+    at a time, the oracle checks a sample of them."""
+    cfg = CONFIGS["decode"]
+    p = gsa.make_params(cfg)
+    dev = {}
+    checked = (0, 5, 13, 22, 31)
+    host = {}
+    for b in range(cfg.B):
+        xb = make_inputs(cfg, slice(b, b + 1))
+        for k, v in xb.items():
+            if k not in dev:
+                dev[k] = torch.empty((cfg.B,) + tuple(v.shape[1:]), dtype=v.dtype, device="cuda")
+            dev[k][b].copy_(v[0])
+        if b in checked:
+            host[b] = xb
+    out, idx, kt, var = U.run_forward(cfg, dev)
+    cfg1 = cfg.with_(B=1)
+    for b in checked:
+        o = oracle.forward(U.oracle_params(cfg1), **host[b], rows_t=np.zeros(1, np.int32), want_scores=True)
+        U.check_e2e_indices(o, idx[b].cpu().numpy(), kt[b].cpu().numpy(), o["scores"], [cfg.Lk])
+        U.check_out(out[b].float().cpu().numpy(), o["out"])
+    assert (kt >= cfg.k_min).all() and (kt <= cfg.k_max).all()
