@@ -165,11 +165,14 @@ def main():
     ap.add_argument("--workload", default="l128k", choices=sorted(CONFIGS))
     ap.add_argument("--impl", default="gsa_b200", choices=["gsa_b200", "reference"])
     ap.add_argument("--slab-rows", type=int, default=0)
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (smaller ncu captures)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "gsa_b200" else args.warmup
     cfg = CONFIGS[args.workload]
+    if args.batch > 0:
+        cfg = cfg.with_(B=args.batch, name=f"{cfg.name}-b{args.batch}")
 
     if args.impl == "reference":
         run_reference(args, cfg)
@@ -186,8 +189,21 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
-    x = make_inputs(cfg)
-    d = {k: v.cuda() for k, v in x.items()}
+    if cfg.B > 4:
+        # many long sequences (decode): generate and upload one batch element at a time
+        x, d = None, {}
+        for b in range(cfg.B):
+            xb = make_inputs(cfg, slice(b, b + 1))
+            for k, v in xb.items():
+                if k not in d:
+                    d[k] = torch.empty((cfg.B,) + tuple(v.shape[1:]), dtype=v.dtype, device="cuda")
+                d[k][b].copy_(v[0])
+        args.no_e2e = True            # the host-buffer leg would pin tens of GB
+        x_cpu_sample = make_inputs(cfg, slice(0, min(cfg.B, 4)))
+    else:
+        x = make_inputs(cfg)
+        d = {k: v.cuda() for k, v in x.items()}
+        x_cpu_sample = x
     p = gsa.make_params(cfg)
     out = torch.empty_like(d["Q"])
     kt = torch.empty((cfg.B, cfg.Lq), dtype=torch.int32, device="cuda")
@@ -284,7 +300,7 @@ def main():
         oracle.build()
         cores = oracle.num_threads()
         n_rows = 256
-        r, dt, n, cores = oracle_sample_rate(cfg, x, n_rows)
+        r, dt, n, cores = oracle_sample_rate(cfg.with_(B=x_cpu_sample["Q"].shape[0]), x_cpu_sample, n_rows)
         cpu_baseline = {"value": r, "unit": UNIT, "cores": cores, "kind": "oracle",
                         "sample": f"{n} stratified query rows of {cfg.name} (full visible context each), {dt:.1f} s"}
 

@@ -20,9 +20,17 @@ cudaError_t launch_indexer_tc(const gsa_params_t& p, RowRange rr, const __nv_bfl
                               float* scores, int64_t row_stride, int32_t* dev_status,
                               cudaStream_t st);
 
+bool indexer_rows_preferred(const gsa_params_t& p, RowRange rr);
+cudaError_t launch_indexer_rows(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* qI,
+                                const __nv_bfloat16* kI, const float* w, const float* bI, float* scores,
+                                int64_t row_stride, cudaStream_t st);
+
 cudaError_t launch_indexer(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* qI,
                            const __nv_bfloat16* kI, const float* w, const float* bI, float* scores,
                            int64_t row_stride, int32_t* dev_status, cudaStream_t st) {
+    // few query rows per sequence (decode): stream the keys once per row instead of filling 32-query tiles
+    if (g_indexer_path == 0 && indexer_rows_preferred(p, rr))
+        return launch_indexer_rows(p, rr, qI, kI, w, bI, scores, row_stride, st);
     if (g_indexer_path == 0 && indexer_tc_supported(p))
         return launch_indexer_tc(p, rr, qI, kI, w, bI, scores, row_stride, dev_status, st);
     return launch_indexer_simple(p, rr, qI, kI, w, bI, scores, row_stride, st);

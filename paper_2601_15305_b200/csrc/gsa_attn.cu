@@ -40,11 +40,11 @@ namespace {
 
 constexpr int kTileKeys = 16;
 constexpr int kWarpsPrefill = 16;          // warps per CTA, V' pre-gated
-constexpr int kWarpsFused = 8;             // warps per CTA when V and g2 pass through registers
+constexpr int kWarpsFused = 12;            // warps per CTA when V and g2 pass through registers
 constexpr int kRangeKeysDefault = 16384;   // keys per L2 range: K + V' rows of 16K tokens = 64 MB at the 1.7B shape
 constexpr int kMaxRanges = 48;
-constexpr int kPartKeys = 256;             // decode: keys per parallel segment
-constexpr int kMaxParts = 8;
+constexpr int kPartKeys = 128;             // decode: fewest keys worth a parallel segment
+constexpr int kMaxParts = 16;              // most segments (and state slots) per index set
 
 struct AttnArgs {
     const __nv_bfloat16* Q;
@@ -60,6 +60,7 @@ struct AttnArgs {
     int64_t idx_rows;         // rows of the idx / kt / state tables
     int32_t Lq, Lk, n_h, n_kv, k_max;
     int32_t mode;             // 0: one key range per launch (range index `range`), 1: parallel parts
+    int32_t max_parts;        // mode 1: segments (= state slots) per index set
     int32_t range, n_cuts;
     float scale_log2;         // sm_scale * log2(e)
 };
@@ -96,9 +97,9 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
     asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
     return d;
 }
-__device__ __forceinline__ int parts_of(int k_eff) {
+__host__ __device__ __forceinline__ int parts_of(int k_eff, int max_parts) {
     const int p = (k_eff + kPartKeys - 1) / kPartKeys;
-    return p < 1 ? 1 : (p > kMaxParts ? kMaxParts : p);
+    return p < 1 ? 1 : (p > max_parts ? max_parts : p);
 }
 
 template <int DH, int G, bool FUSE_G2>
@@ -127,14 +128,14 @@ gsa_sparse_attn_kernel(const AttnArgs a) {
     const bool real_cols = 2 * tig < G;                 // this thread's output columns hold real heads
 
     const int rows = a.rr.rows();
-    const int64_t n_items = (int64_t)rows * n_kv * (a.mode == 1 ? kMaxParts : 1);
+    const int64_t n_items = (int64_t)rows * n_kv * (a.mode == 1 ? a.max_parts : 1);
     const int64_t warps_total = (int64_t)gridDim.x * kWarpsPerCta;
 
     for (int64_t item = (int64_t)blockIdx.x * kWarpsPerCta + warp; item < n_items; item += warps_total) {
         const int g = (int)(item % n_kv);
         int64_t rest = item / n_kv;
         int part = 0;
-        if (a.mode == 1) { part = (int)(rest % kMaxParts); rest /= kMaxParts; }
+        if (a.mode == 1) { part = (int)(rest % a.max_parts); rest /= a.max_parts; }
         const RowId r = row_of(a.rr, a.il, (int)rest);
         const int k_eff = min(a.kt[r.irow], a.k_max);
         int lo, hi, slot = 0;
@@ -147,7 +148,7 @@ gsa_sparse_attn_kernel(const AttnArgs a) {
                 if (a.range + 1 < a.n_cuts) hi = c[1];
             }
         } else {
-            const int np = parts_of(k_eff);
+            const int np = parts_of(k_eff, a.max_parts);
             if (part >= np) continue;
             const int per = ((k_eff + np - 1) / np + kTileKeys - 1) / kTileKeys * kTileKeys;
             lo = part * per;
@@ -264,7 +265,7 @@ gsa_sparse_attn_kernel(const AttnArgs a) {
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         const float2 vf = __bfloat1622float2(v2[e]), gf = __bfloat1622float2(g2v[e]);
-                        v2[e] = __floats2bfloat162_rn(vf.x * fast_sigmoid(gf.x), vf.y * fast_sigmoid(gf.y));
+                        v2[e] = __floats2bfloat162_rn(vf.x * gate_sigmoid(gf.x), vf.y * gate_sigmoid(gf.y));
                     }
                     *reinterpret_cast<uint4*>(my_smem + (i * KPI + vkey) * VSTRIDE + vch * 16) = vv;
                 }
@@ -381,12 +382,12 @@ template <int DH, int G>
 __global__ void __launch_bounds__(1024) gsa_attn_finalize_kernel(const float* __restrict__ state, const int32_t* __restrict__ kt,
                                                                 const __nv_bfloat16* __restrict__ g1, __nv_bfloat16* __restrict__ out,
                                                                 RowRange rr, IdxLayout il, int64_t idx_rows, int Lq, int n_h,
-                                                                int n_kv, int k_max, int mode) {
+                                                                int n_kv, int k_max, int mode, int max_parts) {
     constexpr int STATE_F = G * (DH + 2);
     // one CTA per query row; thread = (KV head, d), all G heads of the group
     const RowId r = row_of(rr, il, (int)blockIdx.x);
     const int k_eff = min(kt[r.irow], k_max);
-    const int np = mode == 1 ? parts_of(k_eff) : 1;
+    const int np = mode == 1 ? parts_of(k_eff, max_parts) : 1;
     for (int i = threadIdx.x; i < n_kv * DH; i += blockDim.x) {
     const int d = i % DH;
     const int g = i / DH;
@@ -432,7 +433,7 @@ __global__ void __launch_bounds__(256) gsa_value_gate_kernel(const uint4* __rest
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const float2 vf = __bfloat1622float2(v2[e]), gf = __bfloat1622float2(g2v[e]);
-            v2[e] = __floats2bfloat162_rn(vf.x * fast_sigmoid(gf.x), vf.y * fast_sigmoid(gf.y));
+            v2[e] = __floats2bfloat162_rn(vf.x * gate_sigmoid(gf.x), vf.y * gate_sigmoid(gf.y));
         }
         Vg[i] = vv;
     }
@@ -468,7 +469,10 @@ AttnPlan plan_attn(const gsa_params_t& p) {
     int nr = (p.Lk + g_range_keys - 1) / g_range_keys;
     if (nr > kMaxRanges) nr = kMaxRanges;
     pl.n_ranges = pl.mode == 0 ? nr : 1;
-    pl.slots = pl.mode == 1 ? kMaxParts : 1;
+    // as many segments per index set as it takes to give every warp slot of the GPU about two items
+    int mp = (int)((2 * (int64_t)sm_count() * kWarpsPrefill + idx_rows * p.n_kv - 1) / (idx_rows * p.n_kv));
+    mp = mp < 1 ? 1 : (mp > kMaxParts ? kMaxParts : mp);
+    pl.slots = pl.mode == 1 ? mp : 1;
     pl.state_bytes = (size_t)pl.slots * idx_rows * row_state;
     pl.cuts_bytes = pl.mode == 0 && pl.n_ranges > 1 ? (size_t)idx_rows * pl.n_ranges * 4 : 0;
     return pl;
@@ -502,6 +506,7 @@ cudaError_t launch_attn_t(AttnArgs a, const gsa_params_t& p, const AttnPlan& pl,
     a.cuts = cuts;
     a.n_cuts = pl.n_ranges;
     a.mode = pl.mode;
+    a.max_parts = pl.slots;
     for (int rg = 0; rg < pl.n_ranges; ++rg) {
         AttnArgs ar = a;
         ar.range = rg;
@@ -511,7 +516,7 @@ cudaError_t launch_attn_t(AttnArgs a, const gsa_params_t& p, const AttnPlan& pl,
             if (t_min >= q_end) break;
             if (t_min > rr_all.q_begin) { ar.rr.q_begin = t_min; ar.rr.R = q_end - t_min; }
         }
-        const int64_t items = (int64_t)ar.rr.rows() * a.n_kv * (pl.mode == 1 ? kMaxParts : 1);
+        const int64_t items = (int64_t)ar.rr.rows() * a.n_kv * (pl.mode == 1 ? pl.slots : 1);
         const int64_t want = (items + kWarpsPerCta - 1) / kWarpsPerCta;
         const int ctas = (int)(want < cap ? want : cap);
         kern<<<ctas, kWarpsPerCta * 32, smem, st>>>(ar);
@@ -520,7 +525,7 @@ cudaError_t launch_attn_t(AttnArgs a, const gsa_params_t& p, const AttnPlan& pl,
     }
     const int fin_threads = a.n_kv * DH < 1024 ? a.n_kv * DH : 1024;
     gsa_attn_finalize_kernel<DH, G><<<(unsigned)rr_all.rows(), fin_threads, 0, st>>>(
-        a.state, a.kt, g1, out, rr_all, a.il, a.idx_rows, p.Lq, p.n_h, p.n_kv, p.k_max, pl.mode);
+        a.state, a.kt, g1, out, rr_all, a.il, a.idx_rows, p.Lq, p.n_h, p.n_kv, p.k_max, pl.mode, pl.slots);
     ++g_launches;
     return cudaGetLastError();
 }
@@ -572,7 +577,7 @@ cudaError_t launch_sparse_attn(const gsa_params_t& p, RowRange rr, const __nv_bf
     a.cuts = cuts;
     a.rr = rr; a.il = il; a.idx_rows = (int64_t)p.B * p.Lq;
     a.Lq = p.Lq; a.Lk = p.Lk; a.n_h = p.n_h; a.n_kv = p.n_kv; a.k_max = p.k_max;
-    a.mode = pl.mode; a.range = 0; a.n_cuts = pl.n_ranges;
+    a.mode = pl.mode; a.max_parts = pl.slots; a.range = 0; a.n_cuts = pl.n_ranges;
     const float sc = p.sm_scale > 0.f ? p.sm_scale : 1.0f / sqrtf((float)p.d_h);
     a.scale_log2 = sc * 1.4426950408889634f;
     const int G = p.n_h / p.n_kv;

@@ -67,7 +67,18 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
 
 __device__ __forceinline__ float fast_sigmoid(float x) {
     // 1 / (1 + 2^(-x log2 e)); ex2.approx and rcp.approx are accurate to a few ulp
-    return __frcp_rn(1.0f + exp2f(-1.4426950408889634f * x));
+    float e, r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fminf(-1.4426950408889634f * x, 126.f)));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + e));
+    return r;
+}
+
+// Sigmoid of a value-gate logit (Eq. 9): 1/2 + 1/2 tanh(x/2), one special-function instruction.
+// tanh.approx is good to 2^-11 relative; the gated value is rounded to bf16 (2^-9) right after.
+__device__ __forceinline__ float gate_sigmoid(float x) {
+    float t;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(0.5f * x));
+    return fmaf(0.5f, t, 0.5f);
 }
 
 __device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gsrc) {

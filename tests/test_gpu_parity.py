@@ -99,6 +99,23 @@ def test_indexer_ragged_batch_decode_shapes():
             U.check_scores(sc[b], want, _vis(cfg, rows))
 
 
+@pytest.mark.parametrize("base,Lq,HI", [("l8k", 1, 8), ("l8k", 3, 8), ("tiny", 2, 4), ("tiny", 4, 2)])
+def test_indexer_few_rows_streams_keys(base, Lq, HI):
+    """Calls with at most 4 query rows per sequence take the key-streaming kernel (decode geometry)."""
+    cfg = CONFIGS[base].with_(name="fewrows", B=3, Lq=Lq, Lk=2117, HI=HI, seed=15)
+    x = make_inputs(cfg)
+    d = U.to_dev(x)
+    bI = torch.linspace(-1.0, 1.5, HI)
+    sc = U.run_scores(cfg, d, bI=bI.cuda()).cpu().numpy()
+    p = U.oracle_params(cfg)
+    for b in range(cfg.B):
+        rows = np.arange(cfg.Lq)
+        want = oracle.scores(p, x["qI"], x["kI"], x["w"], bI, rows, np.full_like(rows, b))
+        U.check_scores(sc[b], want, _vis(cfg, rows))
+        for t in rows:                                   # nothing written past the visible keys
+            assert np.isnan(sc[b, t, cfg.Lk - cfg.Lq + t + 1:cfg.Lk]).all()
+
+
 # ------------------------------------------------------------------------------------------ stage 2
 def _select_and_compare(cfg, sc_dev, rows=None, k_mode=0, **over):
     """sc_dev: [B, Lq, stride] fp32 on the GPU; compares every (or the listed) row of batch 0."""
