@@ -378,45 +378,81 @@ __global__ void __launch_bounds__(256) gsa_range_cuts_kernel(const int32_t* __re
 }
 
 // merge the state slots of a (row, head): out = (sum_p 2^(m_p - M) O_p) / (sum_p 2^(m_p - M) l_p) * sigmoid(g1)
+// A CTA takes kFinRows consecutive query rows; thread = (KV head, d), all G heads of the group.  With a
+// single slot per row (prefill) the loads of all rows are issued before any is used.
+constexpr int kFinRows = 4;
+
 template <int DH, int G>
 __global__ void __launch_bounds__(1024) gsa_attn_finalize_kernel(const float* __restrict__ state, const int32_t* __restrict__ kt,
                                                                 const __nv_bfloat16* __restrict__ g1, __nv_bfloat16* __restrict__ out,
                                                                 RowRange rr, IdxLayout il, int64_t idx_rows, int Lq, int n_h,
                                                                 int n_kv, int k_max, int mode, int max_parts) {
     constexpr int STATE_F = G * (DH + 2);
-    // one CTA per query row; thread = (KV head, d), all G heads of the group
-    const RowId r = row_of(rr, il, (int)blockIdx.x);
-    const int k_eff = min(kt[r.irow], k_max);
-    const int np = mode == 1 ? parts_of(k_eff, max_parts) : 1;
+    const int rows = rr.rows();
+    const int lr0 = blockIdx.x * kFinRows;
     for (int i = threadIdx.x; i < n_kv * DH; i += blockDim.x) {
-    const int d = i % DH;
-    const int g = i / DH;
-    float acc[G], mx[G], den[G];
+        const int d = i % DH;
+        const int g = i / DH;
+        if (mode == 0) {
+            float o[kFinRows][G], l[kFinRows][G], gl[kFinRows][G];
+            int keff[kFinRows];
+            size_t at0[kFinRows];
 #pragma unroll
-    for (int e = 0; e < G; ++e) { acc[e] = 0.f; den[e] = 0.f; mx[e] = -INFINITY; }
-    if (k_eff > 0) {
-        for (int p = 0; p < np; ++p) {
-            const float* st = state + (((int64_t)p * idx_rows + r.irow) * n_kv + g) * STATE_F;
+            for (int q = 0; q < kFinRows; ++q) {
+                const int lr = min(lr0 + q, rows - 1);
+                const RowId r = row_of(rr, il, lr);
+                const float* st = state + ((int64_t)r.irow * n_kv + g) * STATE_F;
+                keff[q] = kt[r.irow];
+                at0[q] = (((size_t)r.b * Lq + r.t) * n_h + g * G) * DH + d;
 #pragma unroll
-            for (int e = 0; e < G; ++e) mx[e] = fmaxf(mx[e], st[G * DH + e]);
-        }
-        for (int p = 0; p < np; ++p) {
-            const float* st = state + (((int64_t)p * idx_rows + r.irow) * n_kv + g) * STATE_F;
+                for (int e = 0; e < G; ++e) {
+                    o[q][e] = st[d * G + e];
+                    l[q][e] = st[G * DH + G + e];
+                    gl[q][e] = __bfloat162float(g1[at0[q] + (size_t)e * DH]);
+                }
+            }
 #pragma unroll
-            for (int e = 0; e < G; ++e) {
-                const float m = st[G * DH + e];
-                const float sc = m == -INFINITY ? 0.f : exp2f(m - mx[e]);
-                acc[e] = fmaf(sc, st[d * G + e], acc[e]);
-                den[e] = fmaf(sc, st[G * DH + G + e], den[e]);
+            for (int q = 0; q < kFinRows; ++q) {
+                if (lr0 + q >= rows) break;
+#pragma unroll
+                for (int e = 0; e < G; ++e) {
+                    const float v = (keff[q] > 0 && l[q][e] > 0.f) ? o[q][e] / l[q][e] * fast_sigmoid(gl[q][e]) : 0.f;
+                    out[at0[q] + (size_t)e * DH] = __float2bfloat16_rn(v);
+                }
+            }
+        } else {
+            for (int q = 0; q < kFinRows && lr0 + q < rows; ++q) {
+                const RowId r = row_of(rr, il, lr0 + q);
+                const int k_eff = min(kt[r.irow], k_max);
+                const int np = parts_of(k_eff, max_parts);
+                float acc[G], mx[G], den[G];
+#pragma unroll
+                for (int e = 0; e < G; ++e) { acc[e] = 0.f; den[e] = 0.f; mx[e] = -INFINITY; }
+                if (k_eff > 0) {
+                    for (int p = 0; p < np; ++p) {
+                        const float* st = state + (((int64_t)p * idx_rows + r.irow) * n_kv + g) * STATE_F;
+#pragma unroll
+                        for (int e = 0; e < G; ++e) mx[e] = fmaxf(mx[e], st[G * DH + e]);
+                    }
+                    for (int p = 0; p < np; ++p) {
+                        const float* st = state + (((int64_t)p * idx_rows + r.irow) * n_kv + g) * STATE_F;
+#pragma unroll
+                        for (int e = 0; e < G; ++e) {
+                            const float m = st[G * DH + e];
+                            const float sc = m == -INFINITY ? 0.f : exp2f(m - mx[e]);
+                            acc[e] = fmaf(sc, st[d * G + e], acc[e]);
+                            den[e] = fmaf(sc, st[G * DH + G + e], den[e]);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int e = 0; e < G; ++e) {
+                    const size_t at = (((size_t)r.b * Lq + r.t) * n_h + g * G + e) * DH + d;
+                    const float v = den[e] > 0.f ? acc[e] / den[e] * fast_sigmoid(__bfloat162float(g1[at])) : 0.f;
+                    out[at] = __float2bfloat16_rn(v);
+                }
             }
         }
-    }
-#pragma unroll
-    for (int e = 0; e < G; ++e) {
-        const size_t at = (((size_t)r.b * Lq + r.t) * n_h + g * G + e) * DH + d;
-        const float v = den[e] > 0.f ? acc[e] / den[e] * fast_sigmoid(__bfloat162float(g1[at])) : 0.f;
-        out[at] = __float2bfloat16_rn(v);
-    }
     }
 }
 
@@ -524,7 +560,7 @@ cudaError_t launch_attn_t(AttnArgs a, const gsa_params_t& p, const AttnPlan& pl,
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     const int fin_threads = a.n_kv * DH < 1024 ? a.n_kv * DH : 1024;
-    gsa_attn_finalize_kernel<DH, G><<<(unsigned)rr_all.rows(), fin_threads, 0, st>>>(
+    gsa_attn_finalize_kernel<DH, G><<<(unsigned)((rr_all.rows() + kFinRows - 1) / kFinRows), fin_threads, 0, st>>>(
         a.state, a.kt, g1, out, rr_all, a.il, a.idx_rows, p.Lq, p.n_h, p.n_kv, p.k_max, pl.mode, pl.slots);
     ++g_launches;
     return cudaGetLastError();

@@ -5,12 +5,15 @@
 //   0  a sample of the row (256 chunks of 32 consecutive scores, evenly spread) is histogrammed;
 //      it gives a threshold key tau that about 1.3 * min(k_max, n) scores of the row should reach
 //      (k_t itself is not known yet: it depends on the variance of the whole row)
-//   1  full read: fp64 sum and sum of squares of every score; every position whose key reaches tau
-//      is appended, in position order, to a candidate list in shared memory (a few percent of the row)
-//      -> Var, k_t
+//   1  full read, no block-wide barrier: the row is cut into at most 512 chunks (512 scores each, or
+//      512 * 2^s for very long rows) that are dealt to the 16 warps round-robin, so each warp sees an
+//      even sample of the row.  Loads are fully coalesced float4s; every score goes into fp64 sum and
+//      sum of squares; a score that reaches tau (one float compare) is appended, in position order, to
+//      the warp's private candidate list in shared memory, and each chunk remembers where its entries
+//      start and how many it has.   -> Var, k_t
 //   2  on chip: radix rounds over the candidates give the exact threshold key T of the k_t-th largest
-//      score and how many keys equal to T are taken; one ordered compaction of the list writes S_t
-//      ascending.
+//      score and how many keys equal to T are taken; the chunks are then walked in position order
+//      (counts per chunk, one block scan, ballot-ordered emission) to write S_t ascending.
 // Equal keys go to the lower position, so the output is unique.  If the list overflows or comes out
 // shorter than k_t (the sample misjudged the row: huge ties, scores sorted by position, ...) the CTA
 // falls back to radix rounds over the whole row in global memory: slower, same result.
@@ -27,8 +30,9 @@ constexpr int kBins = 1 << kBinsLog2;
 constexpr int kBinsPerThread = kBins / kSelThreads;   // 8
 constexpr int kListCap = 8192;                        // entries of the candidate list
 constexpr int kListPerThread = kListCap / kSelThreads;  // 16
-constexpr int kChunkPerThread = 16;                   // consecutive elements per thread and chunk
-constexpr int kChunk = kSelThreads * kChunkPerThread;
+constexpr int kWarpCap = kListCap / kSelWarps;        // entries of one warp's private list: 512
+constexpr int kIterElems = 512;                       // scores one warp iteration covers (4 float4 per lane)
+constexpr int kMaxChunks = 512;
 constexpr int kSampleChunks = 256;                    // sample = 256 chunks of 32 scores
 constexpr int kSamplePerThread = kSampleChunks * 32 / kSelThreads;   // 16
 
@@ -62,6 +66,11 @@ struct SelShared {
     uint32_t warp_tot[2][kSelWarps];
     uint32_t seg_gt[kSelWarps];
     uint32_t seg_eq[kSelWarps];
+    uint16_t ch_off[kMaxChunks];      // chunk c: its entries start at list[(c % 16) * kWarpCap + ch_off[c]]
+    uint16_t ch_cnt[kMaxChunks];      //          and there are ch_cnt[c] of them
+    uint16_t ch_gt[kMaxChunks];       // selected entries of the chunks before c: keys > T ...
+    uint16_t ch_eq[kMaxChunks];       // ... and keys == T (before the cut at need_eq)
+    uint32_t wl_cnt[kSelWarps];       // live entries of each warp's list
     uint32_t found_bin;
     uint32_t found_above;
     uint32_t overflow;
@@ -222,58 +231,92 @@ __global__ void __launch_bounds__(kSelThreads, 2) gsa_select_kernel(const Select
     }
     __syncthreads();
 
-    // ---- pass 1: fp64 moments of every score; ordered list of the candidates ----------------
+    // ---- pass 1: fp64 moments of every score; per-warp ordered lists of the candidates ---------
+    // tau as a float: x >= tau_f  <=>  order_key(x) >= tau for every non-NaN x
+    // (tau == 0, "keep everything", has no float counterpart: use -inf)
+    const float tau_f = tau == 0u ? -INFINITY : __uint_as_float((tau & 0x80000000u) ? (tau & 0x7FFFFFFFu) : ~tau);
+    int cshift = 0;                                           // chunk = kIterElems << cshift scores
+    while (((int64_t)n + ((int64_t)kIterElems << cshift) - 1) / ((int64_t)kIterElems << cshift) > kMaxChunks) ++cshift;
+    const int chunk_elems = kIterElems << cshift;
+    const int nchunks = (n + chunk_elems - 1) / chunk_elems;
     double s1 = 0.0, s2 = 0.0;
-    uint32_t base = 0;
-    {
-        int slot = 0;
-        for (int c0 = 0; c0 < n; c0 += kChunk, slot ^= 1) {
-            const int i0 = c0 + tid * kChunkPerThread;
-            uint32_t keys[kChunkPerThread];
-            uint32_t flags = 0;
-            if (i0 + kChunkPerThread <= n) {
+    uint32_t wcnt = 0;                                        // entries in this warp's list (warp-uniform)
+    bool w_over = false;
+    uint32_t* const wl_idx = sh.list_idx + wid * kWarpCap;
+    uint32_t* const wl_key = sh.list_key + wid * kWarpCap;
+    for (int c = wid; c < nchunks; c += kSelWarps) {
+        const uint32_t c_start = wcnt;
+        const int c_lo = c * chunk_elems, c_hi = min(n, c_lo + chunk_elems);
+        for (int i0 = c_lo; i0 < c_hi; i0 += kIterElems) {
+            float xs[16];
+            if (i0 + kIterElems <= c_hi) {
 #pragma unroll
-                for (int v = 0; v < kChunkPerThread / 4; ++v) {
-                    const float4 x4 = __ldg(reinterpret_cast<const float4*>(grow + i0) + v);
-                    const float xs[4] = {x4.x, x4.y, x4.z, x4.w};
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const double xd = (double)xs[e];
-                        s1 += xd;
-                        s2 = fma(xd, xd, s2);
-                        keys[v * 4 + e] = order_key(xs[e]);
-                        flags |= (keys[v * 4 + e] >= tau ? 1u : 0u) << (v * 4 + e);
-                    }
+                for (int v = 0; v < 4; ++v) {
+                    const float4 x4 = __ldg(reinterpret_cast<const float4*>(grow + i0) + v * 32 + lane);
+                    xs[v * 4] = x4.x; xs[v * 4 + 1] = x4.y; xs[v * 4 + 2] = x4.z; xs[v * 4 + 3] = x4.w;
                 }
             } else {
 #pragma unroll
-                for (int e = 0; e < kChunkPerThread; ++e) {
-                    keys[e] = 0u;
-                    if (i0 + e < n) {
-                        const float x = __ldg(grow + i0 + e);
-                        const double xd = (double)x;
-                        s1 += xd;
-                        s2 = fma(xd, xd, s2);
-                        keys[e] = order_key(x);
-                        flags |= (keys[e] >= tau ? 1u : 0u) << e;
-                    }
+                for (int e = 0; e < 16; ++e) {
+                    const int i = i0 + ((e >> 2) * 32 + lane) * 4 + (e & 3);
+                    xs[e] = i < c_hi ? __ldg(grow + i) : __int_as_float(0x7FC00000);   // NaN: never a candidate
                 }
             }
-            uint32_t total;
-            uint32_t pos = base + block_excl_scan(sh, __popc(flags), slot, total);
-            if (base + total <= (uint32_t)kListCap) {
+            uint32_t flags = 0;
+            const bool full = i0 + kIterElems <= c_hi;
 #pragma unroll
-                for (int e = 0; e < kChunkPerThread; ++e)
-                    if (flags & (1u << e)) {
-                        sh.list_idx[pos] = (uint32_t)(i0 + e);
-                        sh.list_key[pos] = keys[e];
-                        ++pos;
-                    }
-            } else if (tid == 0) {
-                sh.overflow = 1u;                             // block-uniform condition
+            for (int e = 0; e < 16; ++e) {
+                const double xd = (double)xs[e];
+                if (full || i0 + ((e >> 2) * 32 + lane) * 4 + (e & 3) < c_hi) {
+                    s1 += xd;
+                    s2 = fma(xd, xd, s2);
+                }
+                flags |= (xs[e] >= tau_f ? 1u : 0u) << e;
             }
-            base += total;
+            if (__any_sync(0xFFFFFFFFu, flags != 0u)) {
+                // position order inside the iteration is (v, lane, e): one packed scan gives, for each of
+                // the four float4 rounds v, how many candidates the lower lanes hold
+                uint32_t packed = __popc(flags & 0xFu) | (__popc(flags & 0xF0u) << 8) |
+                                  (__popc(flags & 0xF00u) << 16) | (__popc(flags & 0xF000u) << 24);
+                uint32_t inc = packed;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+                    if (lane >= o) inc += u;
+                }
+                const uint32_t tot = __shfl_sync(0xFFFFFFFFu, inc, 31);     // per-v totals, one byte each
+                const uint32_t excl = inc - packed;
+                const uint32_t iter_total = (tot & 0xFFu) + ((tot >> 8) & 0xFFu) + ((tot >> 16) & 0xFFu) + (tot >> 24);
+                if (wcnt + iter_total <= (uint32_t)kWarpCap) {
+                    uint32_t vbase = wcnt;
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        uint32_t pos = vbase + ((excl >> (8 * v)) & 0xFFu);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            if (flags & (1u << (v * 4 + e))) {
+                                // the score is read again (L1) so that xs[] need not stay live
+                                const int i = i0 + (v * 32 + lane) * 4 + e;
+                                wl_idx[pos] = (uint32_t)i;
+                                wl_key[pos] = order_key(__ldg(grow + i));
+                                ++pos;
+                            }
+                        vbase += (tot >> (8 * v)) & 0xFFu;
+                    }
+                } else {
+                    w_over = true;
+                }
+                wcnt += iter_total;
+            }
         }
+        if (lane == 0) {
+            sh.ch_off[c] = (uint16_t)min(c_start, (uint32_t)kWarpCap);
+            sh.ch_cnt[c] = (uint16_t)min(wcnt - c_start, (uint32_t)kWarpCap);
+        }
+    }
+    if (lane == 0) {
+        if (w_over) sh.overflow = 1u;
+        sh.wl_cnt[wid] = min(wcnt, (uint32_t)kWarpCap);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -314,43 +357,73 @@ __global__ void __launch_bounds__(kSelThreads, 2) gsa_select_kernel(const Select
         return;
     }
 
-    const int m = (int)base;                    // candidates found (all of them listed unless overflow)
+    int m = 0;                                  // candidates found (all of them listed unless overflow)
+    for (int w = 0; w < kSelWarps; ++w) m += (int)sh.wl_cnt[w];
     uint32_t T, need_eq;
     if (!overflow && m >= k) {
-        // ---- exact threshold among the candidates ---------------------------------------------
+        // ---- exact threshold among the candidates (the 16 warp lists, padded to kWarpCap) -------
+        // slot i of the padded array belongs to warp i / kWarpCap and is live below that warp's count
         uint32_t cmin = 0xFFFFFFFFu, cmax = 0u;
-        for (int i = tid; i < m; i += kSelThreads) {
-            const uint32_t key = sh.list_key[i];
-            cmin = min(cmin, key); cmax = max(cmax, key);
-        }
+        for (int i = tid; i < kListCap; i += kSelThreads)
+            if ((uint32_t)(i & (kWarpCap - 1)) < sh.wl_cnt[i / kWarpCap]) {
+                const uint32_t key = sh.list_key[i];
+                cmin = min(cmin, key); cmax = max(cmax, key);
+            }
         block_minmax(sh, cmin, cmax);
-        radix_rounds(sh, m, [&](int i) { return sh.list_key[i]; }, cmin, cmax, (uint32_t)k, T, need_eq);
+        // dead slots read as a key outside [cmin, cmax], which no round counts
+        const uint32_t dead = cmin > 0u ? cmin - 1u : cmax + 1u;
+        radix_rounds(sh, kListCap, [&](int i) -> uint32_t {
+            return (uint32_t)(i & (kWarpCap - 1)) < sh.wl_cnt[i / kWarpCap] ? sh.list_key[i] : dead;
+        }, cmin, cmax, (uint32_t)k, T, need_eq);
 
-        // ---- ordered compaction of the list into S_t ----------------------------------------
-        uint32_t gt = 0, eq = 0;
-        const int j0 = tid * kListPerThread;
-#pragma unroll
-        for (int e = 0; e < kListPerThread; ++e)
-            if (j0 + e < m) {
-                const uint32_t key = sh.list_key[j0 + e];
-                gt += key > T;
-                eq += key == T;
+        // ---- emission in position order: chunk by chunk ---------------------------------------
+        // (a) per chunk: how many of its entries are above T / equal to T
+        for (int c = wid; c < nchunks; c += kSelWarps) {
+            const uint32_t off = (uint32_t)(c & (kSelWarps - 1)) * kWarpCap + sh.ch_off[c];
+            const int cnt = sh.ch_cnt[c];
+            uint32_t g = 0, q = 0;
+            for (int j = lane; j < cnt; j += 32) {
+                const uint32_t key = sh.list_key[off + j];
+                g += key > T;
+                q += key == T;
             }
-        uint32_t total;
-        const uint32_t packed = block_excl_scan(sh, (eq << 16) | gt, 0, total);
-        uint32_t g_before = packed & 0xFFFFu, e_before = packed >> 16;
 #pragma unroll
-        for (int e = 0; e < kListPerThread; ++e)
-            if (j0 + e < m) {
-                const uint32_t key = sh.list_key[j0 + e];
-                if (key > T) {
-                    out_idx[g_before + min(e_before, need_eq)] = (int32_t)sh.list_idx[j0 + e];
-                    ++g_before;
-                } else if (key == T) {
-                    if (e_before < need_eq) out_idx[g_before + e_before] = (int32_t)sh.list_idx[j0 + e];
-                    ++e_before;
-                }
+            for (int o = 16; o > 0; o >>= 1) {
+                g += __shfl_xor_sync(0xFFFFFFFFu, g, o);
+                q += __shfl_xor_sync(0xFFFFFFFFu, q, o);
             }
+            if (lane == 0) { sh.ch_gt[c] = (uint16_t)g; sh.ch_eq[c] = (uint16_t)q; }
+        }
+        __syncthreads();
+        // (b) exclusive prefix over the chunks (thread c owns chunk c)
+        {
+            const uint32_t mine = tid < nchunks ? (((uint32_t)sh.ch_eq[tid] << 16) | sh.ch_gt[tid]) : 0u;
+            uint32_t total;
+            const uint32_t before = block_excl_scan(sh, mine, 0, total);
+            __syncthreads();
+            if (tid < nchunks) { sh.ch_gt[tid] = (uint16_t)(before & 0xFFFFu); sh.ch_eq[tid] = (uint16_t)(before >> 16); }
+        }
+        __syncthreads();
+        // (c) each warp writes its chunks; inside a chunk, ballots give the order
+        const uint32_t below = (1u << lane) - 1u;
+        for (int c = wid; c < nchunks; c += kSelWarps) {
+            const uint32_t off = (uint32_t)(c & (kSelWarps - 1)) * kWarpCap + sh.ch_off[c];
+            const int cnt = sh.ch_cnt[c];
+            uint32_t run_gt = sh.ch_gt[c], run_eq = sh.ch_eq[c];
+            for (int j0 = 0; j0 < cnt; j0 += 32) {
+                const int j = j0 + lane;
+                const bool in = j < cnt;
+                const uint32_t key = in ? sh.list_key[off + j] : 0u;
+                const bool gt = in && key > T, eq = in && key == T;
+                const uint32_t bg = __ballot_sync(0xFFFFFFFFu, gt), be = __ballot_sync(0xFFFFFFFFu, eq);
+                const uint32_t g_before = run_gt + __popc(bg & below);
+                const uint32_t e_before = run_eq + __popc(be & below);
+                if (gt || (eq && e_before < need_eq))
+                    out_idx[g_before + min(e_before, need_eq)] = (int32_t)sh.list_idx[off + j];
+                run_gt += __popc(bg);
+                run_eq += __popc(be);
+            }
+        }
     } else {
         // ---- fallback: radix rounds over the whole row, then ordered emission ----------------
         radix_rounds(sh, n, [&](int i) { return order_key(__ldg(grow + i)); }, 0u, 0xFFFFFFFFu,
