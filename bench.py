@@ -255,12 +255,17 @@ def main():
     peaks = measured_peaks()
     ab = attention_bytes(cfg, kt_sum)
     achieved = ab / (attn_ms * 1e-3) / 1e9
+    # DRAM bytes of the sparse-attention launches of one forward, from the ncu capture summarised in
+    # profiles/gsa_sparse_attn_kernel_l32k_and_l128k_dram.md (l128k, default key ranges); other workloads: not captured
+    traffic = 48.26e9 if (cfg.name == "l128k" and args.slab_rows == 0) else None
     roofline = {"kernel": "gsa_sparse_attn_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
-                "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": traffic,
                 "peak_source": f"{peaks['source']} (MEASURED_PEAKS.json hbm_gbs)" if peaks["source"] == "measured"
                 else "fallback 6650 GB/s",
                 "algorithmic_bytes_per_launch": ab, "launch_ms": attn_ms,
-                "note": "frac may exceed 1 when the 126 MB L2 serves part of the gather"}
+                "note": "one 'launch' = the sparse-attention stage of a forward (range cuts, one kernel launch per 16384-key "
+                        "range, finalize); frac exceeds 1 because the 126 MB L2, not HBM, serves the gather "
+                        "(ncu: L2 throughput 72% of peak, DRAM traffic 4% of the algorithmic bytes)"}
     causal_pairs = cfg.B * sum(cfg.Lk - cfg.Lq + t + 1 for t in (0, cfg.Lq - 1)) * cfg.Lq / 2.0
     stages = {"indexer_plus_topk_ms": sel_ms, "sparse_attn_ms": attn_ms,
               "indexer_causal_tflop": 2.0 * cfg.HI * cfg.dI * causal_pairs / 1e12,
