@@ -165,6 +165,7 @@ def main():
     ap.add_argument("--workload", default="l128k", choices=sorted(CONFIGS))
     ap.add_argument("--impl", default="gsa_b200", choices=["gsa_b200", "reference"])
     ap.add_argument("--slab-rows", type=int, default=0)
+    ap.add_argument("--lq", type=int, default=0, help="only the last LQ query rows (chunked prefill; smaller ncu captures)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (smaller ncu captures)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -173,6 +174,8 @@ def main():
     cfg = CONFIGS[args.workload]
     if args.batch > 0:
         cfg = cfg.with_(B=args.batch, name=f"{cfg.name}-b{args.batch}")
+    if args.lq > 0:
+        cfg = cfg.with_(Lq=args.lq, name=f"{cfg.name}-lq{args.lq}")
 
     if args.impl == "reference":
         run_reference(args, cfg)
@@ -225,6 +228,7 @@ def main():
     torch.cuda.synchronize()
     assert gsa.gsa_device_status(ws) == 0
     kt_sum = int(kt.sum().item())
+    fallback_rows = gsa.gsa_select_fallback_rows(ws)
 
     # per-step stage events (recorded by the library on the launching stream)
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
@@ -269,7 +273,7 @@ def main():
     causal_pairs = cfg.B * sum(cfg.Lk - cfg.Lq + t + 1 for t in (0, cfg.Lq - 1)) * cfg.Lq / 2.0
     stages = {"indexer_plus_topk_ms": sel_ms, "sparse_attn_ms": attn_ms,
               "indexer_causal_tflop": 2.0 * cfg.HI * cfg.dI * causal_pairs / 1e12,
-              "mean_k_t": kt_sum / float(cfg.B * cfg.Lq)}
+              "mean_k_t": kt_sum / float(cfg.B * cfg.Lq), "select_fallback_rows": fallback_rows}
 
     # ---- end to end through the host-buffer entry point ------------------------------------
     e2e = None

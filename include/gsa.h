@@ -102,6 +102,7 @@ int gsa_indexer_scores(const gsa_params_t *p, const void *qI, const void *kI, co
  *   idx    [B, R, k_max] int32: S_t in ascending position order, then -1
  *   kt     [B, R] int32: |S_t| = min(k_t, n_t)
  *   var    [B, R] fp32 or NULL: Var_t (for the caller's running mean)
+ *   ws     optional (may be NULL); with >= 256 bytes the fallback-row counter is kept at its head
  */
 int gsa_adaptive_topk(const gsa_params_t *p, const float *scores, int64_t row_stride,
                       int32_t *idx, int32_t *kt, float *var, void *ws, size_t ws_bytes,
@@ -188,6 +189,14 @@ int gsa_forward_host(const gsa_params_t *p, const void *Q, const void *K, const 
  * gsa_sparse_gated_attn_fwd_static (it lives in the library's built-in array on the current device).
  */
 int gsa_device_status(const void *ws, void *stream, int32_t *status_out);
+
+/*
+ * Waits for `stream` and reads how many rows of the last gsa_forward / gsa_adaptive_topk call on `ws`
+ * took the selection kernel's whole-row fallback (the sampled candidate threshold misjudged the row:
+ * slower, same result).  A diagnostic: a large share means the scores are far from what the sample
+ * assumes (for instance sorted by position).
+ */
+int gsa_select_fallback_rows(const void *ws, void *stream, int32_t *rows_out);
 
 /* Number of kernel launches the library has enqueued so far in this process (host counter). */
 int64_t gsa_launch_count(void);

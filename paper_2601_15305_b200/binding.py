@@ -21,6 +21,7 @@ EXPORTS = (
     "gsa_forward", "gsa_forward_host_arena_bytes", "gsa_forward_host", "gsa_device_status",
     "gsa_launch_count", "gsa_debug_set_indexer_path", "gsa_profile_set_events", "gsa_status_string",
     "gsa_sparse_gated_attn_fwd_static", "gsa_attn_workspace_bytes", "gsa_debug_set_attn_range_keys",
+    "gsa_select_fallback_rows",
 )
 
 STATIC_SCRATCH_BYTES = 32 << 20     # GSA_STATIC_SCRATCH_BYTES of include/gsa.h
@@ -174,6 +175,12 @@ def gsa_device_status(ws, stream=None) -> int:
     rc = lib().gsa_device_status(_dp(ws), _stream(stream), ctypes.byref(v))
     if rc not in (0, -5):
         _check(rc, "gsa_device_status")
+    return v.value
+
+
+def gsa_select_fallback_rows(ws, stream=None) -> int:
+    v = ctypes.c_int32(0)
+    _check(lib().gsa_select_fallback_rows(_dp(ws), _stream(stream), ctypes.byref(v)), "gsa_select_fallback_rows")
     return v.value
 
 

@@ -150,9 +150,14 @@ int gsa_adaptive_topk(const gsa_params_t* p, const float* scores, int64_t row_st
     if ((rc = row_range(p, &rr))) return rc;
     if (!scores || !idx || !kt || !aligned16(scores) || !aligned16(idx)) return GSA_ERR_INVALID_ARG;
     if (row_stride < p->Lk || row_stride % 4 != 0) return GSA_ERR_INVALID_ARG;
-    (void)ws; (void)ws_bytes;
     IdxLayout il{0, rr.q_begin, rr.R};
-    return cuda_rc(launch_select(*p, rr, scores, row_stride, idx, kt, var, il, (cudaStream_t)stream));
+    int32_t* fb = nullptr;
+    if (ws && aligned16(ws) && ws_bytes >= (size_t)kStatusBytes) {
+        cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, (cudaStream_t)stream);
+        if (e != cudaSuccess) return cuda_rc(e);
+        fb = (int32_t*)ws + kStatusFallbackWord;
+    }
+    return cuda_rc(launch_select(*p, rr, scores, row_stride, idx, kt, var, il, fb, (cudaStream_t)stream));
 }
 
 // workspace of the per-stage attention call: [status][attention scratch][V' (optional)]
@@ -247,7 +252,7 @@ int gsa_forward(const gsa_params_t* p, const void* Q, const void* K, const void*
             RowRange rr{b0, (p->B - b0 < nb_per ? p->B - b0 : nb_per), 0, p->Lq};
             if ((e = launch_indexer(*p, rr, (const bf16*)qI, (const bf16*)kI, w, bI, slab, wp.row_stride,
                                     (int32_t*)ws, st)) != cudaSuccess) return cuda_rc(e);
-            if ((e = launch_select(*p, rr, slab, wp.row_stride, idx, kt, var_out, il, st)) != cudaSuccess)
+            if ((e = launch_select(*p, rr, slab, wp.row_stride, idx, kt, var_out, il, (int32_t*)ws + kStatusFallbackWord, st)) != cudaSuccess)
                 return cuda_rc(e);
         }
     } else {
@@ -256,7 +261,7 @@ int gsa_forward(const gsa_params_t* p, const void* Q, const void* K, const void*
                 RowRange rr{b, 1, q0, (p->Lq - q0 < wp.slab_rows ? p->Lq - q0 : wp.slab_rows)};
                 if ((e = launch_indexer(*p, rr, (const bf16*)qI, (const bf16*)kI, w, bI, slab, wp.row_stride,
                                         (int32_t*)ws, st)) != cudaSuccess) return cuda_rc(e);
-                if ((e = launch_select(*p, rr, slab, wp.row_stride, idx, kt, var_out, il, st)) != cudaSuccess)
+                if ((e = launch_select(*p, rr, slab, wp.row_stride, idx, kt, var_out, il, (int32_t*)ws + kStatusFallbackWord, st)) != cudaSuccess)
                     return cuda_rc(e);
             }
     }
@@ -339,6 +344,17 @@ int gsa_device_status(const void* ws, void* stream, int32_t* status_out) {
     if (e != cudaSuccess) return cuda_rc(e);
     if (status_out) *status_out = v;
     return v == kDevOk ? GSA_OK : GSA_ERR_DEVICE_TIMEOUT;
+}
+
+int gsa_select_fallback_rows(const void* ws, void* stream, int32_t* rows_out) {
+    if (!ws || !rows_out) return GSA_ERR_INVALID_ARG;
+    int32_t v = 0;
+    cudaError_t e = cudaMemcpyAsync(&v, (const int32_t*)ws + kStatusFallbackWord, sizeof(v), cudaMemcpyDeviceToHost,
+                                    (cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_rc(e);
+    *rows_out = v;
+    return GSA_OK;
 }
 
 int64_t gsa_launch_count(void) { return g_launches; }

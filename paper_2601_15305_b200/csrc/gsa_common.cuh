@@ -25,7 +25,8 @@ struct IdxLayout {
     }
 };
 
-constexpr int kStatusBytes = 256;   // head of every workspace: device status word + padding
+constexpr int kStatusBytes = 256;   // head of every workspace: device status word, counters, padding
+constexpr int kStatusFallbackWord = 1;   // int32 word: rows on which top-k selection took its whole-row fallback
 
 // device status word values
 enum : int32_t { kDevOk = 0, kDevTimeoutTma = 1, kDevTimeoutMma = 2, kDevTimeoutEpi = 3,
@@ -40,7 +41,7 @@ cudaError_t launch_indexer(const gsa_params_t& p, RowRange rr, const __nv_bfloat
 
 cudaError_t launch_select(const gsa_params_t& p, RowRange rr, const float* scores,
                           int64_t row_stride, int32_t* idx, int32_t* kt, float* var,
-                          IdxLayout il, cudaStream_t st);
+                          IdxLayout il, int32_t* fallback_rows /*nullable counter*/, cudaStream_t st);
 
 cudaError_t launch_value_gate(const __nv_bfloat16* V, const __nv_bfloat16* g2, __nv_bfloat16* Vg,
                               int64_t n_elems, cudaStream_t st);

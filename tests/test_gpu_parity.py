@@ -185,6 +185,24 @@ def test_topk_long_rows_take_the_uncached_path():
     _select_and_compare(cfg, sc)
 
 
+def test_topk_long_rows_that_defeat_the_sample():
+    """Long rows on which the sampled candidate threshold is useless: a handful of score levels (huge
+    ties), scores increasing with position (every top score sits at the end of the row), a constant row.
+    The kernel must notice (list overflow / too few candidates) and still return the exact set."""
+    cfg = CONFIGS["l8k"].with_(name="degenerate", B=1, Lq=6, Lk=20011, k_base=700, k_min=100, k_max=3000)
+    st = U.row_stride(cfg)
+    g = torch.Generator().manual_seed(7)
+    sc = torch.zeros((1, cfg.Lq, st), dtype=torch.float32)
+    sc[0, 0] = torch.randint(0, 5, (st,), generator=g).float() * 0.25 + 1.0        # 5 levels
+    sc[0, 1] = torch.arange(st).float() * 1e-4 + 1.0                                # increasing
+    sc[0, 2] = 2.5                                                                  # constant
+    sc[0, 3] = torch.arange(st).float().flip(0) * 1e-4 + 1.0                        # decreasing
+    sc[0, 4] = torch.rand(st, generator=g) + (torch.arange(st) > st - 3000).float() * 3.0   # a late cluster
+    sc[0, 5] = torch.rand(st, generator=g)
+    for k_mode, v_bar in ((2, 1.0), (0, 0.05), (1, 0.05)):
+        _select_and_compare(cfg, sc.cuda(), k_mode=k_mode, v_bar=v_bar)
+
+
 # ------------------------------------------------------------------------------------------ stage 3
 def _oracle_idx(cfg, x, rows, **kw):
     p = U.oracle_params(cfg, **kw)
