@@ -36,7 +36,7 @@ def build(force: bool = False) -> str:
 class _P(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("B", "Lq", "Lk", "n_h", "n_kv", "d_h", "HI", "dI", "k_base", "k_min", "k_max", "k_mode")] + \
-               [("v_bar", ctypes.c_double), ("sm_scale", ctypes.c_double)]
+               [("v_bar", ctypes.c_double), ("sm_scale", ctypes.c_double), ("act", ctypes.c_int32)]
 
 
 @dataclass
@@ -55,6 +55,7 @@ class OracleParams:
     k_mode: int = 0
     v_bar: float = 1.0
     sm_scale: float = 0.0
+    act: int = 0          # 0: sigmoid indexer (Eq. 7), 1: ReLU indexer (Eq. 3)
 
     @classmethod
     def from_config(cls, cfg, **kw) -> "OracleParams":
@@ -65,7 +66,8 @@ class OracleParams:
 
     def c(self) -> _P:
         return _P(self.B, self.Lq, self.Lk, self.n_h, self.n_kv, self.d_h, self.HI, self.dI,
-                  self.k_base, self.k_min, self.k_max, self.k_mode, float(self.v_bar), float(self.sm_scale))
+                  self.k_base, self.k_min, self.k_max, self.k_mode, float(self.v_bar), float(self.sm_scale),
+                  int(self.act))
 
     def visible(self, t: int) -> int:
         return self.Lk - self.Lq + t + 1

@@ -10,6 +10,7 @@
  *
  * Steps, in the paper's order:
  *   Eq. 7   gated lightning indexer     I[t,s] = sum_j w[t,j] * sigmoid(q^I[t,j] . k^I[s] + b_j)
+ *           (act = 1: the ReLU indexer of Eq. 3 that Eq. 7 replaces, sum_j w[t,j] * max(q^I.k^I + b_j, 0))
  *   Eq. 8   adaptive budget             k_t = clamp(floor(k_base * Var(I[t,:]) / Vbar), k_min, k_max)
  *   Eq. 4   top-k_t selection           S_t = the k_t positions with the largest I[t,s]
  *   Eq. 9   value gate G2               V'[s] = V[s] * sigmoid(g2[s])      (elementwise)
@@ -29,7 +30,8 @@
  * Pins (tests/test_oracle_pins.py): closed-form sigmoid values on one-hot inputs,
  * the reflection identity I(q)+I(-q)=sum_j w_j, the open range (0, sum w), two-valued
  * rows with known variance, clamp edges, monotonicity per mode, brute-force top-k
- * with exact ties, reduction to library softmax attention when S_t is everything
+ * with exact ties (ReLU variant: positive homogeneity, I(q) - I(-q) linear in q), reduction to
+ * library softmax attention when S_t is everything
  * and gates are saturated, single-key and equal-logit closed forms, g1 = -40 -> 0.
  * Parity unpinned: nothing (every function above has at least one such pin); the
  * absolute values on random data have no printed reference in the paper.
@@ -50,6 +52,7 @@ typedef struct {
     int32_t k_mode;
     double v_bar;
     double sm_scale; /* <= 0: 1/sqrt(d_h) */
+    int32_t act;     /* 0: sigmoid (Eq. 7), 1: ReLU (Eq. 3) */
 } gsa_oracle_params;
 
 static double sigmoid_d(double x) { return 1.0 / (1.0 + exp(-x)); }
@@ -77,7 +80,7 @@ void gsa_oracle_score_row(const gsa_oracle_params *p, const float *qI_t, const f
             double x = bI ? (double)bI[j] : 0.0;
             for (int c = 0; c < p->dI; ++c)
                 x += (double)qI_t[j * p->dI + c] * (double)kI_b[(size_t)s * p->dI + c];
-            acc += (double)w_t[j] * sigmoid_d(x);
+            acc += (double)w_t[j] * (p->act == 1 ? (x > 0.0 ? x : 0.0) : sigmoid_d(x));
         }
         I_row[s] = acc;
     }

@@ -88,6 +88,39 @@ def test_indexer_reflection_and_range():
         assert np.isnan(a[i, n:]).all()
 
 
+def test_relu_indexer_closed_form_homogeneity_and_linearity():
+    """The ReLU indexer of Eq. 3 (act = 1).  One-hot inputs give max(x, 0) exactly; scaling the queries by
+    a > 0 scales the scores by a (a sigmoid indexer would not); ReLU(x) - ReLU(-x) = x makes
+    I(q) - I(-q) = sum_j w_j (q_j . k), which a library matmul gives."""
+    p = small_params(Lq=1, Lk=3, HI=2, dI=4, act=1)
+    qI = np.zeros((1, 1, 2, 4), np.float32)
+    qI[0, 0, 0, 2] = 2.0          # head 0 reads component 2, doubled
+    qI[0, 0, 1, 0] = -1.0         # head 1 reads component 0, negated
+    kI = np.array([[[0.5, 9.0, 1.5, 9.0], [-2.0, 9.0, -1.0, 9.0], [0.0, 9.0, 0.25, 9.0]]], np.float32)
+    w = np.array([[[0.5, 0.25]]], np.float32)
+    sc = oracle.scores(p, qI, kI, w, None, rows_t=[0])
+    # key 0: 0.5*max(3,0) + 0.25*max(-0.5,0);  key 1: 0.5*max(-2,0) + 0.25*max(2,0);  key 2: 0.5*0.5 + 0
+    np.testing.assert_allclose(sc[0, :3], [1.5, 0.5, 0.25], rtol=0, atol=1e-15)
+    b = np.array([-1.0, 0.75], np.float32)                     # bias inside the ReLU
+    scb = oracle.scores(p, qI, kI, w, b, rows_t=[0])
+    np.testing.assert_allclose(scb[0, :3], [0.5 * 2.0 + 0.25 * 0.25, 0.25 * 2.75, 0.25 * 0.75], atol=1e-15)
+
+    cfg = CONFIGS["tiny"]
+    x = make_inputs(cfg)
+    pr = OracleParams.from_config(cfg, act=1)
+    rows = [3, 200, 511]
+    q = x["qI"].float().numpy()
+    s1 = oracle.scores(pr, q, x["kI"], x["w"], None, rows)
+    s4 = oracle.scores(pr, 4.0 * q, x["kI"], x["w"], None, rows)
+    sm = oracle.scores(pr, -q, x["kI"], x["w"], None, rows)
+    lin = torch.einsum("tjc,sc->tjs", x["qI"][0].double(), x["kI"][0].double())
+    lin = (x["w"][0].double()[:, :, None] * lin).sum(1).numpy()
+    for i, t in enumerate(rows):
+        np.testing.assert_allclose(s4[i, :t + 1], 4.0 * s1[i, :t + 1], rtol=1e-13)
+        np.testing.assert_allclose(s1[i, :t + 1] - sm[i, :t + 1], lin[t, :t + 1], rtol=0, atol=1e-12)
+        assert (s1[i, :t + 1] >= 0).all()
+
+
 def test_indexer_matches_library_matmul():
     """The contraction inside the sigmoid is an ordinary matrix product: compare with
     torch's fp64 einsum + library sigmoid on random data (an independent routine)."""
