@@ -165,6 +165,9 @@ def main():
     ap.add_argument("--workload", default="l128k", choices=sorted(CONFIGS))
     ap.add_argument("--impl", default="gsa_b200", choices=["gsa_b200", "reference"])
     ap.add_argument("--slab-rows", type=int, default=0)
+    ap.add_argument("--act", default="sigmoid", choices=["sigmoid", "relu"], help="indexer activation (Eq. 7 / Eq. 3)")
+    ap.add_argument("--k-mode", type=int, default=0, choices=[0, 1, 2], help="0 Eq. 8, 1 inverse, 2 fixed k = k_base")
+    ap.add_argument("--k-base", type=int, default=0, help="override the base budget (k sweep)")
     ap.add_argument("--lq", type=int, default=0, help="only the last LQ query rows (chunked prefill; smaller ncu captures)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (smaller ncu captures)")
     ap.add_argument("--no-e2e", action="store_true")
@@ -176,6 +179,11 @@ def main():
         cfg = cfg.with_(B=args.batch, name=f"{cfg.name}-b{args.batch}")
     if args.lq > 0:
         cfg = cfg.with_(Lq=args.lq, name=f"{cfg.name}-lq{args.lq}")
+    if args.k_base > 0:
+        cfg = cfg.with_(k_base=args.k_base, name=f"{cfg.name}-k{args.k_base}")
+    variant = dict(act=1 if args.act == "relu" else 0, k_mode=args.k_mode)
+    if variant != dict(act=0, k_mode=0):
+        cfg = cfg.with_(name=f"{cfg.name}-{args.act}-kmode{args.k_mode}")
 
     if args.impl == "reference":
         run_reference(args, cfg)
@@ -207,7 +215,7 @@ def main():
         x = make_inputs(cfg)
         d = {k: v.cuda() for k, v in x.items()}
         x_cpu_sample = x
-    p = gsa.make_params(cfg)
+    p = gsa.make_params(cfg, **variant)
     out = torch.empty_like(d["Q"])
     kt = torch.empty((cfg.B, cfg.Lq), dtype=torch.int32, device="cuda")
     ws = torch.empty(gsa.gsa_workspace_bytes(p, args.slab_rows), dtype=torch.uint8, device="cuda")

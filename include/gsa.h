@@ -67,6 +67,8 @@ typedef struct gsa_params {
     float sm_scale;     /* softmax scale of Eq. 11; <= 0 means 1/sqrt(d_h)                   */
     int32_t q_begin;    /* per-stage calls process query rows q_begin <= t < q_end of every  */
     int32_t q_end;      /* batch element; q_end <= 0 means Lq.  gsa_forward ignores both.    */
+    int32_t act;        /* indexer activation: 0 = sigmoid (Eq. 7, GSA); 1 = ReLU (Eq. 3, the
+                           lightning indexer GSA starts from; scores are then unbounded above) */
 } gsa_params_t;
 
 /*
@@ -79,7 +81,8 @@ int gsa_workspace_bytes(const gsa_params_t *p, int32_t slab_rows, size_t *bytes)
 
 /*
  * Gated lightning indexer, Eq. 7:
- *     I[t,s] = sum_j w[t,j] * sigmoid(qI[t,j,:] . kI[s,:] + bI[j]),   s visible to t.
+ *     I[t,s] = sum_j w[t,j] * sigmoid(qI[t,j,:] . kI[s,:] + bI[j]),   s visible to t
+ *   (p->act == 1: max(., 0) in place of the sigmoid, Eq. 3).
  *   qI     [B, Lq, HI, dI] bf16        kI  [B, Lk, dI] bf16 (one key shared by all heads)
  *   w      [B, Lq, HI]     fp32, the already-activated head weights sigmoid(h_t W^Iw_j)
  *   bI     [HI] fp32 or NULL (= zeros)

@@ -35,18 +35,18 @@ class gsa_params_t(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("B", "Lq", "Lk", "n_h", "n_kv", "d_h", "HI", "dI", "k_base", "k_min", "k_max", "k_mode")] + \
                [("v_bar", ctypes.c_float), ("sm_scale", ctypes.c_float),
-                ("q_begin", ctypes.c_int32), ("q_end", ctypes.c_int32)]
+                ("q_begin", ctypes.c_int32), ("q_end", ctypes.c_int32), ("act", ctypes.c_int32)]
 
 
 def make_params(cfg: GsaConfig = None, *, k_mode: int = 0, sm_scale: float = 0.0, q_begin: int = 0,
-                q_end: int = 0, **over) -> gsa_params_t:
+                q_end: int = 0, act: int = 0, **over) -> gsa_params_t:
     f = dict(B=1, Lq=1, Lk=1, n_h=1, n_kv=1, d_h=64, HI=1, dI=32, k_base=1, k_min=1, k_max=1, v_bar=1.0)
     if cfg is not None:
         f.update(B=cfg.B, Lq=cfg.Lq, Lk=cfg.Lk, n_h=cfg.n_h, n_kv=cfg.n_kv, d_h=cfg.d_h, HI=cfg.HI, dI=cfg.dI,
                  k_base=cfg.k_base, k_min=cfg.k_min, k_max=cfg.k_max, v_bar=cfg.v_bar)
     f.update(over)
     return gsa_params_t(f["B"], f["Lq"], f["Lk"], f["n_h"], f["n_kv"], f["d_h"], f["HI"], f["dI"], f["k_base"],
-                        f["k_min"], f["k_max"], k_mode, float(f["v_bar"]), float(sm_scale), q_begin, q_end)
+                        f["k_min"], f["k_max"], k_mode, float(f["v_bar"]), float(sm_scale), q_begin, q_end, act)
 
 
 _lib = None

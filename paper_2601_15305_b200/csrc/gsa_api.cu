@@ -51,6 +51,7 @@ int check_params(const gsa_params_t* p) {
     if (p->n_h % p->n_kv != 0) return GSA_ERR_INVALID_ARG;
     if (p->k_min < 1 || p->k_min > p->k_max || p->k_base < 1) return GSA_ERR_INVALID_ARG;
     if (p->k_mode < 0 || p->k_mode > 2) return GSA_ERR_INVALID_ARG;
+    if (p->act < 0 || p->act > 1) return GSA_ERR_INVALID_ARG;
     if (p->k_mode != 2 && !(p->v_bar > 0.f)) return GSA_ERR_INVALID_ARG;
     if (!one_of(p->d_h, {64, 128}) || !one_of(p->dI, {32, 64}) || !one_of(p->HI, {1, 2, 4, 8}))
         return GSA_ERR_UNSUPPORTED_SHAPE;

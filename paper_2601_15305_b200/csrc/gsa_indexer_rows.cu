@@ -27,6 +27,7 @@ struct RowsIdxArgs {
     RowRange rr;
     int32_t Lq, Lk;
     int32_t keys_per_cta;
+    int32_t act;
 };
 
 __device__ __forceinline__ void ldg32(const void* p, uint4& lo, uint4& hi) {
@@ -63,7 +64,7 @@ __global__ void __launch_bounds__(kRowsWarps * 32) gsa_indexer_rows_kernel(const
     for (int e = 0; e < 2; ++e) {
         const int h = 2 * tig + e;
         wv[e] = h < HI ? a.w[((size_t)b * a.Lq + t) * HI + h] : 0.f;
-        bv[e] = (a.bI && h < HI) ? a.bI[h] * -1.4426950408889634f : 0.f;
+        bv[e] = (a.bI && h < HI) ? a.bI[h] * (a.act == 1 ? 1.0f : -1.4426950408889634f) : 0.f;
     }
     const unsigned char* kbase = reinterpret_cast<const unsigned char*>(a.kI) + (size_t)b * a.Lk * DI * 2 +
                                  tig * (LANE_ELEMS * 2);
@@ -102,11 +103,15 @@ __global__ void __launch_bounds__(kRowsWarps * 32) gsa_indexer_rows_kernel(const
                 float v = 0.f;
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
-                    float ex, rc;
-                    const float arg = fminf(fmaf(s[hf * 2 + e], -1.4426950408889634f, bv[e]), 80.f);
-                    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(ex) : "f"(arg));
-                    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rc) : "f"(1.0f + ex));
-                    v = fmaf(wv[e], rc, v);
+                    if (a.act == 1) {                                     // Eq. 3: ReLU
+                        v = fmaf(wv[e], fmaxf(s[hf * 2 + e] + bv[e], 0.f), v);
+                    } else {
+                        float ex, rc;
+                        const float arg = fminf(fmaf(s[hf * 2 + e], -1.4426950408889634f, bv[e]), 80.f);
+                        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(ex) : "f"(arg));
+                        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rc) : "f"(1.0f + ex));
+                        v = fmaf(wv[e], rc, v);
+                    }
                 }
                 v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
                 v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
@@ -148,7 +153,7 @@ cudaError_t launch_indexer_rows(const gsa_params_t& p, RowRange rr, const __nv_b
     if (rr.rows() <= 0) return cudaSuccess;
     RowsIdxArgs a;
     a.qI = qI; a.kI = kI; a.w = w; a.bI = bI; a.scores = scores; a.row_stride = row_stride;
-    a.rr = rr; a.Lq = p.Lq; a.Lk = p.Lk; a.keys_per_cta = 0;
+    a.rr = rr; a.Lq = p.Lq; a.Lk = p.Lk; a.keys_per_cta = 0; a.act = p.act;
 #define GSA_ROWS_CASE(DI_, HI_) if (p.dI == DI_ && p.HI == HI_) return launch_rows_t<DI_, HI_>(p, rr, a, st)
     GSA_ROWS_CASE(64, 8); GSA_ROWS_CASE(64, 4); GSA_ROWS_CASE(64, 2); GSA_ROWS_CASE(64, 1);
     GSA_ROWS_CASE(32, 8); GSA_ROWS_CASE(32, 4); GSA_ROWS_CASE(32, 2); GSA_ROWS_CASE(32, 1);

@@ -20,7 +20,7 @@ struct SimpleIdxArgs {
     float* scores;
     int64_t row_stride;
     RowRange rr;
-    int32_t Lq, Lk, HI;
+    int32_t Lq, Lk, HI, act;
 };
 
 template <int DI>
@@ -71,7 +71,7 @@ __global__ void __launch_bounds__(kKeysPerCta) gsa_indexer_simple_kernel(const S
             float x = sb[j];
 #pragma unroll
             for (int c = 0; c < DI; ++c) x = fmaf(q[c], k[c], x);
-            acc = fmaf(sw[qi * HI + j], fast_sigmoid(x), acc);
+            acc = fmaf(sw[qi * HI + j], a.act == 1 ? fmaxf(x, 0.f) : fast_sigmoid(x), acc);
         }
         a.scores[((int64_t)bl * a.rr.R + tr0 + qi) * a.row_stride + s] = acc;
     }
@@ -85,7 +85,7 @@ cudaError_t launch_indexer_simple(const gsa_params_t& p, RowRange rr, const __nv
     if (rr.rows() <= 0) return cudaSuccess;
     SimpleIdxArgs a;
     a.qI = qI; a.kI = kI; a.w = w; a.bI = bI; a.scores = scores; a.row_stride = row_stride;
-    a.rr = rr; a.Lq = p.Lq; a.Lk = p.Lk; a.HI = p.HI;
+    a.rr = rr; a.Lq = p.Lq; a.Lk = p.Lk; a.HI = p.HI; a.act = p.act;
     const int n_max = p.Lk - p.Lq + rr.q_begin + rr.R;                 // visible keys of the last row
     dim3 grid((n_max + kKeysPerCta - 1) / kKeysPerCta,
               rr.nb * ((rr.R + kQueriesPerCta - 1) / kQueriesPerCta));

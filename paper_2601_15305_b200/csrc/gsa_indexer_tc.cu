@@ -123,8 +123,15 @@ __device__ __forceinline__ float rcp_approx(float x) {
 //   w1/a1 + w2/a2 = (w1 a2 + w2 a1) / (a1 a2),   a_j = 1 + 2^(-(x_j + b_j) log2 e).
 // The exponent is clamped at 28 (sigmoid < 4e-9 there), so a product of four a_j stays below
 // 2^116 and cannot overflow.  nb[j] = -b_j log2 e.
-template <int HI>
+// RELU: sum_j w_j * max(x_j + b_j, 0) (Eq. 3), nb[j] = b_j; no special-function work at all.
+template <int HI, bool RELU>
 __device__ __forceinline__ float gated_head_sum(const uint32_t* x, const float* w, const float (&nb)[HI]) {
+    if constexpr (RELU) {
+        float acc = 0.f;
+#pragma unroll
+        for (int j = 0; j < HI; ++j) acc = fmaf(w[j], fmaxf(__uint_as_float(x[j]) + nb[j], 0.f), acc);
+        return acc;
+    }
     float a[HI];
 #pragma unroll
     for (int j = 0; j < HI; ++j)
@@ -165,7 +172,7 @@ __device__ __forceinline__ uint64_t make_kmajor_desc(uint32_t smem_addr) {
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kNCols >> 3) << 17) |
                             ((uint32_t)(kTileKeys >> 4) << 24);
 
-template <int DI, int HI>
+template <int DI, int HI, bool RELU>
 __global__ void __launch_bounds__(kThreads, 1)
 gsa_indexer_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
                       const TcArgs a) {
@@ -283,7 +290,7 @@ gsa_indexer_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         constexpr int QPC = 32 / HI;                        // queries per 32-column chunk
         float bias[HI];
 #pragma unroll
-        for (int j = 0; j < HI; ++j) bias[j] = s_b[j] * -1.4426950408889634f;
+        for (int j = 0; j < HI; ++j) bias[j] = RELU ? s_b[j] : s_b[j] * -1.4426950408889634f;
         for (int i = 0; i < ntiles; ++i) {
             const int buf = i & 1;
             if (!mbar_wait(bar_tfull(buf), (i >> 1) & 1, s_abort)) {
@@ -312,7 +319,7 @@ gsa_indexer_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
 #pragma unroll
                         for (int j = 0; j < HI; ++j) wv[j] = s_w[qi * HI + j];
                     }
-                    const float acc = gated_head_sum<HI>(&r[qq * HI], wv, bias);
+                    const float acc = gated_head_sum<HI, RELU>(&r[qq * HI], wv, bias);
                     if (qi < nq && s <= off + t0 + qi) out_col[(int64_t)qi * a.row_stride] = acc;
                 }
             };
@@ -369,7 +376,7 @@ bool make_rows_tmap(CUtensorMap* tm, const void* base, uint64_t rows, int DI, ui
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int DI, int HI>
+template <int DI, int HI, bool RELU>
 cudaError_t launch_t(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* qI, const __nv_bfloat16* kI,
                      const float* w, const float* bI, float* scores, int64_t row_stride, int32_t* dev_status,
                      cudaStream_t st) {
@@ -396,7 +403,7 @@ cudaError_t launch_t(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* qI
     // one CTA per SM: the kernel allocates all 512 TMEM columns, so a second resident CTA would
     // only sit in tcgen05.alloc until the first one leaves
     constexpr int kSmem = P::ALLOC > 120 * 1024 ? P::ALLOC : 120 * 1024;
-    auto kern = gsa_indexer_tc_kernel<DI, HI>;
+    auto kern = gsa_indexer_tc_kernel<DI, HI, RELU>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
     kern<<<grid, kThreads, kSmem, st>>>(tm_k, tm_q, a);
@@ -418,7 +425,9 @@ cudaError_t launch_indexer_tc(const gsa_params_t& p, RowRange rr, const __nv_bfl
                               int64_t row_stride, int32_t* dev_status, cudaStream_t st) {
     if (rr.rows() <= 0) return cudaSuccess;
 #define GSA_TC_CASE(DI_, HI_) \
-    if (p.dI == DI_ && p.HI == HI_) return launch_t<DI_, HI_>(p, rr, qI, kI, w, bI, scores, row_stride, dev_status, st)
+    if (p.dI == DI_ && p.HI == HI_) \
+        return p.act == 1 ? launch_t<DI_, HI_, true>(p, rr, qI, kI, w, bI, scores, row_stride, dev_status, st) \
+                          : launch_t<DI_, HI_, false>(p, rr, qI, kI, w, bI, scores, row_stride, dev_status, st)
     GSA_TC_CASE(64, 8); GSA_TC_CASE(64, 4); GSA_TC_CASE(64, 2); GSA_TC_CASE(64, 1);
     GSA_TC_CASE(32, 8); GSA_TC_CASE(32, 4); GSA_TC_CASE(32, 2); GSA_TC_CASE(32, 1);
 #undef GSA_TC_CASE

@@ -33,7 +33,7 @@ def row_stride(cfg: GsaConfig) -> int:
     return (cfg.Lk + 31) // 32 * 32
 
 
-def run_scores(cfg, d, q_begin=0, q_end=0, bI=None, poison=True):
+def run_scores(cfg, d, q_begin=0, q_end=0, bI=None, poison=True, **over):
     """gsa_indexer_scores for rows [q_begin, q_end) of every batch element -> [B, R, stride] fp32 (NaN-poisoned)."""
     qe = q_end or cfg.Lq
     R = qe - q_begin
@@ -41,7 +41,7 @@ def run_scores(cfg, d, q_begin=0, q_end=0, bI=None, poison=True):
     sc = torch.full((cfg.B, R, st), float("nan"), device="cuda", dtype=torch.float32) if poison else \
         torch.empty((cfg.B, R, st), device="cuda", dtype=torch.float32)
     ws = torch.zeros(1024, dtype=torch.uint8, device="cuda")
-    p = gsa.make_params(cfg, q_begin=q_begin, q_end=qe)
+    p = gsa.make_params(cfg, q_begin=q_begin, q_end=qe, **over)
     gsa.gsa_indexer_scores(p, d["qI"], d["kI"], d["w"], bI, sc, st, ws)
     assert gsa.gsa_device_status(ws) == 0
     return sc

@@ -33,8 +33,8 @@ def test_exports_match_header(lib):
 
 
 def test_params_struct_layout_matches_header():
-    # 12 int32, 2 float, 2 int32, no padding
-    assert ctypes.sizeof(binding.gsa_params_t) == 16 * 4
+    # 12 int32, 2 float, 3 int32, no padding
+    assert ctypes.sizeof(binding.gsa_params_t) == 17 * 4
 
 
 def test_workspace_bytes_and_argument_errors(lib):

@@ -116,6 +116,42 @@ def test_indexer_few_rows_streams_keys(base, Lq, HI):
             assert np.isnan(sc[b, t, cfg.Lk - cfg.Lq + t + 1:cfg.Lk]).all()
 
 
+@pytest.mark.parametrize("path", [0, 1])
+def test_relu_indexer_scores(tiny, path):
+    """act = 1: the ReLU indexer of Eq. 3 (no special-function work; scores are >= 0 and unbounded)."""
+    cfg, x, d = tiny
+    bI = torch.tensor([0.25, -0.5, 0.0, 1.0], dtype=torch.float32)
+    gsa.gsa_debug_set_indexer_path(path)
+    try:
+        sc = U.run_scores(cfg, d, bI=bI.cuda(), act=1)[0].cpu().numpy()
+    finally:
+        gsa.gsa_debug_set_indexer_path(0)
+    rows = np.arange(cfg.Lq)
+    want = oracle.scores(U.oracle_params(cfg, act=1), x["qI"], x["kI"], x["w"], bI, rows)
+    for t in rows:
+        g, w = sc[t, :t + 1].astype(np.float64), want[t, :t + 1]
+        assert (g >= 0).all()
+        # relative 1e-3 as for the sigmoid scores, plus an absolute floor because ReLU scores reach 0
+        assert (np.abs(g - w) <= U.SCORE_REL_TOL * np.abs(w) + 1e-6).all()
+    # few query rows: the key-streaming kernel
+    cfg2 = CONFIGS["l8k"].with_(name="relu_rows", B=2, Lq=2, Lk=1500, seed=16)
+    x2 = make_inputs(cfg2)
+    sc2 = U.run_scores(cfg2, U.to_dev(x2), act=1).cpu().numpy()
+    for b in range(cfg2.B):
+        want2 = oracle.scores(U.oracle_params(cfg2, act=1), x2["qI"], x2["kI"], x2["w"], None, np.arange(2), np.full(2, b))
+        for t in range(2):
+            n = cfg2.Lk - cfg2.Lq + t + 1
+            assert (np.abs(sc2[b, t, :n] - want2[t, :n]) <= U.SCORE_REL_TOL * np.abs(want2[t, :n]) + 1e-6).all()
+
+
+def test_forward_relu_indexer_fixed_budget(l8k):
+    """The 'sparse only' indexer setting of the paper's comparison (ReLU scores, fixed k) through the whole path."""
+    cfg, x, d = l8k
+    rows = sample_rows(cfg, 16).numpy()
+    mism, kt = _forward_and_compare(cfg, x, d, rows, act=1, k_mode=2)
+    assert (kt[0].cpu().numpy() == np.minimum(cfg.k_base, np.arange(cfg.Lq) + 1)).all()
+
+
 # ------------------------------------------------------------------------------------------ stage 2
 def _select_and_compare(cfg, sc_dev, rows=None, k_mode=0, **over):
     """sc_dev: [B, Lq, stride] fp32 on the GPU; compares every (or the listed) row of batch 0."""
