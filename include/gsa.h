@@ -177,6 +177,8 @@ int gsa_forward(const gsa_params_t *p, const void *Q, const void *K, const void 
  * gsa_forward on HOST buffers (pinned memory recommended): copies the nine inputs to a
  * caller-provided device arena, runs gsa_forward there, copies `out` (and kt_out if
  * not NULL) back and waits for `stream`.  All tensor pointers are host pointers.
+ * The large tensors (Q, K, V, gate logits) are copied on a second stream that exists for the
+ * duration of the call, under the indexer and the selection, which need only qI, kI and w.
  * `arena` is device memory of at least gsa_forward_host_arena_bytes(p, slab_rows).
  */
 int gsa_forward_host_arena_bytes(const gsa_params_t *p, int32_t slab_rows, size_t *bytes);

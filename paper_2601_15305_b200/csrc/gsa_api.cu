@@ -212,10 +212,14 @@ int gsa_sparse_gated_attn_fwd(const gsa_params_t* p, const void* Q, const void* 
                                       g2use, idx, kt, il, (bf16*)out, scratch, st));
 }
 
-int gsa_forward(const gsa_params_t* p, const void* Q, const void* K, const void* V, const void* qI,
-                const void* kI, const float* w, const float* bI, const void* g1_logits,
-                const void* g2_logits, void* out, int32_t* idx_out, int32_t* kt_out, float* var_out,
-                int32_t slab_rows, void* ws, size_t ws_bytes, void* stream) {
+// The whole path.  `kv_ready` (may be NULL) is an event the stream waits for before anything reads
+// Q, K, V or the gate logits: the indexer and the selection need only qI, kI and w, so a caller that is
+// still copying the large tensors can let those copies run under the first two stages.
+static int forward_impl(const gsa_params_t* p, const void* Q, const void* K, const void* V, const void* qI,
+                        const void* kI, const float* w, const float* bI, const void* g1_logits,
+                        const void* g2_logits, void* out, int32_t* idx_out, int32_t* kt_out, float* var_out,
+                        int32_t slab_rows, void* ws, size_t ws_bytes, void* stream, cudaEvent_t kv_ready,
+                        AttnProgress* progress) {
     int rc = check_params(p);
     if (rc) return rc;
     if (!Q || !K || !V || !qI || !kI || !w || !g1_logits || !out || slab_rows < 0) return GSA_ERR_INVALID_ARG;
@@ -234,17 +238,6 @@ int gsa_forward(const gsa_params_t* p, const void* Q, const void* K, const void*
     const IdxLayout il{0, 0, p->Lq};
 
     if (g_prof_ev[0]) cudaEventRecord(g_prof_ev[0], st);
-    // Eq. 9: value gate (independent of the indexer)
-    const bf16* Vuse = (const bf16*)V;
-    const bf16* g2use = (const bf16*)g2_logits;
-    if (g2_logits && wp.prepass) {
-        bf16* Vg = (bf16*)(wsb + wp.vg_off);
-        e = launch_value_gate((const bf16*)V, (const bf16*)g2_logits, Vg,
-                              (int64_t)p->B * p->Lk * p->n_kv * p->d_h, st);
-        if (e != cudaSuccess) return cuda_rc(e);
-        Vuse = Vg;
-        g2use = nullptr;
-    }
 
     // Eq. 7, 8, 4 slab by slab: score rows live only inside the workspace
     if (wp.slab_rows >= p->Lq) {
@@ -267,13 +260,33 @@ int gsa_forward(const gsa_params_t* p, const void* Q, const void* K, const void*
             }
     }
 
-    // Eq. 11, 12, 10 over all rows
     if (g_prof_ev[1]) cudaEventRecord(g_prof_ev[1], st);
+    if (kv_ready && (e = cudaStreamWaitEvent(st, kv_ready, 0)) != cudaSuccess) return cuda_rc(e);
+    // Eq. 9: value gate (touches only V, so its place in the order is free; the pipeline of Sec. 3.2 lists it first)
+    const bf16* Vuse = (const bf16*)V;
+    const bf16* g2use = (const bf16*)g2_logits;
+    if (g2_logits && wp.prepass) {
+        bf16* Vg = (bf16*)(wsb + wp.vg_off);
+        e = launch_value_gate((const bf16*)V, (const bf16*)g2_logits, Vg,
+                              (int64_t)p->B * p->Lk * p->n_kv * p->d_h, st);
+        if (e != cudaSuccess) return cuda_rc(e);
+        Vuse = Vg;
+        g2use = nullptr;
+    }
+    // Eq. 11, 12, 10 over all rows
     RowRange all{0, p->B, 0, p->Lq};
     e = launch_sparse_attn(*p, all, (const bf16*)Q, (const bf16*)K, Vuse, (const bf16*)g1_logits, g2use, idx,
-                           kt, il, (bf16*)out, wsb + wp.attn_off, st);
+                           kt, il, (bf16*)out, wsb + wp.attn_off, st, progress);
     if (g_prof_ev[2]) cudaEventRecord(g_prof_ev[2], st);
     return cuda_rc(e);
+}
+
+int gsa_forward(const gsa_params_t* p, const void* Q, const void* K, const void* V, const void* qI,
+                const void* kI, const float* w, const float* bI, const void* g1_logits,
+                const void* g2_logits, void* out, int32_t* idx_out, int32_t* kt_out, float* var_out,
+                int32_t slab_rows, void* ws, size_t ws_bytes, void* stream) {
+    return forward_impl(p, Q, K, V, qI, kI, w, bI, g1_logits, g2_logits, out, idx_out, kt_out, var_out, slab_rows,
+                        ws, ws_bytes, stream, nullptr, nullptr);
 }
 
 int gsa_forward_host_arena_bytes(const gsa_params_t* p, int32_t slab_rows, size_t* bytes) {
@@ -313,20 +326,72 @@ int gsa_forward_host(const gsa_params_t* p, const void* Q, const void* K, const 
     char *dQ = take(q), *dG1 = take(q), *dOut = take(q), *dK = take(kv), *dV = take(kv), *dG2 = take(kv);
     char *dqI = take(qi), *dkI = take(ki), *dw = take(wb), *dbI = take(256), *dkt = take(ktb);
     char* dws = a + off;
+    // The small indexer inputs go first on the caller's stream; the large tensors follow on a second
+    // stream and are awaited only before the value gate / attention, so they copy under the indexer and
+    // the selection.  (The stream and the two events live for this call only.)
     cudaError_t e;
-#define GSA_H2D(dst, src, n) if ((e = cudaMemcpyAsync(dst, src, n, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_rc(e)
-    GSA_H2D(dQ, Q, q); GSA_H2D(dK, K, kv); GSA_H2D(dV, V, kv); GSA_H2D(dqI, qI, qi); GSA_H2D(dkI, kI, ki);
-    GSA_H2D(dw, w, wb); GSA_H2D(dG1, g1_logits, q);
-    if (g2_logits) GSA_H2D(dG2, g2_logits, kv);
-    if (bI) GSA_H2D(dbI, bI, (size_t)p->HI * 4);
+    cudaStream_t cs = nullptr;
+    cudaEvent_t ev_go = nullptr, ev_kv = nullptr;
+    if ((e = cudaStreamCreateWithFlags(&cs, cudaStreamNonBlocking)) != cudaSuccess) return cuda_rc(e);
+    auto cleanup = [&]() {
+        if (ev_go) cudaEventDestroy(ev_go);
+        if (ev_kv) cudaEventDestroy(ev_kv);
+        if (cs) { cudaStreamSynchronize(cs); cudaStreamDestroy(cs); }
+    };
+#define GSA_TRY(call) if ((e = (call)) != cudaSuccess) { cleanup(); return cuda_rc(e); }
+    GSA_TRY(cudaEventCreateWithFlags(&ev_go, cudaEventDisableTiming));
+    GSA_TRY(cudaEventCreateWithFlags(&ev_kv, cudaEventDisableTiming));
+    GSA_TRY(cudaEventRecord(ev_go, st));                   // earlier work on `st` may still use the arena
+    GSA_TRY(cudaStreamWaitEvent(cs, ev_go, 0));
+#define GSA_H2D(dst, src, n, s_) GSA_TRY(cudaMemcpyAsync(dst, src, n, cudaMemcpyHostToDevice, s_))
+    GSA_H2D(dqI, qI, qi, st); GSA_H2D(dkI, kI, ki, st); GSA_H2D(dw, w, wb, st);
+    if (bI) GSA_H2D(dbI, bI, (size_t)p->HI * 4, st);
+    GSA_H2D(dV, V, kv, cs);
+    if (g2_logits) GSA_H2D(dG2, g2_logits, kv, cs);
+    GSA_H2D(dK, K, kv, cs); GSA_H2D(dQ, Q, q, cs); GSA_H2D(dG1, g1_logits, q, cs);
 #undef GSA_H2D
-    rc = gsa_forward(p, dQ, dK, dV, dqI, dkI, (const float*)dw, bI ? (const float*)dbI : nullptr, dG1,
-                     g2_logits ? dG2 : nullptr, dOut, nullptr, (int32_t*)dkt, nullptr, slab_rows, dws,
-                     arena_bytes - off, st);
-    if (rc) return rc;
-    if ((e = cudaMemcpyAsync(out, dOut, q, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_rc(e);
-    if (kt_out && (e = cudaMemcpyAsync(kt_out, dkt, ktb, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_rc(e);
-    if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_rc(e);
+    GSA_TRY(cudaEventRecord(ev_kv, cs));
+    // output rows become final key range by key range; each block goes back to the host on the copy
+    // stream while the later ranges are still being computed
+    constexpr int kMaxBlocks = 64;
+    cudaEvent_t ev_rows[kMaxBlocks] = {};
+    AttnProgress prog;
+    prog.events = ev_rows; prog.cap = kMaxBlocks; prog.n = 0;
+    for (int i = 0; i < kMaxBlocks; ++i) {
+        if ((e = cudaEventCreateWithFlags(&ev_rows[i], cudaEventDisableTiming)) != cudaSuccess) break;
+    }
+    auto cleanup_rows = [&]() { for (int i = 0; i < kMaxBlocks; ++i) if (ev_rows[i]) cudaEventDestroy(ev_rows[i]); };
+    if (e != cudaSuccess) { cleanup_rows(); cleanup(); return cuda_rc(e); }
+    rc = forward_impl(p, dQ, dK, dV, dqI, dkI, (const float*)dw, bI ? (const float*)dbI : nullptr, dG1,
+                      g2_logits ? dG2 : nullptr, dOut, nullptr, (int32_t*)dkt, nullptr, slab_rows, dws,
+                      arena_bytes - off, st, ev_kv, &prog);
+    if (rc) { cleanup_rows(); cleanup(); return rc; }
+    const size_t row_bytes = (size_t)p->n_h * p->d_h * 2;
+    int covered_to = 0;
+    for (int i = 0; i < prog.n && e == cudaSuccess; ++i) {
+        e = cudaStreamWaitEvent(cs, ev_rows[i], 0);
+        for (int b = 0; b < p->B && e == cudaSuccess; ++b) {
+            const size_t o = ((size_t)b * p->Lq + prog.t_lo[i]) * row_bytes;
+            e = cudaMemcpyAsync((char*)out + o, dOut + o, (size_t)(prog.t_hi[i] - prog.t_lo[i]) * row_bytes,
+                                cudaMemcpyDeviceToHost, cs);
+        }
+        covered_to = prog.t_hi[i];
+    }
+    if (e == cudaSuccess && covered_to < p->Lq) {
+        // (more row blocks than events: the rest goes after the last kernel)
+        for (int b = 0; b < p->B && e == cudaSuccess; ++b) {
+            const size_t o = ((size_t)b * p->Lq + covered_to) * row_bytes;
+            e = cudaMemcpyAsync((char*)out + o, dOut + o, (size_t)(p->Lq - covered_to) * row_bytes,
+                                cudaMemcpyDeviceToHost, st);
+        }
+    }
+    if (e == cudaSuccess && kt_out) e = cudaMemcpyAsync(kt_out, dkt, ktb, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(cs);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    cleanup_rows();
+    if (e != cudaSuccess) { cleanup(); return cuda_rc(e); }
+#undef GSA_TRY
+    cleanup();
     int32_t dev = 0;
     return gsa_device_status(dws, stream, &dev);
 }

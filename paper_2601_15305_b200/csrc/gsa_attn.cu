@@ -516,7 +516,7 @@ AttnPlan plan_attn(const gsa_params_t& p) {
 
 template <int DH, int G, bool FUSE_G2>
 cudaError_t launch_attn_t(AttnArgs a, const gsa_params_t& p, const AttnPlan& pl, const __nv_bfloat16* g1,
-                          __nv_bfloat16* out, int32_t* cuts, cudaStream_t st) {
+                          __nv_bfloat16* out, int32_t* cuts, cudaStream_t st, AttnProgress* prog) {
     constexpr int VSTAGES = FUSE_G2 ? 1 : 2;
     constexpr int kWarpsPerCta = FUSE_G2 ? kWarpsFused : kWarpsPrefill;
     constexpr size_t smem = (size_t)kWarpsPerCta * VSTAGES * kTileKeys * (DH * 2 + 16);
@@ -543,6 +543,24 @@ cudaError_t launch_attn_t(AttnArgs a, const gsa_params_t& p, const AttnPlan& pl,
     a.n_cuts = pl.n_ranges;
     a.mode = pl.mode;
     a.max_parts = pl.slots;
+    const int fin_threads = a.n_kv * DH < 1024 ? a.n_kv * DH : 1024;
+    // normalise + G1 + bf16 for rows t_lo <= t < t_hi of every batch element, then tell the caller
+    auto finalize = [&](int t_lo, int t_hi) -> cudaError_t {
+        if (t_hi <= t_lo) return cudaSuccess;
+        RowRange fr = rr_all;
+        fr.q_begin = t_lo; fr.R = t_hi - t_lo;
+        gsa_attn_finalize_kernel<DH, G><<<(unsigned)((fr.rows() + kFinRows - 1) / kFinRows), fin_threads, 0, st>>>(
+            a.state, a.kt, g1, out, fr, a.il, a.idx_rows, p.Lq, p.n_h, p.n_kv, p.k_max, pl.mode, pl.slots);
+        ++g_launches;
+        cudaError_t fe = cudaGetLastError();
+        if (fe == cudaSuccess && prog && prog->n < prog->cap && prog->n < 64) {
+            fe = cudaEventRecord(prog->events[prog->n], st);
+            prog->t_lo[prog->n] = t_lo; prog->t_hi[prog->n] = t_hi;
+            ++prog->n;
+        }
+        return fe;
+    };
+    int finalized_to = rr_all.q_begin;                      // rows below this are final
     for (int rg = 0; rg < pl.n_ranges; ++rg) {
         AttnArgs ar = a;
         ar.range = rg;
@@ -558,22 +576,25 @@ cudaError_t launch_attn_t(AttnArgs a, const gsa_params_t& p, const AttnPlan& pl,
         kern<<<ctas, kWarpsPerCta * 32, smem, st>>>(ar);
         ++g_launches;
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        if (pl.mode == 0 && rg + 1 < pl.n_ranges) {
+            // rows whose last visible key lies in this range are complete
+            const int64_t t_done = (int64_t)(rg + 1) * g_range_keys - off;
+            const int t_hi = (int)(t_done < finalized_to ? finalized_to : (t_done > q_end ? q_end : t_done));
+            if ((e = finalize(finalized_to, t_hi)) != cudaSuccess) return e;
+            finalized_to = t_hi;
+        }
     }
-    const int fin_threads = a.n_kv * DH < 1024 ? a.n_kv * DH : 1024;
-    gsa_attn_finalize_kernel<DH, G><<<(unsigned)((rr_all.rows() + kFinRows - 1) / kFinRows), fin_threads, 0, st>>>(
-        a.state, a.kt, g1, out, rr_all, a.il, a.idx_rows, p.Lq, p.n_h, p.n_kv, p.k_max, pl.mode, pl.slots);
-    ++g_launches;
-    return cudaGetLastError();
+    return finalize(finalized_to, q_end);
 }
 
 template <int DH, bool FUSE_G2>
 cudaError_t launch_attn_g(const AttnArgs& a, const gsa_params_t& p, const AttnPlan& pl, const __nv_bfloat16* g1,
-                          __nv_bfloat16* out, int32_t* cuts, int G, cudaStream_t st) {
+                          __nv_bfloat16* out, int32_t* cuts, int G, cudaStream_t st, AttnProgress* prog) {
     switch (G) {
-        case 1: return launch_attn_t<DH, 1, FUSE_G2>(a, p, pl, g1, out, cuts, st);
-        case 2: return launch_attn_t<DH, 2, FUSE_G2>(a, p, pl, g1, out, cuts, st);
-        case 4: return launch_attn_t<DH, 4, FUSE_G2>(a, p, pl, g1, out, cuts, st);
-        case 8: return launch_attn_t<DH, 8, FUSE_G2>(a, p, pl, g1, out, cuts, st);
+        case 1: return launch_attn_t<DH, 1, FUSE_G2>(a, p, pl, g1, out, cuts, st, prog);
+        case 2: return launch_attn_t<DH, 2, FUSE_G2>(a, p, pl, g1, out, cuts, st, prog);
+        case 4: return launch_attn_t<DH, 4, FUSE_G2>(a, p, pl, g1, out, cuts, st, prog);
+        case 8: return launch_attn_t<DH, 8, FUSE_G2>(a, p, pl, g1, out, cuts, st, prog);
     }
     return cudaErrorInvalidValue;
 }
@@ -603,7 +624,7 @@ cudaError_t launch_sparse_attn(const gsa_params_t& p, RowRange rr, const __nv_bf
                                const __nv_bfloat16* K, const __nv_bfloat16* V,
                                const __nv_bfloat16* g1, const __nv_bfloat16* g2, const int32_t* idx,
                                const int32_t* kt, IdxLayout il, __nv_bfloat16* out, void* scratch,
-                               cudaStream_t st) {
+                               cudaStream_t st, AttnProgress* progress) {
     if (rr.rows() <= 0) return cudaSuccess;
     const AttnPlan pl = plan_attn(p);
     AttnArgs a;
@@ -618,9 +639,11 @@ cudaError_t launch_sparse_attn(const gsa_params_t& p, RowRange rr, const __nv_bf
     a.scale_log2 = sc * 1.4426950408889634f;
     const int G = p.n_h / p.n_kv;
     if (p.d_h == 128)
-        return g2 ? launch_attn_g<128, true>(a, p, pl, g1, out, cuts, G, st) : launch_attn_g<128, false>(a, p, pl, g1, out, cuts, G, st);
+        return g2 ? launch_attn_g<128, true>(a, p, pl, g1, out, cuts, G, st, progress)
+                  : launch_attn_g<128, false>(a, p, pl, g1, out, cuts, G, st, progress);
     if (p.d_h == 64)
-        return g2 ? launch_attn_g<64, true>(a, p, pl, g1, out, cuts, G, st) : launch_attn_g<64, false>(a, p, pl, g1, out, cuts, G, st);
+        return g2 ? launch_attn_g<64, true>(a, p, pl, g1, out, cuts, G, st, progress)
+                  : launch_attn_g<64, false>(a, p, pl, g1, out, cuts, G, st, progress);
     return cudaErrorInvalidValue;
 }
 

@@ -46,11 +46,22 @@ cudaError_t launch_select(const gsa_params_t& p, RowRange rr, const float* score
 cudaError_t launch_value_gate(const __nv_bfloat16* V, const __nv_bfloat16* g2, __nv_bfloat16* Vg,
                               int64_t n_elems, cudaStream_t st);
 
+// Optional progress report of launch_sparse_attn: output rows become final range by range (a query
+// row is final once the key range holding its last visible key has been processed).  events[i], which
+// the caller created, is recorded when rows t_lo[i] <= t < t_hi[i] of every batch element are final.
+struct AttnProgress {
+    cudaEvent_t* events;
+    int cap;
+    int n;
+    int32_t t_lo[64], t_hi[64];
+};
+
 cudaError_t launch_sparse_attn(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* Q,
                                const __nv_bfloat16* K, const __nv_bfloat16* V,
                                const __nv_bfloat16* g1, const __nv_bfloat16* g2 /*nullable*/,
                                const int32_t* idx, const int32_t* kt, IdxLayout il,
-                               __nv_bfloat16* out, void* scratch, cudaStream_t st);
+                               __nv_bfloat16* out, void* scratch, cudaStream_t st,
+                               AttnProgress* progress = nullptr);
 
 // bytes of device scratch launch_sparse_attn needs for `p` (softmax state slots, range cuts)
 size_t attn_scratch_bytes(const gsa_params_t& p);

@@ -399,6 +399,35 @@ def test_forward_host_buffers_match_device_call(tiny):
     assert torch.equal(kt_h, kt_dev.cpu())
 
 
+def test_forward_many_key_ranges_device_and_host_paths():
+    """Key ranges of 1024 keys on a 3000-token sequence: three attention launches with carried softmax
+    state, rows finalised range by range; the host-buffer call streams finished rows back early."""
+    cfg = CONFIGS["tiny"].with_(name="ranges", B=2, Lq=3000, Lk=3000, k_base=300, k_min=64, k_max=600, seed=17,
+                               v_bar=2.0e-3)
+    x = make_inputs(cfg)
+    d = U.to_dev(x)
+    gsa.gsa_debug_set_attn_range_keys(1024)
+    try:
+        out, idx, kt, var = U.run_forward(cfg, d)
+        p = gsa.make_params(cfg)
+        pin = {k: v.pin_memory() for k, v in x.items()}
+        out_h = torch.empty_like(x["Q"]).pin_memory()
+        kt_h = torch.empty((cfg.B, cfg.Lq), dtype=torch.int32).pin_memory()
+        arena = torch.empty(gsa.gsa_forward_host_arena_bytes(p, 0), dtype=torch.uint8, device="cuda")
+        gsa.gsa_forward_host(p, pin["Q"], pin["K"], pin["V"], pin["qI"], pin["kI"], pin["w"], None, pin["g1"],
+                             pin["g2"], out_h, kt_h, 0, arena)
+    finally:
+        gsa.gsa_debug_set_attn_range_keys(0)
+    assert torch.equal(out_h.view(torch.int16), out.cpu().view(torch.int16))
+    assert torch.equal(kt_h, kt.cpu())
+    po = U.oracle_params(cfg)
+    for b in range(cfg.B):
+        rows = np.array([0, 5, 1023, 1024, 1500, 2047, 2048, 2999])
+        o = oracle.forward(po, **x, rows_t=rows, rows_b=np.full_like(rows, b), want_scores=True)
+        U.check_e2e_indices(o, idx[b][rows].cpu().numpy(), kt[b][rows].cpu().numpy(), o["scores"], _vis(cfg, rows))
+        U.check_out(out[b][rows].float().cpu().numpy(), o["out"])
+
+
 def test_argument_errors_do_not_launch(tiny):
     cfg, x, d = tiny
     p = gsa.make_params(cfg)
