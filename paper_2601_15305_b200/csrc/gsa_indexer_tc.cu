@@ -11,9 +11,10 @@
 // A CTA works on one query group and a run of key tiles at or below the diagonal (tiles above
 // it are never touched).  Warp roles: warp 0 feeds shared memory by TMA (k^I tiles through a
 // ring of stages, the q^I tile once), warp 1 issues the MMAs and owns the TMEM allocation,
-// warps 2..9 are the epilogue.  Two 256-column accumulators alternate, so the MMAs of tile i+1
+// warps 2..17 are the epilogue.  Two 256-column accumulators alternate, so the MMAs of tile i+1
 // overlap the epilogue of tile i; the epilogue (exp2 + reciprocal per sigmoid on the
-// special-function unit) is the longer of the two.
+// special-function unit) is the longer of the two, which is why it gets sixteen warps (four per
+// scheduler), each reading its 64 columns 16 at a time.
 //
 // Every mbarrier wait is bounded: when a wait runs out the CTA records it in the status word,
 // stops issuing work, drains what it has in flight and exits with its TMEM released.
@@ -29,8 +30,10 @@ namespace {
 constexpr int kTileKeys = 128;
 constexpr int kNCols = 256;            // N of one MMA = (queries x heads) of a group
 constexpr int kStages = 6;
-constexpr int kThreads = 320;          // 10 warps
-constexpr int kEpiWarps = 8;
+constexpr int kEpiWarps = 16;          // 4 per scheduler: keeps the special-function unit fed
+constexpr int kThreads = 64 + kEpiWarps * 32;
+constexpr int kColsPerWarp = kNCols / (kEpiWarps / 4);   // accumulator columns one epilogue warp handles
+constexpr int kChunkCols = 16;         // columns per tcgen05.ld
 
 struct TcArgs {
     const float* w;
@@ -104,6 +107,24 @@ __device__ __forceinline__ void tc_wait_ld(uint32_t (&r)[32]) {
           "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
           "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
           "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+        :
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld16(uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.wait::ld.sync.aligned;"
+        : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+          "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
         :
         : "memory");
 }
@@ -230,9 +251,11 @@ gsa_indexer_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
     }
     if (warp >= 2) {
         const int e = threadIdx.x - 64;                               // 0..255 = (query, head) column
-        const int qi = e / HI, j = e % HI;
-        s_w[e] = qi < nq ? a.w[((size_t)b * a.Lq + t0 + qi) * HI + j] : 0.f;
-        if (e < 8) s_b[e] = (a.bI && e < HI) ? a.bI[e] : 0.f;
+        if (e < kNCols) {
+            const int qi = e / HI, j = e % HI;
+            s_w[e] = qi < nq ? a.w[((size_t)b * a.Lq + t0 + qi) * HI + j] : 0.f;
+            if (e < 8) s_b[e] = (a.bI && e < HI) ? a.bI[e] : 0.f;
+        }
     }
     tc_fence_before();
     __syncthreads();
@@ -286,8 +309,9 @@ gsa_indexer_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         // ================= epilogue: sigmoid, head weights, head sum, store ===================
         const int ew = warp - 2;
         const int quad = warp & 3;                          // TMEM lanes this warp may touch: 32*quad ..
-        const int half = ew >> 2;                           // which 128 of the 256 columns
-        constexpr int QPC = 32 / HI;                        // queries per 32-column chunk
+        const int part = ew >> 2;                           // which kColsPerWarp of the 256 columns
+        constexpr int QPC = kChunkCols / HI;                // queries per 16-column chunk
+        constexpr int NCHUNK = kColsPerWarp / kChunkCols;
         float bias[HI];
 #pragma unroll
         for (int j = 0; j < HI; ++j) bias[j] = RELU ? s_b[j] : s_b[j] * -1.4426950408889634f;
@@ -299,12 +323,12 @@ gsa_indexer_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
             }
             tc_fence_after();
             const int s = (tile0 + i) * kTileKeys + quad * 32 + lane;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * kNCols + half * 128;
-            // columns are read 32 at a time, the next chunk's load in flight behind the current
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * kNCols + part * kColsPerWarp;
+            // columns are read 16 at a time, the next chunk's load in flight behind the current
             // chunk's arithmetic
             float* const out_col = a.scores + ((int64_t)bl * a.rr.R + tr0) * a.row_stride + s;
-            auto do_chunk = [&](const uint32_t (&r)[32], int c) {
-                const int q_first = (half * 128 + c * 32) / HI;
+            auto do_chunk = [&](const uint32_t (&r)[kChunkCols], int c) {
+                const int q_first = (part * kColsPerWarp + c * kChunkCols) / HI;
 #pragma unroll
                 for (int qq = 0; qq < QPC; ++qq) {
                     const int qi = q_first + qq;
@@ -323,19 +347,17 @@ gsa_indexer_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
                     if (qi < nq && s <= off + t0 + qi) out_col[(int64_t)qi * a.row_stride] = acc;
                 }
             };
-            uint32_t ra[32], rb[32];
-            tc_ld32(taddr, ra);
-            tc_wait_ld(ra);
-            tc_ld32(taddr + 32, rb);
-            do_chunk(ra, 0);
-            tc_wait_ld(rb);
-            tc_ld32(taddr + 64, ra);
-            do_chunk(rb, 1);
-            tc_wait_ld(ra);
-            tc_ld32(taddr + 96, rb);
-            do_chunk(ra, 2);
-            tc_wait_ld(rb);
-            do_chunk(rb, 3);
+            uint32_t ra[kChunkCols], rb[kChunkCols];
+            tc_ld16(taddr, ra);
+#pragma unroll
+            for (int c = 0; c < NCHUNK; c += 2) {
+                tc_wait_ld16(ra);
+                tc_ld16(taddr + (c + 1) * kChunkCols, rb);
+                do_chunk(ra, c);
+                tc_wait_ld16(rb);
+                if (c + 2 < NCHUNK) tc_ld16(taddr + (c + 2) * kChunkCols, ra);
+                do_chunk(rb, c + 1);
+            }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_tempty(buf));
