@@ -182,3 +182,25 @@ def forward(p: OracleParams, Q, K, V, qI, kI, w, g1, g2, bI=None, rows_t: Sequen
     if want_scores:
         res["scores"] = sc
     return res
+
+
+def project_rows_total(p: OracleParams) -> int:
+    """Rows of the stacked, transposed weight matrix: q^I, k^I, 8 head-weight rows, g1, g2."""
+    return p.HI * p.dI + p.dI + 8 + p.n_h * p.d_h + p.n_kv * p.d_h
+
+
+def project(p: OracleParams, d_model: int, H, Wt, rows_m: Sequence[int]):
+    """Upstream projections (text below Eq. 7, Eq. 9, Eq. 10) of the listed token rows of H [M, d_model].
+    Returns dict(qI [n, HI*dI], kI [n, dI], w [n, HI] (after the sigmoid), g1 [n, n_h*d_h], g2 [n, n_kv*d_h]), fp64."""
+    H, Wt = _f32(H), _f32(Wt)
+    rows_m = _i32(rows_m).reshape(-1)
+    assert H.ndim == 2 and H.shape[1] == d_model and Wt.shape == (project_rows_total(p), d_model)
+    assert rows_m.min(initial=0) >= 0 and rows_m.max(initial=0) < H.shape[0]
+    n = len(rows_m)
+    out = dict(qI=np.empty((n, p.HI * p.dI)), kI=np.empty((n, p.dI)), w=np.empty((n, p.HI)),
+               g1=np.empty((n, p.n_h * p.d_h)), g2=np.empty((n, p.n_kv * p.d_h)))
+    c = p.c()
+    lib().gsa_oracle_project_rows(ctypes.byref(c), ctypes.c_int(d_model), _ptr(H), _ptr(Wt), _ptr(rows_m),
+                                  ctypes.c_int(n), _ptr(out["qI"]), _ptr(out["kI"]), _ptr(out["w"]),
+                                  _ptr(out["g1"]), _ptr(out["g2"]))
+    return out

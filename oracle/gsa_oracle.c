@@ -175,6 +175,34 @@ void gsa_oracle_attn_row(const gsa_oracle_params *p, const float *Q_t, const flo
     free(z);
 }
 
+/* ---- upstream projections (text below Eq. 7; Eq. 9; Eq. 10) ---------------- */
+/* One token's projections from its hidden state h [d_model]:
+ *   q^I_j = h W^Iq_j,  k^I = h W^Ik,  head weight sigmoid(h W^Iw_j),  g1 logits = h W^g_O,  g2 logits = h W^g_V.
+ * Wt holds the weight matrices transposed and stacked, one row of d_model per output column, in the
+ * order q^I (HI*dI rows), k^I (dI), head weights (8 rows, the first HI used), g1 (n_h*d_h), g2 (n_kv*d_h). */
+void gsa_oracle_project_rows(const gsa_oracle_params *p, int d_model, const float *H, const float *Wt,
+                             const int32_t *rows_m, int n_rows, double *qI, double *kI, double *w,
+                             double *g1, double *g2)
+{
+    const int nq = p->HI * p->dI, nk = p->dI, ng1 = p->n_h * p->d_h, ng2 = p->n_kv * p->d_h;
+    const int o_k = nq, o_w = nq + nk, o_g1 = o_w + 8, o_g2 = o_g1 + ng1;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int r = 0; r < n_rows; ++r) {
+        const float *h = H + (size_t)rows_m[r] * d_model;
+        for (int n = 0; n < o_g2 + ng2; ++n) {
+            if (n >= o_w + p->HI && n < o_g1) continue;              /* unused rows of the weight block */
+            const float *wt = Wt + (size_t)n * d_model;
+            double acc = 0.0;
+            for (int c = 0; c < d_model; ++c) acc += (double)h[c] * (double)wt[c];
+            if (n < o_k)        qI[(size_t)r * nq + n] = acc;
+            else if (n < o_w)   kI[(size_t)r * nk + (n - o_k)] = acc;
+            else if (n < o_g1)  w[(size_t)r * p->HI + (n - o_w)] = sigmoid_d(acc);
+            else if (n < o_g2)  g1[(size_t)r * ng1 + (n - o_g1)] = acc;
+            else                g2[(size_t)r * ng2 + (n - o_g2)] = acc;
+        }
+    }
+}
+
 /* ---- drivers over a list of (batch, query) rows -------------------------- */
 
 /* scores of the listed rows: out[r, 0..n_t) in a [n_rows, Lk] double array */

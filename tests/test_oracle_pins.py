@@ -378,6 +378,42 @@ def test_forward_is_composition_of_stages():
 
 
 # ----------------------------------------------------------------------------- printed numbers
+def test_projections_copy_columns_closed_form_sigmoid_and_library_matmul():
+    """Upstream projections.  One-hot weight rows copy a column of H into a known output slot (a wrong block
+    order or offset moves it); head-weight rows of zeros / ln3 give sigmoid 1/2 and 3/4; random weights equal
+    a library matmul per block."""
+    p = small_params(HI=3, dI=4, n_h=4, n_kv=2, d_h=8)
+    d_model = 16
+    n_tot = oracle.project_rows_total(p)
+    assert n_tot == 12 + 4 + 8 + 32 + 16
+    rng = np.random.default_rng(3)
+    H = rng.standard_normal((5, d_model)).astype(np.float32)
+    H[:, 7] = 1.0                                           # a constant column for the closed-form sigmoid
+    Wt = np.zeros((n_tot, d_model), np.float32)
+    Wt[5, 2] = 1.0        # q^I slot 5 (head 1, component 1) <- H[:, 2]
+    Wt[12 + 3, 9] = -2.0  # k^I component 3               <- -2 H[:, 9]
+    Wt[16 + 1, 7] = LN3   # head weight 1: sigmoid(ln 3) = 3/4
+    Wt[24 + 31, 0] = 1.0  # last g1 slot                   <- H[:, 0]
+    Wt[56 + 0, 15] = 0.5  # first g2 slot                  <- H[:, 15] / 2
+    o = oracle.project(p, d_model, H, Wt, [0, 4, 2])
+    Hs = H[[0, 4, 2]].astype(np.float64)
+    np.testing.assert_allclose(o["qI"][:, 5], Hs[:, 2], atol=1e-15)
+    assert np.count_nonzero(o["qI"]) == 3
+    np.testing.assert_allclose(o["kI"][:, 3], -2.0 * Hs[:, 9], atol=1e-15)
+    np.testing.assert_allclose(o["w"][:, 1], 0.75, atol=1e-7)
+    np.testing.assert_allclose(o["w"][:, [0, 2]], 0.5, atol=1e-15)
+    np.testing.assert_allclose(o["g1"][:, 31], Hs[:, 0], atol=1e-15)
+    np.testing.assert_allclose(o["g2"][:, 0], 0.5 * Hs[:, 15], atol=1e-15)
+    Wt = rng.standard_normal((n_tot, d_model)).astype(np.float32)
+    o = oracle.project(p, d_model, H, Wt, np.arange(5))
+    full = H.astype(np.float64) @ Wt.astype(np.float64).T
+    np.testing.assert_allclose(o["qI"], full[:, :12], rtol=1e-13, atol=1e-13)
+    np.testing.assert_allclose(o["kI"], full[:, 12:16], rtol=1e-13, atol=1e-13)
+    np.testing.assert_allclose(o["w"], 1.0 / (1.0 + np.exp(-full[:, 16:19])), rtol=1e-13)
+    np.testing.assert_allclose(o["g1"], full[:, 24:56], rtol=1e-13, atol=1e-13)
+    np.testing.assert_allclose(o["g2"], full[:, 56:72], rtol=1e-13, atol=1e-13)
+
+
 def test_paper_printed_cost_model():
     """Appendix A prints d^I H^I/(d n_h) ~ 0.002 and a 12.8x speed-up for its parameters."""
     vals = {}
