@@ -172,6 +172,7 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (smaller ncu captures)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-projection", action="store_true", help="skip timing the upstream projection GEMM")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "gsa_b200" else args.warmup
     cfg = CONFIGS[args.workload]
@@ -283,6 +284,34 @@ def main():
               "indexer_causal_tflop": 2.0 * cfg.HI * cfg.dI * causal_pairs / 1e12,
               "mean_k_t": kt_sum / float(cfg.B * cfg.Lq), "select_fallback_rows": fallback_rows}
 
+    # ---- the upstream projection GEMM (outside the timed step: its outputs are the step's inputs) ----
+    projection = None
+    if not args.no_projection and cfg.Lq == cfg.Lk:
+        d_model = 2048
+        n_cols = gsa.gsa_project_columns(p)
+        M = cfg.B * cfg.Lk
+        gen = torch.Generator(device="cuda").manual_seed(5)
+        Hs = torch.randn(M, d_model, generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        Wt = (torch.randn(n_cols, d_model, generator=gen, device="cuda", dtype=torch.float32) / d_model ** 0.5).to(torch.bfloat16)
+        po = {k: torch.empty_like(d[k]) for k in ("qI", "kI", "w", "g1", "g2")}
+        ws_p = torch.zeros(1024, dtype=torch.uint8, device="cuda")
+        run_p = lambda: gsa.gsa_project(p, d_model, Hs, Wt, po["qI"], po["kI"], po["w"], po["g1"], po["g2"], ws_p, stream)
+        for _ in range(3):
+            run_p()
+        pe0, pe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        pe0.record(stream)
+        for _ in range(5):
+            run_p()
+        pe1.record(stream)
+        torch.cuda.synchronize()
+        assert gsa.gsa_device_status(ws_p) == 0
+        p_ms = pe0.elapsed_time(pe1) / 5
+        tf = 2.0 * M * d_model * n_cols / (p_ms * 1e-3) / 1e12
+        projection = {"kernel": "gsa_project_kernel", "ms": p_ms, "tflops": tf, "bound": "tensor",
+                      "peak": peaks["bf16_tflops"], "frac": tf / peaks["bf16_tflops"],
+                      "shape": f"M={M} tokens, K={d_model}, N={n_cols} stacked output columns"}
+        del Hs, Wt, po
+
     # ---- end to end through the host-buffer entry point ------------------------------------
     e2e = None
     if not args.no_e2e:
@@ -326,7 +355,8 @@ def main():
                 "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                 "config": workload_config(cfg), "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
-                "roofline": roofline, "cpu_baseline": cpu_baseline, "stages": stages}
+                "roofline": roofline, "cpu_baseline": cpu_baseline, "stages": stages,
+                "upstream_projection": projection}
         print(json.dumps(line))
     if world > 1:
         import torch.distributed as dist

@@ -96,6 +96,22 @@ int gsa_indexer_scores(const gsa_params_t *p, const void *qI, const void *kI, co
                        size_t ws_bytes, void *stream);
 
 /*
+ * Upstream projections of the layer (text below Eq. 7; Eq. 9; Eq. 10) as one tensor-core GEMM:
+ *     q^I_j = h W^Iq_j,   k^I = h W^Ik,   w_j = sigmoid(h W^Iw_j),   g1 logits = h W^g_O,   g2 logits = h W^g_V.
+ * Needs Lq == Lk (one hidden state per position).  The outputs are exactly the inputs of gsa_forward.
+ *   H      [B * Lk, d_model] bf16 hidden states, d_model a multiple of 8
+ *   Wt     [gsa_project_columns(p), d_model] bf16: the weight matrices transposed and stacked, one
+ *          row of d_model per output column, in the order q^I (HI*dI rows; head-major), k^I (dI),
+ *          head weights (8 rows, the first HI used), g1 (n_h*d_h), g2 (n_kv*d_h)
+ *   qI [B,Lk,HI,dI], kI [B,Lk,dI], g1_logits [B,Lk,n_h,d_h], g2_logits [B,Lk,n_kv,d_h] bf16 (fp32
+ *   accumulation, rounded once); w [B,Lk,HI] fp32, after the sigmoid
+ *   ws     workspace, ws_bytes >= 256 (device status word)
+ */
+int gsa_project_columns(const gsa_params_t *p, int32_t *columns);
+int gsa_project(const gsa_params_t *p, int32_t d_model, const void *H, const void *Wt, void *qI, void *kI,
+                float *w, void *g1_logits, void *g2_logits, void *ws, size_t ws_bytes, void *stream);
+
+/*
  * Adaptive sparsity controller, Eq. 8 then Eq. 4, one row at a time:
  *     Var_t = population variance of the n_t visible scores (accumulated in fp64),
  *     k_t   = clamp(floor(k_base * Var_t / v_bar), k_min, k_max)   (k_mode 0),

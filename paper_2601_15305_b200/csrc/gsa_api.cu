@@ -143,6 +143,31 @@ int gsa_indexer_scores(const gsa_params_t* p, const void* qI, const void* kI, co
                                   (int32_t*)ws, st));
 }
 
+int gsa_project_columns(const gsa_params_t* p, int32_t* columns) {
+    int rc = check_params(p);
+    if (rc) return rc;
+    if (!columns) return GSA_ERR_INVALID_ARG;
+    *columns = project_columns(*p);
+    return GSA_OK;
+}
+
+int gsa_project(const gsa_params_t* p, int32_t d_model, const void* H, const void* Wt, void* qI, void* kI,
+                float* w, void* g1_logits, void* g2_logits, void* ws, size_t ws_bytes, void* stream) {
+    int rc = check_params(p);
+    if (rc) return rc;
+    if (p->Lq != p->Lk) return GSA_ERR_INVALID_ARG;           // one hidden state per position, queries = keys
+    if (d_model < 64 || d_model % 8 != 0) return GSA_ERR_UNSUPPORTED_SHAPE;
+    if ((int64_t)p->B * p->Lk >= (1ll << 31)) return GSA_ERR_UNSUPPORTED_SHAPE;
+    const void* ptrs[] = {H, Wt, qI, kI, w, g1_logits, g2_logits};
+    for (const void* q : ptrs) if (!q || !aligned16(q)) return GSA_ERR_INVALID_ARG;
+    if (!ws || ws_bytes < (size_t)kStatusBytes || !aligned16(ws)) return GSA_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, st);
+    if (e != cudaSuccess) return cuda_rc(e);
+    return cuda_rc(launch_project(*p, d_model, (const bf16*)H, (const bf16*)Wt, (bf16*)qI, (bf16*)kI, w,
+                                  (bf16*)g1_logits, (bf16*)g2_logits, (int32_t*)ws, st));
+}
+
 int gsa_adaptive_topk(const gsa_params_t* p, const float* scores, int64_t row_stride, int32_t* idx,
                       int32_t* kt, float* var, void* ws, size_t ws_bytes, void* stream) {
     int rc = check_params(p);

@@ -72,6 +72,12 @@ void set_attn_range_keys(int keys);
 // its start, then the gated values of the allocation-free entry point)
 cudaError_t static_scratch_address(void** ptr);
 
+// upstream projections: C = H * Wt^T routed to q^I, k^I, head weights (sigmoid), g1 and g2 logits
+int project_columns(const gsa_params_t& p);
+cudaError_t launch_project(const gsa_params_t& p, int d_model, const __nv_bfloat16* H, const __nv_bfloat16* Wt,
+                           __nv_bfloat16* qI, __nv_bfloat16* kI, float* w, __nv_bfloat16* g1, __nv_bfloat16* g2,
+                           int32_t* dev_status, cudaStream_t st);
+
 // ---- device helpers ------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return (uint32_t)__cvta_generic_to_shared(p);

@@ -132,7 +132,12 @@ gsa_indexer_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
     const int tile0 = blockIdx.x * a.tiles_per_cta;
     const int ntiles = min(a.tiles_per_cta, tiles_group - tile0);
     if (ntiles <= 0) return;                                          // whole CTA, before any barrier
-    if (*reinterpret_cast<volatile int32_t*>(a.dev_status) != kDevOk) return;   // an earlier CTA gave up
+    {   // an earlier CTA gave up: leave, all threads together (one thread reads the word)
+        __shared__ int s_go;
+        if (threadIdx.x == 0) s_go = *reinterpret_cast<volatile int32_t*>(a.dev_status) == kDevOk;
+        __syncthreads();
+        if (!s_go) return;
+    }
 
     extern __shared__ unsigned char dyn_smem_raw[];
     const uint32_t raw_u32 = smem_u32(dyn_smem_raw);

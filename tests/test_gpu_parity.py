@@ -507,3 +507,38 @@ def test_forward_decode_full_size():
         U.check_e2e_indices(o, idx[b].cpu().numpy(), kt[b].cpu().numpy(), o["scores"], [cfg.Lk])
         U.check_out(out[b].float().cpu().numpy(), o["out"])
     assert (kt >= cfg.k_min).all() and (kt <= cfg.k_max).all()
+
+
+# ------------------------------------------------------------------------------------------ projections
+@pytest.mark.parametrize("base,L,d_model", [("tiny", 300, 192), ("l8k", 1000, 2048)])
+def test_project_matches_oracle(base, L, d_model):
+    """gsa_project (tcgen05 GEMM + routing epilogue) against the fp64 oracle: ragged token count and a
+    last column tile that is only partly used."""
+    cfg = CONFIGS[base].with_(name="proj", B=2, Lq=L, Lk=L)
+    p = gsa.make_params(cfg)
+    n_cols = gsa.gsa_project_columns(p)
+    g = torch.Generator().manual_seed(23)
+    M = cfg.B * L
+    H = torch.randn(M, d_model, generator=g).to(torch.bfloat16)
+    Wt = (torch.randn(n_cols, d_model, generator=g) / d_model ** 0.5).to(torch.bfloat16)
+    dev = lambda *s, dt=torch.bfloat16: torch.full(s, float("nan"), dtype=dt, device="cuda")
+    qI, kI = dev(cfg.B, L, cfg.HI, cfg.dI), dev(cfg.B, L, cfg.dI)
+    w = dev(cfg.B, L, cfg.HI, dt=torch.float32)
+    g1, g2 = dev(cfg.B, L, cfg.n_h, cfg.d_h), dev(cfg.B, L, cfg.n_kv, cfg.d_h)
+    ws = torch.zeros(1024, dtype=torch.uint8, device="cuda")
+    gsa.gsa_project(p, d_model, H.cuda(), Wt.cuda(), qI, kI, w, g1, g2, ws)
+    assert gsa.gsa_device_status(ws) == 0
+    rows = np.unique(np.concatenate([np.arange(0, M, 37), [0, 127, 128, M - 1]]))
+    o = oracle.project(U.oracle_params(cfg), d_model, H, Wt, rows)
+    sel = torch.from_numpy(rows).cuda()
+
+    def close_bf16(got, want):          # fp32 accumulation rounded to bf16 once: half an ulp = 2^-9 relative
+        got = got.reshape(M, -1)[sel].float().cpu().numpy().astype(np.float64)
+        assert np.isfinite(got).all()
+        assert (np.abs(got - want) <= 2.0 ** -8 * np.abs(want) + 1e-5).all()
+
+    close_bf16(qI, o["qI"]); close_bf16(kI, o["kI"]); close_bf16(g1, o["g1"]); close_bf16(g2, o["g2"])
+    gw = w.reshape(M, -1)[sel].cpu().numpy().astype(np.float64)
+    assert np.abs(gw - o["w"]).max() <= 2e-6          # fp32 sigmoid of an fp32-accumulated logit
+    for t in (qI, kI, w, g1, g2):                      # every element written
+        assert not torch.isnan(t.float()).any()
