@@ -112,6 +112,16 @@ int gsa_project(const gsa_params_t *p, int32_t d_model, const void *H, const voi
                 float *w, void *g1_logits, void *g2_logits, void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * Output projection (Sec. 2.1: the heads are concatenated and projected by W_O):
+ *     u[token, :] = out[token, :, :] (n_h * d_h values) * W_O,    the same tensor-core GEMM kernel.
+ *   attn_out [B, Lq, n_h, d_h] bf16 (the `out` of gsa_forward);  Wo_t [d_model, n_h*d_h] bf16 (W_O
+ *   transposed: one row per output column);  u [B, Lq, d_model] bf16;  d_model a multiple of 8
+ *   ws     workspace, ws_bytes >= 256 (device status word)
+ */
+int gsa_output_projection(const gsa_params_t *p, int32_t d_model, const void *attn_out, const void *Wo_t,
+                          void *u, void *ws, size_t ws_bytes, void *stream);
+
+/*
  * Adaptive sparsity controller, Eq. 8 then Eq. 4, one row at a time:
  *     Var_t = population variance of the n_t visible scores (accumulated in fp64),
  *     k_t   = clamp(floor(k_base * Var_t / v_bar), k_min, k_max)   (k_mode 0),

@@ -204,3 +204,15 @@ def project(p: OracleParams, d_model: int, H, Wt, rows_m: Sequence[int]):
                                   ctypes.c_int(n), _ptr(out["qI"]), _ptr(out["kI"]), _ptr(out["w"]),
                                   _ptr(out["g1"]), _ptr(out["g2"]))
     return out
+
+
+def out_project(X, Wt, rows_m: Sequence[int]) -> np.ndarray:
+    """Output projection (concatenated heads times W_O) of the listed token rows: X [M, K], Wt [N, K] -> [n, N] fp64."""
+    X, Wt = _f32(X), _f32(Wt)
+    rows_m = _i32(rows_m).reshape(-1)
+    assert X.ndim == 2 and Wt.ndim == 2 and X.shape[1] == Wt.shape[1]
+    assert rows_m.min(initial=0) >= 0 and rows_m.max(initial=0) < X.shape[0]
+    u = np.empty((len(rows_m), Wt.shape[0]))
+    lib().gsa_oracle_out_project_rows(ctypes.c_int(X.shape[1]), ctypes.c_int(Wt.shape[0]), _ptr(X), _ptr(Wt),
+                                      _ptr(rows_m), ctypes.c_int(len(rows_m)), _ptr(u))
+    return u

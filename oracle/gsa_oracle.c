@@ -203,6 +203,22 @@ void gsa_oracle_project_rows(const gsa_oracle_params *p, int d_model, const floa
     }
 }
 
+/* ---- output projection (Sec. 2.1: concatenated heads times W_O) -------------- */
+/* u[token, n] = sum_c X[token, c] * Wt[n, c] for the listed tokens; X is the gated attention output
+ * with its n_h heads concatenated ([tokens, K]), Wt the transposed weight ([N, K]). */
+void gsa_oracle_out_project_rows(int K, int N, const float *X, const float *Wt, const int32_t *rows_m,
+                                 int n_rows, double *u)
+{
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int r = 0; r < n_rows; ++r)
+        for (int n = 0; n < N; ++n) {
+            double acc = 0.0;
+            for (int c = 0; c < K; ++c)
+                acc += (double)X[(size_t)rows_m[r] * K + c] * (double)Wt[(size_t)n * K + c];
+            u[(size_t)r * N + n] = acc;
+        }
+}
+
 /* ---- drivers over a list of (batch, query) rows -------------------------- */
 
 /* scores of the listed rows: out[r, 0..n_t) in a [n_rows, Lk] double array */

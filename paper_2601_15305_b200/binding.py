@@ -21,7 +21,7 @@ EXPORTS = (
     "gsa_forward", "gsa_forward_host_arena_bytes", "gsa_forward_host", "gsa_device_status",
     "gsa_launch_count", "gsa_debug_set_indexer_path", "gsa_profile_set_events", "gsa_status_string",
     "gsa_sparse_gated_attn_fwd_static", "gsa_attn_workspace_bytes", "gsa_debug_set_attn_range_keys",
-    "gsa_select_fallback_rows", "gsa_project", "gsa_project_columns",
+    "gsa_select_fallback_rows", "gsa_project", "gsa_project_columns", "gsa_output_projection",
 )
 
 STATIC_SCRATCH_BYTES = 32 << 20     # GSA_STATIC_SCRATCH_BYTES of include/gsa.h
@@ -128,6 +128,12 @@ def gsa_project(p, d_model: int, H, Wt, qI, kI, w, g1, g2, ws, stream=None) -> N
     _check(lib().gsa_project(ctypes.byref(p), ctypes.c_int32(d_model), _dp(H, BF16), _dp(Wt, BF16), _dp(qI, BF16),
                              _dp(kI, BF16), _dp(w, F32), _dp(g1, BF16), _dp(g2, BF16), _dp(ws),
                              ctypes.c_size_t(ws.numel() * ws.element_size()), _stream(stream)), "gsa_project")
+
+
+def gsa_output_projection(p, d_model: int, attn_out, Wo_t, u, ws, stream=None) -> None:
+    _check(lib().gsa_output_projection(ctypes.byref(p), ctypes.c_int32(d_model), _dp(attn_out, BF16), _dp(Wo_t, BF16),
+                                       _dp(u, BF16), _dp(ws), ctypes.c_size_t(ws.numel() * ws.element_size()),
+                                       _stream(stream)), "gsa_output_projection")
 
 
 def gsa_adaptive_topk(p, scores, row_stride: int, idx, kt, var=None, ws=None, stream=None) -> None:

@@ -168,6 +168,22 @@ int gsa_project(const gsa_params_t* p, int32_t d_model, const void* H, const voi
                                   (bf16*)g1_logits, (bf16*)g2_logits, (int32_t*)ws, st));
 }
 
+int gsa_output_projection(const gsa_params_t* p, int32_t d_model, const void* attn_out, const void* Wo_t, void* u,
+                          void* ws, size_t ws_bytes, void* stream) {
+    int rc = check_params(p);
+    if (rc) return rc;
+    if (d_model < 8 || d_model % 8 != 0) return GSA_ERR_UNSUPPORTED_SHAPE;
+    if ((int64_t)p->B * p->Lq >= (1ll << 31)) return GSA_ERR_UNSUPPORTED_SHAPE;
+    const void* ptrs[] = {attn_out, Wo_t, u};
+    for (const void* q : ptrs) if (!q || !aligned16(q)) return GSA_ERR_INVALID_ARG;
+    if (!ws || ws_bytes < (size_t)kStatusBytes || !aligned16(ws)) return GSA_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, st);
+    if (e != cudaSuccess) return cuda_rc(e);
+    return cuda_rc(launch_gemm_bf16(p->B * p->Lq, p->n_h * p->d_h, d_model, (const bf16*)attn_out, (const bf16*)Wo_t,
+                                    (bf16*)u, (int32_t*)ws, st));
+}
+
 int gsa_adaptive_topk(const gsa_params_t* p, const float* scores, int64_t row_stride, int32_t* idx,
                       int32_t* kt, float* var, void* ws, size_t ws_bytes, void* stream) {
     int rc = check_params(p);

@@ -78,6 +78,9 @@ cudaError_t launch_project(const gsa_params_t& p, int d_model, const __nv_bfloat
                            __nv_bfloat16* qI, __nv_bfloat16* kI, float* w, __nv_bfloat16* g1, __nv_bfloat16* g2,
                            int32_t* dev_status, cudaStream_t st);
 
+cudaError_t launch_gemm_bf16(int M, int K, int N, const __nv_bfloat16* A, const __nv_bfloat16* Bt, __nv_bfloat16* C,
+                             int32_t* dev_status, cudaStream_t st);
+
 // ---- device helpers ------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return (uint32_t)__cvta_generic_to_shared(p);

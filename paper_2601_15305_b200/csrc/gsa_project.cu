@@ -233,4 +233,28 @@ cudaError_t launch_project(const gsa_params_t& p, int d_model, const __nv_bfloat
     return cudaGetLastError();
 }
 
+
+// C[M, N] = A[M, K] * Bt[N, K]^T, bf16 in, fp32 accumulate, bf16 out: the same kernel with a single
+// output block (used for the output projection W_O).
+cudaError_t launch_gemm_bf16(int M, int K, int N, const __nv_bfloat16* A, const __nv_bfloat16* Bt, __nv_bfloat16* C,
+                             int32_t* dev_status, cudaStream_t st) {
+    ProjArgs a;
+    a.qI = C; a.kI = nullptr; a.w = nullptr; a.g1 = nullptr; a.g2 = nullptr; a.dev_status = dev_status;
+    a.M = M; a.K = K; a.N = N;
+    a.n_q = N; a.n_k = 0; a.HI = 0; a.n_g1 = 0; a.n_g2 = 0;
+    a.m_tiles = (M + kTileM - 1) / kTileM;
+    a.n_tiles = (N + kTileN - 1) / kTileN;
+    CUtensorMap tm_a, tm_b;
+    if (!make_kblock_tmap(&tm_a, A, (uint64_t)M, (uint64_t)K, kTileM)) return cudaErrorUnknown;
+    if (!make_kblock_tmap(&tm_b, Bt, (uint64_t)N, (uint64_t)K, kTileN)) return cudaErrorUnknown;
+    cudaError_t e = cudaFuncSetAttribute(gsa_project_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal);
+    if (e != cudaSuccess) return e;
+    int sms = 148, dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int tiles = a.m_tiles * a.n_tiles;
+    gsa_project_kernel<<<tiles < sms ? tiles : sms, kPThreads, kSmemTotal, st>>>(tm_a, tm_b, a);
+    ++g_launches;
+    return cudaGetLastError();
+}
+
 }  // namespace gsa

@@ -542,3 +542,22 @@ def test_project_matches_oracle(base, L, d_model):
     assert np.abs(gw - o["w"]).max() <= 2e-6          # fp32 sigmoid of an fp32-accumulated logit
     for t in (qI, kI, w, g1, g2):                      # every element written
         assert not torch.isnan(t.float()).any()
+
+
+def test_output_projection_matches_oracle():
+    cfg = CONFIGS["l8k"].with_(name="wo", B=1, Lq=777, Lk=777)
+    p = gsa.make_params(cfg)
+    d_model = 2048
+    g = torch.Generator().manual_seed(29)
+    K = cfg.n_h * cfg.d_h
+    X = torch.randn(cfg.B, cfg.Lq, cfg.n_h, cfg.d_h, generator=g).to(torch.bfloat16)
+    Wt = (torch.randn(d_model, K, generator=g) / K ** 0.5).to(torch.bfloat16)
+    u = torch.full((cfg.B, cfg.Lq, d_model), float("nan"), dtype=torch.bfloat16, device="cuda")
+    ws = torch.zeros(1024, dtype=torch.uint8, device="cuda")
+    gsa.gsa_output_projection(p, d_model, X.cuda(), Wt.cuda(), u, ws)
+    assert gsa.gsa_device_status(ws) == 0
+    rows = np.unique(np.concatenate([np.arange(0, cfg.Lq, 41), [127, 128, cfg.Lq - 1]]))
+    want = oracle.out_project(X.reshape(-1, K), Wt, rows)
+    got = u.reshape(-1, d_model)[torch.from_numpy(rows).cuda()].float().cpu().numpy().astype(np.float64)
+    assert (np.abs(got - want) <= 2.0 ** -8 * np.abs(want) + 1e-5).all()     # fp32 accumulate, one bf16 rounding
+    assert not torch.isnan(u.float()).any()

@@ -414,6 +414,19 @@ def test_projections_copy_columns_closed_form_sigmoid_and_library_matmul():
     np.testing.assert_allclose(o["g2"], full[:, 56:72], rtol=1e-13, atol=1e-13)
 
 
+def test_output_projection_one_hot_and_library_matmul():
+    rng = np.random.default_rng(4)
+    X = rng.standard_normal((6, 10)).astype(np.float32)
+    Wt = np.zeros((4, 10), np.float32)
+    Wt[2, 7] = 3.0                                       # output 2 <- 3 * input 7
+    u = oracle.out_project(X, Wt, [5, 1])
+    np.testing.assert_allclose(u[:, 2], 3.0 * X[[5, 1], 7].astype(np.float64), atol=1e-15)
+    assert np.count_nonzero(u) == 2
+    Wt = rng.standard_normal((4, 10)).astype(np.float32)
+    np.testing.assert_allclose(oracle.out_project(X, Wt, np.arange(6)), X.astype(np.float64) @ Wt.astype(np.float64).T,
+                               rtol=1e-13, atol=1e-13)
+
+
 def test_paper_printed_cost_model():
     """Appendix A prints d^I H^I/(d n_h) ~ 0.002 and a 12.8x speed-up for its parameters."""
     vals = {}
