@@ -5,17 +5,21 @@
 //   0  a sample of the row (256 chunks of 32 consecutive scores, evenly spread) is histogrammed;
 //      it gives a threshold key tau that about 1.3 * min(k_max, n) scores of the row should reach
 //      (k_t itself is not known yet: it depends on the variance of the whole row)
-//   1  full read, no block-wide barrier: the row is cut into at most 512 chunks (128 * 2^s scores each)
-//      that are dealt to the 16 warps round-robin, so each warp sees an even sample of the row.  Loads are fully coalesced float4s; every score goes into fp64 sum and
-//      sum of squares; a score that reaches tau (one float compare) is appended, in position order, to
-//      the warp's private candidate list in shared memory, and each chunk remembers where its entries
-//      start and how many it has.   -> Var, k_t
-//   2  on chip: radix rounds over the candidates give the exact threshold key T of the k_t-th largest
-//      score and how many keys equal to T are taken; the chunks are then walked in position order
-//      (counts per chunk, one block scan, ballot-ordered emission) to write S_t ascending.
+//   1  full read, no block-wide barrier: the row is cut into chunks of 512 consecutive scores that
+//      are dealt to the 16 warps round-robin, so each warp sees an even sample of the row.  Loads are
+//      fully coalesced float4s, one chunk ahead, turned through shared memory so that a lane holds 16
+//      consecutive scores; every score goes into fp64 sum and sum of squares; the position of a score
+//      that reaches tau (one float compare) goes into the candidate list in shared memory: a warp scan
+//      of the lanes' counts orders the chunk's candidates, one shared-memory atomic claims their space,
+//      and a table remembers where each chunk's entries start and how many there are.   -> Var, k_t
+//   2  on chip: the candidates' keys are fetched (one per thread and round); radix rounds over them give
+//      the exact threshold key T of the k_t-th largest score and how many keys equal to T are taken;
+//      the chunks are then walked in position order (counts per thread, one block scan, emission) to
+//      write S_t ascending.
 // Equal keys go to the lower position, so the output is unique.  If the list overflows or comes out
 // shorter than k_t (the sample misjudged the row: huge ties, scores sorted by position, ...) the CTA
-// falls back to radix rounds over the whole row in global memory: slower, same result.
+// falls back to radix rounds over the whole row in global memory: slower, same result.  Rows of more
+// than 2048 chunks (1 Mi scores) always take that path.
 #include "gsa_common.cuh"
 
 namespace gsa {
@@ -29,8 +33,10 @@ constexpr int kBins = 1 << kBinsLog2;
 constexpr int kBinsPerThread = kBins / kSelThreads;   // 8
 constexpr int kListCap = 8192;                        // entries of the candidate lists (all warps)
 constexpr int kListPerThread = kListCap / kSelThreads;  // 16
-constexpr int kWarpCap = kListCap / kSelWarps;        // entries of one warp's private list: 512
-constexpr int kMaxChunks = 512;
+constexpr int kIter = 512;                            // scores a warp takes per iteration (= one chunk)
+constexpr int kMaxChunks = 2048;                      // rows of up to kIter * kMaxChunks = 1 Mi scores are listed
+constexpr int kStageFloats = kListCap / kSelWarps;    // a warp's staging area inside list_key: 512 floats
+static_assert(kStageFloats == kIter, "one iteration must fit the warp's staging area");
 constexpr int kSampleChunks = 256;                    // sample = 256 chunks of 32 scores
 constexpr int kSamplePerThread = kSampleChunks * 32 / kSelThreads;   // 16
 
@@ -56,8 +62,8 @@ __device__ __forceinline__ uint32_t order_key(float x) {
 
 struct SelShared {
     uint32_t hist[kBins];
-    uint16_t list_rel[kListCap];      // candidate position relative to the start of its chunk
-    uint32_t list_key[kListCap];
+    uint32_t list_pos[kListCap];      // candidate positions; the entries of one chunk are consecutive and ascending
+    uint32_t list_key[kListCap];      // their order keys (pass 1 stages scores in here first)
     double red_a[kSelWarps];
     double red_b[kSelWarps];
     uint32_t red_min[kSelWarps];
@@ -65,11 +71,9 @@ struct SelShared {
     uint32_t warp_tot[2][kSelWarps];
     uint32_t seg_gt[kSelWarps];
     uint32_t seg_eq[kSelWarps];
-    uint16_t ch_off[kMaxChunks];      // chunk c: its entries start at list[(c % 16) * kWarpCap + ch_off[c]]
+    uint16_t ch_off[kMaxChunks];      // table chunk c (128 or 512 consecutive scores): its entries start at list[ch_off[c]]
     uint16_t ch_cnt[kMaxChunks];      //          and there are ch_cnt[c] of them
-    uint16_t ch_gt[kMaxChunks];       // selected entries of the chunks before c: keys > T ...
-    uint16_t ch_eq[kMaxChunks];       // ... and keys == T (before the cut at need_eq)
-    uint32_t wl_cnt[kSelWarps];       // live entries of each warp's list
+    uint32_t list_total;              // entries handed out so far
     uint32_t found_bin;
     uint32_t found_above;
     uint32_t overflow;
@@ -165,34 +169,6 @@ __device__ __forceinline__ void radix_rounds(SelShared& sh, int count, KeyOf key
     need_eq = want;
 }
 
-// The same over the 16 per-warp candidate lists: each warp walks its own list (no dead slots).
-__device__ __forceinline__ void radix_rounds_lists(SelShared& sh, uint32_t lo, uint32_t hi, uint32_t want,
-                                                   uint32_t& T, uint32_t& need_eq) {
-    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    const uint32_t* const wl_key = sh.list_key + wid * kWarpCap;
-    const int my_cnt = (int)sh.wl_cnt[wid];
-    while (true) {
-        const uint32_t span = hi - lo;
-        const int shift = shift_for(span);
-        for (int i = tid; i < kBins; i += kSelThreads) sh.hist[i] = 0u;
-        __syncthreads();
-        for (int j = lane; j < my_cnt; j += 32) {
-            const uint32_t key = wl_key[j];
-            if (key - lo <= span) atomicAdd(&sh.hist[(key - lo) >> shift], 1u);
-        }
-        __syncthreads();
-        uint32_t fb, fa;
-        find_bin(sh, want, fb, fa);
-        want -= fa;
-        const uint32_t nlo = lo + (fb << shift);
-        const uint32_t nhi = shift == 0 ? nlo : min(hi, nlo + ((1u << shift) - 1u));
-        lo = nlo; hi = nhi;
-        if (shift == 0) break;
-    }
-    T = lo;
-    need_eq = want;
-}
-
 // block-wide exclusive scan of one value per thread; returns the exclusive prefix and the total.
 // `slot` alternates 0/1 between consecutive calls so one barrier per call suffices.
 __device__ __forceinline__ uint32_t block_excl_scan(SelShared& sh, uint32_t v, int slot, uint32_t& total) {
@@ -242,14 +218,22 @@ __global__ void __launch_bounds__(kSelThreads, 2) gsa_select_kernel(const Select
     const int64_t orow = a.il.row(b, t);
     int32_t* __restrict__ out_idx = a.idx + orow * a.k_max;
     const bool short_row = n <= kListCap;                     // the whole row fits the list: no sampling
+    const int nchunks = (n + kIter - 1) / kIter;              // chunks of 512 consecutive scores (long rows)
+    const bool listed = !short_row && nchunks <= kMaxChunks;  // longer rows go straight to the whole-row path
+    // the table of list segments has one entry per 128 scores (8 lanes of an iteration) while that fits,
+    // else one per 512: finer entries spread the emission over more threads
+    const int lpc_shift = nchunks * 4 <= kMaxChunks ? 3 : 5;
+    const int lpc = 1 << lpc_shift;                           // lanes per table chunk
+    const int ntab = (n + 16 * lpc - 1) / (16 * lpc);         // table chunks of 16 * lpc scores
 
-    if (tid == 0) sh.overflow = 0u;
+    if (tid == 0) { sh.overflow = 0u; sh.list_total = 0u; }
 
     // ---- pass 0 (long rows): candidate threshold from a sample --------------------------------
     // 256 chunks of 32 consecutive scores, evenly spread, give (a) an estimate of the row's variance and
     // with it an upper estimate k_hi of the budget, (b) a key tau that about 1.3 * k_hi scores reach.
-    float tau_f = -INFINITY;
-    if (!short_row) {
+    float tau_f = listed ? -INFINITY : INFINITY;              // not listed: nothing is a candidate
+    uint32_t tau_key = 0u;                                    // the same threshold as an order key
+    if (listed) {
         const int chunks = n >> 5;                            // full chunks of 32
         uint32_t skey[kSamplePerThread];
         uint32_t smin = 0xFFFFFFFFu, smax = 0u;
@@ -307,20 +291,16 @@ __global__ void __launch_bounds__(kSelThreads, 2) gsa_select_kernel(const Select
         const uint32_t tau = smin + (fb << shift);            // lower edge of that bin
         // as a float: x >= tau_f  <=>  order_key(x) >= tau for every non-NaN x
         tau_f = __uint_as_float((tau & 0x80000000u) ? (tau & 0x7FFFFFFFu) : ~tau);
+        tau_key = tau;
     }
     __syncthreads();
 
-    // ---- pass 1: fp64 moments of every score; candidates into lists ----------------------------
+    // ---- pass 1: fp64 moments of every score; candidates into the list -------------------------
     double s1 = 0.0, s2 = 0.0;
-    uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;                   // range of the keys that went into the list(s)
-    // The row is cut into rounds of 128 consecutive scores (one coalesced float4 load of a warp) and
-    // chunks of 2^cshift rounds, at most 512 chunks; chunk c belongs to warp c % 16.
-    constexpr int kRound = 128;
-    const int n_rounds = (n + kRound - 1) / kRound;
-    int cshift = 0;
-    while (((n_rounds + (1 << cshift) - 1) >> cshift) > kMaxChunks) ++cshift;
-    const int chunk_elems = kRound << cshift;
-    const int nchunks = (n_rounds + (1 << cshift) - 1) >> cshift;
+    uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;                   // range of the keys that went into the list
+    // Long rows are cut into chunks of 512 consecutive scores, dealt to the 16 warps round-robin (chunk c
+    // belongs to warp c % 16), one chunk per warp iteration.  Rows with more than kMaxChunks chunks are
+    // not listed at all (tau_f = +inf below): they take the whole-row path.
     if (short_row) {
         // the list is simply the row, in order
         for (int i = tid; i < n; i += kSelThreads) {
@@ -334,114 +314,105 @@ __global__ void __launch_bounds__(kSelThreads, 2) gsa_select_kernel(const Select
             kmax = max(kmax, key);
         }
     } else {
-        const int rpc_mask = (1 << cshift) - 1;               // rounds per chunk - 1
-        uint32_t wcnt = 0;                                    // entries in this warp's list (warp-uniform)
+        const int my_iters = wid < nchunks ? (nchunks - wid + kSelWarps - 1) / kSelWarps : 0;
+        kmin = tau_key;                                       // every listed key reaches the threshold
         bool w_over = false;
-        uint16_t* const wl_rel = sh.list_rel + wid * kWarpCap;
-        uint32_t* const wl_key = sh.list_key + wid * kWarpCap;
-        // the warp walks its chunks (wid, wid + 16, ...) round by round, four rounds per iteration
-        const int my_chunks = wid < nchunks ? (nchunks - wid + kSelWarps - 1) / kSelWarps : 0;
-        const int my_rounds = my_chunks << cshift;
-        auto round_start = [&](int j) -> int {                // first score of the warp's j-th round
-            return (wid + kSelWarps * (j >> cshift)) * chunk_elems + (j & rpc_mask) * kRound;
-        };
-        for (int j0 = 0; j0 < my_rounds; j0 += 4) {
-            int rs[4];
+        // The 512 scores of an iteration arrive by coalesced 16-byte loads (lane l gets scores 4l..4l+3 of
+        // each 128) and are turned, through shared memory, so that lane l holds scores 16l..16l+15: a
+        // lane's candidates are then consecutive in position order and one warp scan of the counts places
+        // them.  The staging buffer is the warp's part of list_key, which is filled only after this pass.
+        // 16-byte slot q (= position / 4) is kept at q ^ ((q >> 3) & 3): no bank conflicts either way.
+        float4* const tb = reinterpret_cast<float4*>(sh.list_key + wid * kStageFloats);
+        const int wslot = lane ^ ((lane >> 3) & 3);
+        const int rsw = (lane >> 1) & 3;
+        // loads run one iteration ahead
+        float4 ld[4];
+        if (my_iters > 0 && (wid + 1) * kIter <= n) {
+            const float4* const gp = reinterpret_cast<const float4*>(grow + wid * kIter) + lane;
 #pragma unroll
-            for (int v = 0; v < 4; ++v) rs[v] = j0 + v < my_rounds ? round_start(j0 + v) : n;   // n: nothing there
-            uint32_t flags = 0;
-            if (rs[3] + kRound <= n && rs[0] + kRound <= n && rs[1] + kRound <= n && rs[2] + kRound <= n) {
-                float4 x4[4];
+            for (int v = 0; v < 4; ++v) ld[v] = __ldg(gp + 32 * v);
+        }
+        for (int j = 0; j < my_iters; ++j) {
+            const int c = wid + kSelWarps * j;                // this iteration's chunk
+            const int rs0 = c * kIter;                        // its first score
+            uint32_t flags = 0;                               // bit e: score rs0 + 16 lane + e is a candidate
+            if (rs0 + kIter <= n) {
+                __syncwarp();                                 // the previous iteration's slots have been read
 #pragma unroll
-                for (int v = 0; v < 4; ++v) x4[v] = __ldg(reinterpret_cast<const float4*>(grow + rs[v]) + lane);
+                for (int v = 0; v < 4; ++v) tb[wslot + 32 * v] = ld[v];
+                __syncwarp();
 #pragma unroll
-                for (int v = 0; v < 4; ++v) {
-                    const float xs[4] = {x4[v].x, x4[v].y, x4[v].z, x4[v].w};
+                for (int u = 0; u < 4; ++u) {
+                    const float4 xv = tb[4 * lane + (u ^ rsw)];
+                    const float xs[4] = {xv.x, xv.y, xv.z, xv.w};
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         const double xd = (double)xs[e];
                         s1 += xd;
                         s2 = fma(xd, xd, s2);
-                        flags |= (xs[e] >= tau_f ? 1u : 0u) << (v * 4 + e);
+                        flags |= (xs[e] >= tau_f ? 1u : 0u) << (u * 4 + e);
                     }
                 }
-            } else {
+            } else {                                          // the row's last, partial chunk
 #pragma unroll
-                for (int v = 0; v < 4; ++v)
+                for (int e = 0; e < 16; ++e) {
+                    const int i = rs0 + lane * 16 + e;
+                    if (i < n) {
+                        const float x = __ldg(grow + i);
+                        const double xd = (double)x;
+                        s1 += xd;
+                        s2 = fma(xd, xd, s2);
+                        flags |= (x >= tau_f ? 1u : 0u) << e;
+                    }
+                }
+            }
+            // next iteration's loads, issued before the scan and the list stores so that this work covers
+            // part of their latency
+            if (j + 1 < my_iters && rs0 + (kSelWarps + 1) * kIter <= n) {
+                const float4* const gp = reinterpret_cast<const float4*>(grow + rs0 + kSelWarps * kIter) + lane;
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int i = rs[v] + lane * 4 + e;
-                        if (i < n) {
-                            const float x = __ldg(grow + i);
-                            const double xd = (double)x;
-                            s1 += xd;
-                            s2 = fma(xd, xd, s2);
-                            flags |= (x >= tau_f ? 1u : 0u) << (v * 4 + e);
+                for (int v = 0; v < 4; ++v) ld[v] = __ldg(gp + 32 * v);
+            }
+            const uint32_t cnt = __popc(flags);
+            uint32_t inc = cnt;                               // candidates of lanes 0..lane
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+                if (lane >= o) inc += u;
+            }
+            const uint32_t iter_total = __shfl_sync(0xFFFFFFFFu, inc, 31);
+            // the iteration's entries are consecutive in the list: lane 31 claims the space; the last lane
+            // of every table chunk (8 or 32 lanes) notes where the chunk's entries start and how many there are
+            if (listed) {
+                uint32_t base = 0;
+                if (lane == 31 && iter_total != 0u) base = atomicAdd(&sh.list_total, iter_total);
+                base = __shfl_sync(0xFFFFFFFFu, base, 31);
+                const int first = lane & ~(lpc - 1);                        // first lane of this lane's chunk
+                uint32_t before = __shfl_sync(0xFFFFFFFFu, inc, first > 0 ? first - 1 : 0);
+                if (first == 0) before = 0u;                                // candidates of the chunks before it
+                if ((lane & (lpc - 1)) == lpc - 1) {
+                    const int tc = (c << (5 - lpc_shift)) + (lane >> lpc_shift);
+                    if (tc < ntab) {
+                        sh.ch_off[tc] = (uint16_t)min(base + before, (uint32_t)kListCap);
+                        sh.ch_cnt[tc] = (uint16_t)(inc - before);
+                    }
+                }
+                if (iter_total != 0u) {
+                    if (base + iter_total <= (uint32_t)kListCap) {
+                        uint32_t pos = base + inc - cnt;
+                        const uint32_t ib = (uint32_t)(rs0 + lane * 16);
+                        uint32_t f = flags;
+                        while (f) {                           // one candidate per pass and lane
+                            sh.list_pos[pos++] = ib + (uint32_t)(__ffs(f) - 1);
+                            f &= f - 1;
                         }
+                    } else {
+                        w_over = true;
                     }
-            }
-            // position order inside the iteration is (round v, lane, e): one packed scan gives, for each of
-            // the four rounds, how many candidates the lower lanes hold (bytes: at most 128 per round)
-            const uint32_t packed = __popc(flags & 0xFu) | (__popc(flags & 0xF0u) << 8) |
-                                    (__popc(flags & 0xF00u) << 16) | (__popc(flags & 0xF000u) << 24);
-            uint32_t inc = packed;
-            uint32_t t0 = 0, t1 = 0, t2 = 0, t3 = 0;
-            if (__any_sync(0xFFFFFFFFu, flags != 0u)) {
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-                    if (lane >= o) inc += u;
-                }
-                const uint32_t tot = __shfl_sync(0xFFFFFFFFu, inc, 31);
-                t0 = tot & 0xFFu; t1 = (tot >> 8) & 0xFFu; t2 = (tot >> 16) & 0xFFu; t3 = tot >> 24;
-            }
-            const uint32_t excl = inc - packed;
-            // entries of the rounds before round v (two 16-bit fields per word)
-            const uint32_t base_lo = t0 << 16;                              // rounds 0, 1: 0, t0
-            const uint32_t base_hi = ((t0 + t1 + t2) << 16) | (t0 + t1);   // rounds 2, 3
-            const uint32_t iter_total = t0 + t1 + t2 + t3;
-            if (iter_total != 0u) {
-                if (wcnt + iter_total <= (uint32_t)kWarpCap) {
-                    uint32_t f = flags;
-                    while (f) {                                           // one candidate per pass and lane
-                        const int bit = __ffs(f) - 1;
-                        f &= f - 1;
-                        const int v = bit >> 2;
-                        const uint32_t own_before = __popc(flags & ((1u << bit) - 1u) & (0xFu << (v * 4)));
-                        const uint32_t base_v = (((v & 2) ? base_hi : base_lo) >> ((v & 1) * 16)) & 0xFFFFu;
-                        const uint32_t pos = wcnt + base_v + ((excl >> (8 * v)) & 0xFFu) + own_before;
-                        const int rsv = v == 0 ? rs[0] : (v == 1 ? rs[1] : (v == 2 ? rs[2] : rs[3]));
-                        const int i = rsv + lane * 4 + (bit & 3);
-                        wl_rel[pos] = (uint16_t)(((j0 + v) & rpc_mask) * kRound + lane * 4 + (bit & 3));
-                        const uint32_t key = order_key(__ldg(grow + i));  // read again (L1)
-                        wl_key[pos] = key;
-                        kmin = min(kmin, key);
-                        kmax = max(kmax, key);
-                    }
-                } else {
-                    w_over = true;
                 }
             }
-            // chunk table: where each chunk's entries start in this warp's list and how many there are
-            if (lane == 0) {
-                const uint32_t tv[4] = {t0, t1, t2, t3};
-                uint32_t run = wcnt;
-#pragma unroll
-                for (int v = 0; v < 4; ++v)
-                    if (j0 + v < my_rounds) {
-                        const int c = wid + kSelWarps * ((j0 + v) >> cshift);
-                        if (((j0 + v) & rpc_mask) == 0) sh.ch_off[c] = (uint16_t)min(run, (uint32_t)kWarpCap);
-                        run += tv[v];
-                        if (((j0 + v) & rpc_mask) == rpc_mask)
-                            sh.ch_cnt[c] = (uint16_t)(min(run, (uint32_t)kWarpCap) - sh.ch_off[c]);
-                    }
-            }
-            wcnt += iter_total;
         }
-        if (lane == 0) {
-            if (w_over) sh.overflow = 1u;
-            sh.wl_cnt[wid] = min(wcnt, (uint32_t)kWarpCap);
-        }
+        if (w_over && lane == 0) sh.overflow = 1u;
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -450,6 +421,17 @@ __global__ void __launch_bounds__(kSelThreads, 2) gsa_select_kernel(const Select
     }
     if (lane == 0) { sh.red_a[wid] = s1; sh.red_b[wid] = s2; }
     __syncthreads();
+    // keys of the listed candidates (the staging buffers inside list_key are free now)
+    int m = 0;                                  // candidates found (all of them listed unless overflow)
+    if (listed) {
+        m = (int)min(sh.list_total, (uint32_t)kListCap);
+        if (sh.overflow == 0u)
+            for (int q = tid; q < m; q += kSelThreads) {
+                const uint32_t key = order_key(__ldg(grow + sh.list_pos[q]));
+                sh.list_key[q] = key;
+                kmax = max(kmax, key);
+            }
+    }
     if (tid == 0) {
         double ta = 0.0, tb = 0.0;
         for (int i = 0; i < kSelWarps; ++i) { ta += sh.red_a[i]; tb += sh.red_b[i]; }
@@ -504,19 +486,17 @@ __global__ void __launch_bounds__(kSelThreads, 2) gsa_select_kernel(const Select
         return;
     }
 
-    int m = 0;                                  // candidates found (all of them listed unless overflow)
-    for (int w = 0; w < kSelWarps; ++w) m += (int)sh.wl_cnt[w];
     if (!overflow && m >= k) {
-        // ---- exact threshold among the candidates (each warp walks its own list) ----------------
-        radix_rounds_lists(sh, kmin, kmax, (uint32_t)k, T, need_eq);
+        // ---- exact threshold among the candidates ------------------------------------------------
+        radix_rounds(sh, m, [&](int i) { return sh.list_key[i]; }, kmin, kmax, (uint32_t)k, T, need_eq);
 
-        // ---- emission in position order: thread c owns chunk c (a handful of entries, in order) ----
+        // ---- emission in position order: thread t owns table chunks t*cpt .. t*cpt + cpt - 1 -------
+        const int cpt = (ntab + kSelThreads - 1) / kSelThreads;             // 1 .. 4
+        const int c_lo = min(ntab, tid * cpt), c_hi = min(ntab, c_lo + cpt);
         uint32_t g = 0, q = 0;
-        uint32_t off = 0;
-        int cnt = 0;
-        if (tid < nchunks) {
-            off = (uint32_t)(tid & (kSelWarps - 1)) * kWarpCap + sh.ch_off[tid];
-            cnt = sh.ch_cnt[tid];
+        for (int c = c_lo; c < c_hi; ++c) {
+            const uint32_t off = sh.ch_off[c];
+            const int cnt = sh.ch_cnt[c];
             for (int j = 0; j < cnt; ++j) {
                 const uint32_t key = sh.list_key[off + j];
                 g += key > T;
@@ -526,15 +506,18 @@ __global__ void __launch_bounds__(kSelThreads, 2) gsa_select_kernel(const Select
         uint32_t total;
         const uint32_t before = block_excl_scan(sh, (q << 16) | g, 0, total);
         uint32_t g_before = before & 0xFFFFu, e_before = before >> 16;
-        const int c_base = tid * chunk_elems;
-        for (int j = 0; j < cnt; ++j) {
-            const uint32_t key = sh.list_key[off + j];
-            if (key > T) {
-                out_idx[g_before + min(e_before, need_eq)] = c_base + (int32_t)sh.list_rel[off + j];
-                ++g_before;
-            } else if (key == T) {
-                if (e_before < need_eq) out_idx[g_before + e_before] = c_base + (int32_t)sh.list_rel[off + j];
-                ++e_before;
+        for (int c = c_lo; c < c_hi; ++c) {
+            const uint32_t off = sh.ch_off[c];
+            const int cnt = sh.ch_cnt[c];
+            for (int j = 0; j < cnt; ++j) {
+                const uint32_t key = sh.list_key[off + j];
+                if (key > T) {
+                    out_idx[g_before + min(e_before, need_eq)] = (int32_t)sh.list_pos[off + j];
+                    ++g_before;
+                } else if (key == T) {
+                    if (e_before < need_eq) out_idx[g_before + e_before] = (int32_t)sh.list_pos[off + j];
+                    ++e_before;
+                }
             }
         }
     } else {

@@ -239,6 +239,30 @@ def test_topk_long_rows_that_defeat_the_sample():
         _select_and_compare(cfg, sc.cuda(), k_mode=k_mode, v_bar=v_bar)
 
 
+def test_topk_row_lengths_around_the_chunk_and_list_boundaries():
+    """Visible lengths n just below / at / above the short-row limit (8192) and multiples of the 512-score
+    chunk, and rows whose last chunk holds a single score."""
+    cfg = CONFIGS["l8k"].with_(name="edges", B=1, Lq=1540, Lk=9730, k_base=900, k_min=64, k_max=2048)
+    st = U.row_stride(cfg)
+    g = torch.Generator().manual_seed(8)
+    sc = (torch.rand((1, cfg.Lq, st), generator=g) ** 4).cuda()          # long right tail
+    # rows t = 0 .. 1539 see n = 8191 .. 9730 keys: 8191, 8192, 8193 and 8704 = 17 * 512, 9216, 9217, 9728
+    rows = np.array([0, 1, 2, 3, 511, 512, 513, 514, 1024, 1025, 1026, 1027, 1535, 1536, 1537, 1538, 1539])
+    for k_mode, v_bar in ((0, 0.07), (2, 1.0)):
+        _select_and_compare(cfg, sc, rows=rows, k_mode=k_mode, v_bar=v_bar)
+
+
+def test_topk_rows_longer_than_the_candidate_table():
+    """Rows of more than 2048 * 512 visible scores are not listed: they take the whole-row path."""
+    cfg = CONFIGS["l8k"].with_(name="verylong", B=1, Lq=2, Lk=1048576 + 777, k_base=1500, k_min=100, k_max=4096)
+    st = U.row_stride(cfg)
+    g = torch.Generator().manual_seed(9)
+    sc = (torch.randn((1, cfg.Lq, st), generator=g) * 0.05 + 1.0).cuda()
+    ws = torch.zeros(1024, dtype=torch.uint8, device="cuda")
+    for k_mode, v_bar in ((0, 0.0025), (2, 1.0)):
+        _select_and_compare(cfg, sc, k_mode=k_mode, v_bar=v_bar)
+
+
 # ------------------------------------------------------------------------------------------ stage 3
 def _oracle_idx(cfg, x, rows, **kw):
     p = U.oracle_params(cfg, **kw)
