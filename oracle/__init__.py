@@ -216,3 +216,36 @@ def out_project(X, Wt, rows_m: Sequence[int]) -> np.ndarray:
     lib().gsa_oracle_out_project_rows(ctypes.c_int(X.shape[1]), ctypes.c_int(Wt.shape[0]), _ptr(X), _ptr(Wt),
                                       _ptr(rows_m), ctypes.c_int(len(rows_m)), _ptr(u))
     return u
+
+
+def attn_bwd(p: OracleParams, Q, K, V, g1, g2, idx, keff, dout, rows_t, rows_b=None):
+    """Backward of Eq. 9-12 and Eq. 10 for the listed rows with given index sets: derivatives of
+    sum_r <dout[r], out[r]>.  dout: [n, n_h, d_h].  Returns dict(dQ, dg1: [n, n_h, d_h];
+    dK, dV, dg2: [B, Lk, n_kv, d_h] summed over the listed rows), all float64."""
+    rows_b, rows_t = _rows(p, rows_t, rows_b)
+    Q, K, V, g1, g2, dout = _f32(Q), _f32(K), _f32(V), _f32(g1), _f32(g2), _f32(dout)
+    idx, keff = _i32(idx), _i32(keff).reshape(-1)
+    n = len(rows_t)
+    assert idx.shape == (n, p.k_max) and keff.shape == (n,) and dout.shape == (n, p.n_h, p.d_h)
+    for r in range(n):
+        assert (idx[r, :keff[r]] >= 0).all() and (idx[r, :keff[r]] < p.Lk).all()
+    dQ = np.empty((n, p.n_h, p.d_h), dtype=np.float64)
+    dg1 = np.empty_like(dQ)
+    dK = np.empty((p.B, p.Lk, p.n_kv, p.d_h), dtype=np.float64)
+    dV = np.empty_like(dK)
+    dg2 = np.empty_like(dK)
+    c = p.c()
+    lib().gsa_oracle_attn_bwd_rows(ctypes.byref(c), _ptr(Q), _ptr(K), _ptr(V), _ptr(g1), _ptr(g2), _ptr(rows_b),
+                                   _ptr(rows_t), ctypes.c_int(n), _ptr(idx), _ptr(keff), _ptr(dout),
+                                   _ptr(dQ), _ptr(dg1), _ptr(dK), _ptr(dV), _ptr(dg2))
+    return dict(dQ=dQ, dg1=dg1, dK=dK, dV=dV, dg2=dg2)
+
+
+def vbar_update(v_bar: float, momentum: float, var) -> tuple:
+    """(new v_bar, batch-mean variance): EMA of the score variance across the batch (text below Eq. 8)."""
+    v = _f32(var).reshape(-1)
+    f = lib().gsa_oracle_vbar_update
+    f.restype = ctypes.c_double
+    m = ctypes.c_double(0.0)
+    new = f(ctypes.c_double(v_bar), ctypes.c_double(momentum), _ptr(v), ctypes.c_int64(v.size), ctypes.byref(m))
+    return float(new), float(m.value)

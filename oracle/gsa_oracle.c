@@ -33,6 +33,9 @@
  * with exact ties (ReLU variant: positive homogeneity, I(q) - I(-q) linear in q), reduction to
  * library softmax attention when S_t is everything
  * and gates are saturated, single-key and equal-logit closed forms, g1 = -40 -> 0.
+ * Training side (end of this file): the backward of Eq. 9-12 and Eq. 10 is pinned by central differences
+ * of the forward above, by library autograd on the forward written as masked dense attention, and by the
+ * single-key / shift-invariance closed forms; the running mean of the variance by a worked example.
  * Parity unpinned: nothing (every function above has at least one such pin); the
  * absolute values on random data have no printed reference in the paper.
  */
@@ -296,4 +299,108 @@ void gsa_oracle_forward_rows(const gsa_oracle_params *p, const float *Q, const f
                             out + (size_t)r * qrow);
         if (!scores_out) free(row);
     }
+}
+
+/* ---- training side of the path --------------------------------------------- */
+/* Backward of Eq. 9-12 and Eq. 10 for the listed rows with given index sets: the derivatives of
+ *   loss = sum over listed rows of <dout[r], out[r]>
+ * with respect to Q, K, V and the two gate logits.  The index sets are constants (top-k selection
+ * has no derivative; the indexer is trained by its own loss, Sec. 5.1).  Written from the chain rule
+ * on the forward definition, per head h of query row t with KV head g:
+ *   v'_j = V[s_j] * sigmoid(g2[s_j])                                   (Eq. 9)
+ *   z_j  = scale * q . k_j,   a = softmax_j(z),   o = sum_j a_j v'_j   (Eq. 11-12)
+ *   out  = o * sigmoid(g1)                                             (Eq. 10)
+ * so, with do = dout * sigmoid(g1):
+ *   dg1   = dout * o * sigmoid'(g1)
+ *   da_j  = do . v'_j,   dz_j = a_j (da_j - sum_i a_i da_i)
+ *   dq    = scale * sum_j dz_j k_j,      dK[s_j] += scale * dz_j q
+ *   dv'_j = a_j do  ->  dV[s_j] += dv'_j * sigmoid(g2[s_j]),  dg2[s_j] += dv'_j * V[s_j] * sigmoid'(g2[s_j])
+ * dQ, dg1: [n_rows, n_h, d_h]; dK, dV, dg2: [B, Lk, n_kv, d_h], zeroed here, summed over the listed rows.
+ * Threads split the KV heads, so no two threads add into the same element. */
+void gsa_oracle_attn_bwd_rows(const gsa_oracle_params *p, const float *Q, const float *K,
+                              const float *V, const float *g1, const float *g2,
+                              const int32_t *rows_b, const int32_t *rows_t, int n_rows,
+                              const int32_t *idx, const int32_t *keff, const float *dout,
+                              double *dQ, double *dg1, double *dK, double *dV, double *dg2)
+{
+    const int d = p->d_h, grp = p->n_h / p->n_kv;
+    const double scale = p->sm_scale > 0.0 ? p->sm_scale : 1.0 / sqrt((double)d);
+    const size_t qrow = (size_t)p->n_h * d, kvb = (size_t)p->Lk * p->n_kv * d;
+    memset(dK, 0, sizeof(double) * kvb * (size_t)p->B);
+    memset(dV, 0, sizeof(double) * kvb * (size_t)p->B);
+    memset(dg2, 0, sizeof(double) * kvb * (size_t)p->B);
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int g = 0; g < p->n_kv; ++g) {
+        double *a = (double *)malloc(sizeof(double) * (size_t)(p->k_max > 0 ? p->k_max : 1));
+        double *da = (double *)malloc(sizeof(double) * (size_t)(p->k_max > 0 ? p->k_max : 1));
+        double *dov = (double *)malloc(sizeof(double) * (size_t)d);
+        for (int r = 0; r < n_rows; ++r) {
+            const int b = rows_b[r], t = rows_t[r], ke = keff[r];
+            const int32_t *S = idx + (size_t)r * p->k_max;
+            for (int h = g * grp; h < (g + 1) * grp; ++h) {
+                const float *q = Q + ((size_t)b * p->Lq + t) * qrow + (size_t)h * d;
+                const float *gl = g1 + ((size_t)b * p->Lq + t) * qrow + (size_t)h * d;
+                const float *dy = dout + (size_t)r * qrow + (size_t)h * d;
+                double zmax = -INFINITY, den = 0.0;
+                for (int j = 0; j < ke; ++j) {
+                    const float *ks = K + b * kvb + ((size_t)S[j] * p->n_kv + g) * d;
+                    double dot = 0.0;
+                    for (int c = 0; c < d; ++c) dot += (double)q[c] * (double)ks[c];
+                    a[j] = dot * scale;
+                    if (a[j] > zmax) zmax = a[j];
+                }
+                for (int j = 0; j < ke; ++j) { a[j] = exp(a[j] - zmax); den += a[j]; }
+                for (int j = 0; j < ke; ++j) a[j] /= den;
+                /* o, do, dg1 */
+                for (int c = 0; c < d; ++c) {
+                    double o = 0.0;
+                    for (int j = 0; j < ke; ++j) {
+                        const size_t at = b * kvb + ((size_t)S[j] * p->n_kv + g) * d + c;
+                        o += a[j] * ((double)V[at] * sigmoid_d((double)g2[at]));
+                    }
+                    const double s1 = sigmoid_d((double)gl[c]);
+                    dov[c] = (double)dy[c] * s1;
+                    dg1[(size_t)r * qrow + (size_t)h * d + c] = (double)dy[c] * o * s1 * (1.0 - s1);
+                }
+                /* da_j and the softmax backward */
+                double dsum = 0.0;
+                for (int j = 0; j < ke; ++j) {
+                    double acc = 0.0;
+                    for (int c = 0; c < d; ++c) {
+                        const size_t at = b * kvb + ((size_t)S[j] * p->n_kv + g) * d + c;
+                        acc += dov[c] * ((double)V[at] * sigmoid_d((double)g2[at]));
+                    }
+                    da[j] = acc;
+                    dsum += a[j] * acc;
+                }
+                for (int c = 0; c < d; ++c) dQ[(size_t)r * qrow + (size_t)h * d + c] = 0.0;
+                for (int j = 0; j < ke; ++j) {
+                    const double dz = a[j] * (da[j] - dsum);
+                    const size_t row = b * kvb + ((size_t)S[j] * p->n_kv + g) * d;
+                    for (int c = 0; c < d; ++c) {
+                        dQ[(size_t)r * qrow + (size_t)h * d + c] += scale * dz * (double)K[row + c];
+                        dK[row + c] += scale * dz * (double)q[c];
+                        const double s2 = sigmoid_d((double)g2[row + c]);
+                        const double dvg = a[j] * dov[c];
+                        dV[row + c] += dvg * s2;
+                        dg2[row + c] += dvg * (double)V[row + c] * s2 * (1.0 - s2);
+                    }
+                }
+            }
+        }
+        free(a); free(da); free(dov);
+    }
+}
+
+/* Running mean of the score variance (text below Eq. 8: the normaliser of the budget is an exponential
+ * moving average of the score variance across the batch).  The paper gives neither the momentum nor the
+ * start value: both are the caller's.  mean_var = mean of the n row variances; returns
+ * momentum * v_bar + (1 - momentum) * mean_var. */
+double gsa_oracle_vbar_update(double v_bar, double momentum, const float *var, int64_t n, double *mean_var)
+{
+    double s = 0.0;
+    for (int64_t i = 0; i < n; ++i) s += (double)var[i];
+    const double m = n > 0 ? s / (double)n : 0.0;
+    if (mean_var) *mean_var = m;
+    return momentum * v_bar + (1.0 - momentum) * m;
 }

@@ -427,6 +427,118 @@ def test_output_projection_one_hot_and_library_matmul():
                                rtol=1e-13, atol=1e-13)
 
 
+# ------------------------------------------------------------------ backward of Eq. 9-12, 10
+def _rand_index_sets(p, seed):
+    """ascending random subsets of the visible keys, sizes 1 .. k_max"""
+    g = np.random.default_rng(seed)
+    rows_b, rows_t, idx, keff = [], [], [], []
+    for b in range(p.B):
+        for t in range(p.Lq):
+            n = p.visible(t)
+            k = int(g.integers(1, min(n, p.k_max) + 1))
+            row = np.full(p.k_max, -1, np.int32)
+            row[:k] = np.sort(g.choice(n, size=k, replace=False))
+            rows_b.append(b); rows_t.append(t); idx.append(row); keff.append(k)
+    return np.array(rows_b, np.int32), np.array(rows_t, np.int32), np.stack(idx), np.array(keff, np.int32)
+
+
+def _bwd_problem(seed=0, **kw):
+    p = small_params(**{**dict(B=2, Lq=5, Lk=9, n_h=4, n_kv=2, d_h=8, k_max=5), **kw})
+    x = _rand_attn_inputs(p, seed)
+    x = {k: (v.float() * 0.5).to(torch.bfloat16) for k, v in x.items()}
+    rows_b, rows_t, idx, keff = _rand_index_sets(p, seed + 1)
+    g = torch.Generator().manual_seed(seed + 2)
+    dout = torch.randn(len(rows_t), p.n_h, p.d_h, generator=g).to(torch.bfloat16)
+    return p, x, rows_b, rows_t, idx, keff, dout
+
+
+def test_attn_backward_matches_central_differences_of_the_forward_oracle():
+    """d/dx of L = sum <dout, out(x)> by central differences of the (pinned) forward, for sampled elements
+    of every input tensor.  Steps of 2^-8 on bf16 values are exact in fp32, the forward runs in fp64."""
+    p, x, rows_b, rows_t, idx, keff, dout = _bwd_problem(0)
+    got = oracle.attn_bwd(p, **x, idx=idx, keff=keff, dout=dout, rows_t=rows_t, rows_b=rows_b)
+    dq_full = np.zeros((p.B, p.Lq, p.n_h, p.d_h))
+    dg1_full = np.zeros_like(dq_full)
+    dq_full[rows_b, rows_t] = got["dQ"]
+    dg1_full[rows_b, rows_t] = got["dg1"]
+    grads = dict(Q=dq_full, g1=dg1_full, K=got["dK"], V=got["dV"], g2=got["dg2"])
+    dy = dout.double().numpy()
+
+    def loss(xx):
+        out = oracle.attn(p, **xx, idx=idx, keff=keff, rows_t=rows_t, rows_b=rows_b)
+        return float((out * dy).sum())
+
+    eps = 2.0 ** -8
+    rng = np.random.default_rng(5)
+    for name, gr in grads.items():
+        base = x[name].float().numpy()
+        flat = rng.choice(base.size, size=40, replace=False)
+        scale = np.abs(gr).max()
+        assert scale > 1e-3, name                      # the gradient is really there
+        for f in flat:
+            at = np.unravel_index(f, base.shape)
+            hi, lo = base.copy(), base.copy()
+            hi[at] += eps
+            lo[at] -= eps
+            fd = (loss({**x, name: hi}) - loss({**x, name: lo})) / (2 * eps)
+            assert abs(fd - gr[at]) <= 2e-4 * scale + 1e-9, (name, at, fd, gr[at])
+
+
+def test_attn_backward_matches_library_autograd_on_masked_dense_attention():
+    """The forward written with torch's library softmax / matmul in fp64 (a mask of -inf outside S_t) and
+    differentiated by autograd."""
+    p, x, rows_b, rows_t, idx, keff, dout = _bwd_problem(3, B=1, Lq=6, Lk=8)
+    got = oracle.attn_bwd(p, **x, idx=idx, keff=keff, dout=dout, rows_t=rows_t, rows_b=rows_b)
+    t64 = {k: v[0].double().clone().requires_grad_(True) for k, v in x.items()}
+    grp = p.n_h // p.n_kv
+    mask = torch.full((p.Lq, p.Lk), -math.inf, dtype=torch.float64)
+    for r, t in enumerate(rows_t):
+        mask[t, idx[r, : keff[r]]] = 0.0
+    Vg = t64["V"] * torch.sigmoid(t64["g2"])                                  # Eq. 9
+    outs = []
+    for h in range(p.n_h):
+        g = h // grp
+        z = (t64["Q"][:, h] @ t64["K"][:, g].T) / math.sqrt(p.d_h) + mask      # Eq. 11
+        outs.append(torch.softmax(z, dim=-1) @ Vg[:, g])                       # Eq. 12
+    out = torch.stack(outs, dim=1) * torch.sigmoid(t64["g1"])                  # Eq. 10
+    (out * dout.double().reshape(p.Lq, p.n_h, p.d_h)).sum().backward()
+    np.testing.assert_allclose(got["dQ"], t64["Q"].grad.numpy(), rtol=1e-9, atol=1e-12)
+    np.testing.assert_allclose(got["dg1"], t64["g1"].grad.numpy(), rtol=1e-9, atol=1e-12)
+    np.testing.assert_allclose(got["dK"][0], t64["K"].grad.numpy(), rtol=1e-9, atol=1e-12)
+    np.testing.assert_allclose(got["dV"][0], t64["V"].grad.numpy(), rtol=1e-9, atol=1e-12)
+    np.testing.assert_allclose(got["dg2"][0], t64["g2"].grad.numpy(), rtol=1e-9, atol=1e-12)
+
+
+def test_attn_backward_single_key_and_shift_invariance():
+    """One selected key: the softmax is the constant 1, so dQ = dK = 0 exactly and dV[s] = dout * sigmoid(g1) *
+    sigmoid(g2[s]).  Any row: softmax ignores a common shift of its logits, so the logit derivatives of one
+    (row, head) sum to zero, i.e. sum_s dK[s] = 0 when a single row with one head per KV head is listed."""
+    p = small_params(B=1, Lq=4, Lk=4, n_h=2, n_kv=2, d_h=8, k_max=3)
+    x = _rand_attn_inputs(p, 7)
+    dout = torch.randn(1, p.n_h, p.d_h, generator=torch.Generator().manual_seed(8)).to(torch.bfloat16)
+    idx = np.array([[2, -1, -1]], np.int32)
+    got = oracle.attn_bwd(p, **x, idx=idx, keff=[1], dout=dout, rows_t=[3])
+    assert (got["dQ"] == 0).all() and (got["dK"] == 0).all()
+    s1 = torch.sigmoid(x["g1"][0, 3].double())
+    s2 = torch.sigmoid(x["g2"][0, 2].double())
+    want = dout[0].double() * s1 * s2                   # heads map one-to-one onto KV heads here
+    np.testing.assert_allclose(got["dV"][0, 2], want.numpy(), rtol=1e-13)
+    assert (got["dV"][0, [0, 1, 3]] == 0).all() and (got["dg2"][0, [0, 1, 3]] == 0).all()
+    idx = np.array([[0, 1, 3]], np.int32)
+    got = oracle.attn_bwd(p, **x, idx=idx, keff=[3], dout=dout, rows_t=[3])
+    assert np.abs(got["dK"][0]).max() > 1e-3
+    assert np.abs(got["dK"][0].sum(axis=0)).max() <= 1e-14
+    assert (got["dK"][0, 2] == 0).all()                 # a key outside S_t gets nothing
+
+
+def test_vbar_update_closed_form():
+    new, mean = oracle.vbar_update(0.5, 0.75, np.array([1.0, 2.0, 3.0, 6.0], np.float32))
+    assert mean == 3.0 and new == 0.75 * 0.5 + 0.25 * 3.0
+    new, mean = oracle.vbar_update(0.5, 0.0, np.array([0.25], np.float32))
+    assert (new, mean) == (0.25, 0.25)
+    assert oracle.vbar_update(0.5, 1.0, np.array([9.0, 1.0], np.float32))[0] == 0.5
+
+
 def test_paper_printed_cost_model():
     """Appendix A prints d^I H^I/(d n_h) ~ 0.002 and a 12.8x speed-up for its parameters."""
     vals = {}
