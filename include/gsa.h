@@ -122,6 +122,43 @@ int gsa_output_projection(const gsa_params_t *p, int32_t d_model, const void *at
                           void *u, void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * Backward of sparse gated attention: Eq. 9, 11, 12 and 10 differentiated for rows [q_begin, q_end)
+ * with the index sets held fixed (top-k selection has no derivative; Sec. 5.1 trains the indexer with
+ * its own loss).  With out = o * sigmoid(g1), o = sum_j a_j v'_j, a = softmax_j(sm_scale * q.k_j) over
+ * j in S_t and v' = V * sigmoid(g2), and dout the derivative of the loss with respect to `out`:
+ *     dg1 = dout * o * sigmoid'(g1),        do = dout * sigmoid(g1),
+ *     dz_j = a_j (do.v'_j - sum_i a_i do.v'_i),   dQ = sm_scale * sum_j dz_j k_j,
+ *     dK[s] = sm_scale * sum over (t, h, j: s_j = s) of dz_j q,    dv'[s] = sum of a_j do,
+ *     dV = dv' * sigmoid(g2),   dg2 = dv' * V * sigmoid'(g2).
+ *   Q, K, V, g1_logits, g2_logits, idx, kt   as given to gsa_sparse_gated_attn_fwd (g2_logits required)
+ *   out    [B, Lq, n_h, d_h] bf16: what the forward call wrote (rows of the range are read)
+ *   dout   [B, Lq, n_h, d_h] bf16 (rows of the range are read)
+ *   dQ, dg1  [B, Lq, n_h, d_h] bf16: rows of the range are written, other rows are left alone
+ *   dK, dV, dg2  [B, Lk, n_kv, d_h] bf16: every element is written; sums over the rows of the range,
+ *          accumulated in fp32 (in an order that depends on scheduling) and rounded once
+ *   ws     workspace of gsa_attn_bwd_workspace_bytes(p) bytes: status word, V', fp32 dK and dV'
+ * Returns GSA_ERR_WORKSPACE if ws is too small; nothing is launched on an argument error.
+ */
+int gsa_attn_bwd_workspace_bytes(const gsa_params_t *p, size_t *bytes);
+int gsa_sparse_gated_attn_bwd(const gsa_params_t *p, const void *Q, const void *K, const void *V,
+                              const void *g1_logits, const void *g2_logits, const int32_t *idx,
+                              const int32_t *kt, const void *out, const void *dout, void *dQ, void *dK,
+                              void *dV, void *dg1, void *dg2, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Running mean of the score variance: the normaliser v_bar of Eq. 8 is an exponential moving average of
+ * the score variance across the batch.  The paper gives neither momentum nor start value: both are the
+ * caller's.
+ *     mean_var = mean of var[0 .. n),      v_bar <- momentum * v_bar + (1 - momentum) * mean_var
+ *   var       n fp32 row variances on the device (the `var` output of gsa_forward / gsa_adaptive_topk)
+ *   v_bar     one fp32 on the device, read and written; copy it into gsa_params_t.v_bar for the next step
+ *   mean_var  one fp32 on the device or NULL
+ *   momentum  in [0, 1]
+ * The sum is taken in fp64 in a fixed order: the result does not depend on scheduling.
+ */
+int gsa_vbar_update(const float *var, int64_t n, float momentum, float *v_bar, float *mean_var, void *stream);
+
+/*
  * Adaptive sparsity controller, Eq. 8 then Eq. 4, one row at a time:
  *     Var_t = population variance of the n_t visible scores (accumulated in fp64),
  *     k_t   = clamp(floor(k_base * Var_t / v_bar), k_min, k_max)   (k_mode 0),

@@ -22,6 +22,7 @@ EXPORTS = (
     "gsa_launch_count", "gsa_debug_set_indexer_path", "gsa_profile_set_events", "gsa_status_string",
     "gsa_sparse_gated_attn_fwd_static", "gsa_attn_workspace_bytes", "gsa_debug_set_attn_range_keys",
     "gsa_select_fallback_rows", "gsa_project", "gsa_project_columns", "gsa_output_projection",
+    "gsa_attn_bwd_workspace_bytes", "gsa_sparse_gated_attn_bwd", "gsa_vbar_update",
 )
 
 STATIC_SCRATCH_BYTES = 32 << 20     # GSA_STATIC_SCRATCH_BYTES of include/gsa.h
@@ -148,6 +149,27 @@ def gsa_sparse_gated_attn_fwd(p, Q, K, V, g1, g2, idx, kt, out, ws=None, stream=
                                            _dp(g2, BF16), _dp(idx, I32), _dp(kt, I32), _dp(out, BF16), _dp(ws),
                                            ctypes.c_size_t(0 if ws is None else ws.numel() * ws.element_size()),
                                            _stream(stream)), "gsa_sparse_gated_attn_fwd")
+
+
+def gsa_attn_bwd_workspace_bytes(p) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().gsa_attn_bwd_workspace_bytes(ctypes.byref(p), ctypes.byref(n)), "gsa_attn_bwd_workspace_bytes")
+    return int(n.value)
+
+
+def gsa_sparse_gated_attn_bwd(p, Q, K, V, g1, g2, idx, kt, out, dout, dQ, dK, dV, dg1, dg2, ws, stream=None) -> None:
+    _check(lib().gsa_sparse_gated_attn_bwd(ctypes.byref(p), _dp(Q, BF16), _dp(K, BF16), _dp(V, BF16), _dp(g1, BF16),
+                                           _dp(g2, BF16), _dp(idx, I32), _dp(kt, I32), _dp(out, BF16),
+                                           _dp(dout, BF16), _dp(dQ, BF16), _dp(dK, BF16), _dp(dV, BF16),
+                                           _dp(dg1, BF16), _dp(dg2, BF16), _dp(ws),
+                                           ctypes.c_size_t(ws.numel() * ws.element_size()), _stream(stream)),
+           "gsa_sparse_gated_attn_bwd")
+
+
+def gsa_vbar_update(var, momentum: float, v_bar, mean_var=None, stream=None) -> None:
+    """v_bar (one fp32 on the device) <- momentum * v_bar + (1 - momentum) * mean(var)."""
+    _check(lib().gsa_vbar_update(_dp(var, F32), ctypes.c_int64(var.numel()), ctypes.c_float(momentum),
+                                 _dp(v_bar, F32), _dp(mean_var, F32), _stream(stream)), "gsa_vbar_update")
 
 
 def gsa_sparse_gated_attn_fwd_static(p, Q, K, V, g1, g2, idx, kt, out, stream=None) -> None:

@@ -209,6 +209,58 @@ static size_t attn_ws_bytes(const gsa_params_t& p, bool with_prepass) {
     return n;
 }
 
+// workspace of the backward call: [status][V' bf16][dK fp32][dV' fp32]
+static size_t attn_bwd_ws_bytes(const gsa_params_t& p) {
+    const size_t n = (size_t)p.B * p.Lk * p.n_kv * p.d_h;
+    return kStatusBytes + align_up(n * 2, 256) + 2 * align_up(n * 4, 256);
+}
+
+int gsa_attn_bwd_workspace_bytes(const gsa_params_t* p, size_t* bytes) {
+    int rc = check_params(p);
+    if (rc) return rc;
+    if (!bytes) return GSA_ERR_INVALID_ARG;
+    *bytes = attn_bwd_ws_bytes(*p);
+    return GSA_OK;
+}
+
+int gsa_sparse_gated_attn_bwd(const gsa_params_t* p, const void* Q, const void* K, const void* V,
+                              const void* g1_logits, const void* g2_logits, const int32_t* idx,
+                              const int32_t* kt, const void* out, const void* dout, void* dQ, void* dK,
+                              void* dV, void* dg1, void* dg2, void* ws, size_t ws_bytes, void* stream) {
+    int rc = check_params(p);
+    if (rc) return rc;
+    RowRange rr;
+    if ((rc = row_range(p, &rr))) return rc;
+    if (!attn_bwd_supported(*p)) return GSA_ERR_UNSUPPORTED_SHAPE;
+    const void* ptrs[] = {Q, K, V, g1_logits, g2_logits, idx, out, dout, dQ, dK, dV, dg1, dg2};
+    for (const void* q : ptrs) if (!q || !aligned16(q)) return GSA_ERR_INVALID_ARG;
+    if (!kt) return GSA_ERR_INVALID_ARG;
+    if (!ws || !aligned16(ws) || ws_bytes < attn_bwd_ws_bytes(*p)) return GSA_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t n = (size_t)p->B * p->Lk * p->n_kv * p->d_h;
+    char* wsb = (char*)ws;
+    bf16* Vg = (bf16*)(wsb + kStatusBytes);
+    float* dK32 = (float*)(wsb + kStatusBytes + align_up(n * 2, 256));
+    float* dV32 = (float*)((char*)dK32 + align_up(n * 4, 256));
+    cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(dK32, 0, 2 * align_up(n * 4, 256), st);
+    if (e == cudaSuccess) e = launch_value_gate((const bf16*)V, (const bf16*)g2_logits, Vg, (int64_t)n, st);
+    IdxLayout il{0, rr.q_begin, rr.R};
+    if (e == cudaSuccess)
+        e = launch_sparse_attn_bwd(*p, rr, (const bf16*)Q, (const bf16*)K, Vg, (const bf16*)g1_logits,
+                                   (const bf16*)out, (const bf16*)dout, idx, kt, il, (bf16*)dQ, (bf16*)dg1,
+                                   dK32, dV32, st);
+    if (e == cudaSuccess)
+        e = launch_attn_bwd_finish(dK32, dV32, (const bf16*)V, (const bf16*)g2_logits, (bf16*)dK, (bf16*)dV,
+                                   (bf16*)dg2, (int64_t)n, st);
+    return cuda_rc(e);
+}
+
+int gsa_vbar_update(const float* var, int64_t n, float momentum, float* v_bar, float* mean_var, void* stream) {
+    if (!var || !v_bar || n < 1 || !(momentum >= 0.f && momentum <= 1.f)) return GSA_ERR_INVALID_ARG;
+    return cuda_rc(launch_vbar_update(var, n, momentum, v_bar, mean_var, (cudaStream_t)stream));
+}
+
 int gsa_attn_workspace_bytes(const gsa_params_t* p, int32_t with_value_gate_prepass, size_t* bytes) {
     int rc = check_params(p);
     if (rc) return rc;

@@ -1,0 +1,381 @@
+// Backward of sparse gated attention (Eq. 9-12 and Eq. 10 differentiated; the index sets S_t are
+// constants: top-k selection has no derivative and the indexer is trained by its own loss, Sec. 5.1).
+//
+// With out = o * sigmoid(g1), o = sum_j a_j v'_j, a = softmax_j(scale * q.k_j), v' = V * sigmoid(g2):
+//   do    = dout * sigmoid(g1)
+//   dg1   = dout * o * sigmoid'(g1)          = dout * out * (1 - sigmoid(g1))       (o * sigmoid = out)
+//   delta = sum_j a_j (do . v'_j) = do . o   = sum_d dout_d * out_d
+//   dz_j  = a_j (do . v'_j - delta),   dq = scale * sum_j dz_j k_j,   dK[s_j] += scale * dz_j q
+//   dv'_j = a_j do  ->  dV = dv' * sigmoid(g2),   dg2 = dv' * V * sigmoid'(g2)      (post-pass)
+// so the saved forward output is all the state the backward needs; the softmax statistics are
+// recomputed from K in a first sweep over S_t.
+//
+// One warp per (query row, KV head).  Per 16 selected keys the K and V' rows are copied (16-byte
+// asynchronous copies) into a private shared-memory tile and every product runs on the tensor cores
+// (bf16 mma.sync, fp32 accumulation) with the keys as M:
+//   S^T[key, head]  = K  . Q^T       dP^T[key, head] = V' . do^T             (A: tile via ldmatrix)
+//   dQ^T[d, head]  += K^T . dS^T                                             (A: tile via ldmatrix.trans)
+//   dK[key, d]      = dS^T . Q       dV'[key, d]     = P^T . do              (m16n8k8: heads are K)
+// dK and dV' are sums over every query that selected the key: they are accumulated in fp32 with
+// vector reductions (red.global.add.v2.f32) into workspace arrays, and a streaming post-pass applies
+// the value gate's derivative and rounds to bf16.  The kernel is bound by those reductions:
+// 2 * n_kv * d_h fp32 additions in L2 per selected (query, key) pair.
+#include "gsa_common.cuh"
+
+namespace gsa {
+
+namespace {
+
+constexpr int kBwdWarps = 4;
+constexpr float kLog2e = 1.4426950408889634f;
+
+struct BwdArgs {
+    const __nv_bfloat16* Q;
+    const __nv_bfloat16* K;
+    const __nv_bfloat16* Vg;      // V' = bf16(V * sigmoid(g2)), as the forward uses it
+    const __nv_bfloat16* g1;
+    const __nv_bfloat16* out;     // the forward's output
+    const __nv_bfloat16* dout;
+    const int32_t* idx;
+    const int32_t* kt;
+    __nv_bfloat16* dQ;
+    __nv_bfloat16* dg1;
+    float* dK32;
+    float* dV32;
+    RowRange rr;
+    IdxLayout il;
+    int32_t Lq, Lk, n_h, n_kv, k_max;
+    float scale;
+};
+
+__device__ __forceinline__ uint32_t movmatrix_t(uint32_t a) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+// D(16x8, fp32) = A(16x8, bf16, row) * B(8x8, bf16, col)
+__device__ __forceinline__ void mma_bf16_1688(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%7,%8,%9,%10};\n"
+        : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+        : "r"(a0), "r"(a1), "r"(b0), "f"(0.f), "f"(0.f), "f"(0.f), "f"(0.f));
+}
+__device__ __forceinline__ void red_add_v2(float* addr, float x, float y) {
+    asm volatile("red.global.add.v2.f32 [%0], {%1, %2};" ::"l"(addr), "f"(x), "f"(y) : "memory");
+}
+
+template <int DH, int G>
+__global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(const BwdArgs a) {
+    constexpr int ROW = (DH + 8) * 2;                  // bytes of a padded tile row (odd multiple of 16)
+    constexpr int KTILE = 16 * ROW, QTILE = 8 * ROW;
+    constexpr int WARP_SMEM = 2 * KTILE + 2 * QTILE + 64;
+    constexpr int KS = DH / 16;                        // k-steps of the S^T / dP^T products, m-tiles of dQ^T
+    constexpr int EPL = DH / 32;                       // elements of a head row per lane (row staging)
+    constexpr int CPR = DH / 8;                        // 16-byte chunks per tile row
+    extern __shared__ __align__(16) unsigned char bwd_smem[];
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int gid = lane >> 2, tig = lane & 3;
+    const int64_t item = (int64_t)blockIdx.x * kBwdWarps + warp;
+    const int64_t n_items = (int64_t)a.rr.rows() * a.n_kv;
+    if (item >= n_items) return;                       // (no block-wide barrier below)
+    // long rows first: late rows have the most keys
+    const int lr = a.rr.rows() - 1 - (int)(item / a.n_kv);
+    const int g = (int)(item % a.n_kv);
+    const int b = a.rr.b0 + lr / a.rr.R;
+    const int t = a.rr.q_begin + lr % a.rr.R;
+    const int64_t qrow = (int64_t)b * a.Lq + t;
+    const int64_t irow = a.il.row(b, t);
+    const int ke = a.kt[irow];
+    const int32_t* __restrict__ S = a.idx + irow * a.k_max;
+
+    unsigned char* const ws = bwd_smem + warp * WARP_SMEM;
+    unsigned char* const k_tile = ws;
+    unsigned char* const v_tile = ws + KTILE;
+    unsigned char* const q_tile = ws + 2 * KTILE;       // rows = the group's heads (rows >= G are zero)
+    unsigned char* const d_tile = ws + 2 * KTILE + QTILE;
+    float* const s_delta = reinterpret_cast<float*>(ws + 2 * KTILE + 2 * QTILE);   // [8]
+    const uint32_t k_s32 = (uint32_t)__cvta_generic_to_shared(k_tile);
+    const uint32_t v_s32 = (uint32_t)__cvta_generic_to_shared(v_tile);
+    const uint32_t q_s32 = (uint32_t)__cvta_generic_to_shared(q_tile);
+    const uint32_t d_s32 = (uint32_t)__cvta_generic_to_shared(d_tile);
+
+    // ---- per row: do = dout * sigmoid(g1), dg1, delta; Q and do staged as tiles -------------------
+#pragma unroll
+    for (int hl = 0; hl < 8; ++hl) {
+        __nv_bfloat16* qd = reinterpret_cast<__nv_bfloat16*>(q_tile + hl * ROW) + lane * EPL;
+        __nv_bfloat16* dd = reinterpret_cast<__nv_bfloat16*>(d_tile + hl * ROW) + lane * EPL;
+        float part = 0.f;
+        if (hl < G) {
+            const int64_t at = (qrow * a.n_h + (g * G + hl)) * DH + lane * EPL;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) {
+                const float dy = __bfloat162float(a.dout[at + e]);
+                const float y = __bfloat162float(a.out[at + e]);
+                const float sg = 1.0f / (1.0f + __expf(-__bfloat162float(a.g1[at + e])));
+                qd[e] = a.Q[at + e];
+                dd[e] = __float2bfloat16(dy * sg);
+                a.dg1[at + e] = __float2bfloat16(dy * y * (1.0f - sg));
+                part = fmaf(dy, y, part);
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) { qd[e] = __float2bfloat16(0.f); dd[e] = __float2bfloat16(0.f); }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
+        if (lane == 0) s_delta[hl] = part;
+    }
+    __syncwarp();
+    const float delta[2] = {s_delta[2 * tig], s_delta[2 * tig + 1]};
+
+    // B operands of S^T = K Q^T and dP^T = V' do^T: (k = d, n = head), kept for the whole row
+    uint32_t qb[2 * KS], dob[2 * KS];
+#pragma unroll
+    for (int k2 = 0; k2 < KS / 2; ++k2) {
+        const uint32_t off = (lane & 7) * ROW + (lane >> 3) * 16 + k2 * 64;
+        ldmatrix_x4(qb[4 * k2], qb[4 * k2 + 1], qb[4 * k2 + 2], qb[4 * k2 + 3], q_s32 + off);
+        ldmatrix_x4(dob[4 * k2], dob[4 * k2 + 1], dob[4 * k2 + 2], dob[4 * k2 + 3], d_s32 + off);
+    }
+
+    const float c2 = a.scale * kLog2e;
+    const size_t kv_row = (size_t)a.n_kv * DH;           // elements between consecutive keys
+    const __nv_bfloat16* const kbase = a.K + ((size_t)b * a.Lk * a.n_kv + g) * DH;
+    const __nv_bfloat16* const vbase = a.Vg + ((size_t)b * a.Lk * a.n_kv + g) * DH;
+
+    // copies the rows of 16 selected keys (positions held by lanes 0..15 of pos16) into a tile
+    auto fetch_tile = [&](const __nv_bfloat16* base, uint32_t tile_s32, int32_t pos16) {
+#pragma unroll
+        for (int i = 0; i < 16 * CPR / 32; ++i) {
+            const int chunk = i * 32 + lane;
+            const int r = chunk / CPR, c = chunk % CPR;
+            const int32_t p = __shfl_sync(0xFFFFFFFFu, pos16, r);
+            cp_async16(tile_s32 + r * ROW + c * 16, base + (size_t)p * kv_row + c * 8);
+        }
+    };
+    // S^T (or dP^T) of the staged tile: rows gid, gid + 8 = keys, columns 2 tig, 2 tig + 1 = heads
+    auto tile_times = [&](uint32_t tile_s32, const uint32_t (&bf)[2 * KS], float (&acc)[4]) {
+        acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
+        const uint32_t addr = tile_s32 + (lane & 15) * ROW + (lane >> 4) * 16;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            uint32_t a0, a1, a2, a3;
+            ldmatrix_x4(a0, a1, a2, a3, addr + ks * 32);
+            mma_bf16_16816(acc, a0, a1, a2, a3, bf[2 * ks], bf[2 * ks + 1]);
+        }
+    };
+
+    // ---- sweep 1: softmax statistics per head (log2 domain) ----------------------------------------
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+    for (int j0 = 0; j0 < ke; j0 += 16) {
+        const int32_t pos16 = S[min(j0 + (lane & 15), ke - 1)];
+        fetch_tile(kbase, k_s32, pos16);
+        cp_async_commit();
+        cp_async_wait<0>();
+        __syncwarp();
+        float s[4];
+        tile_times(k_s32, qb, s);
+        const bool v0 = j0 + gid < ke, v1 = j0 + gid + 8 < ke;
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const float x0 = v0 ? s[e] * c2 : -INFINITY, x1 = v1 ? s[2 + e] * c2 : -INFINITY;
+            const float m_new = fmaxf(m_run[e], fmaxf(x0, x1));
+            if (m_new > -INFINITY) {
+                l_run[e] = l_run[e] * ex2_approx(m_run[e] - m_new) + ex2_approx(x0 - m_new) + ex2_approx(x1 - m_new);
+                m_run[e] = m_new;
+            }
+        }
+        __syncwarp();
+    }
+    float lse2[2];
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+#pragma unroll
+        for (int o = 4; o < 32; o <<= 1) {               // merge the eight lanes that share the column
+            const float m_o = __shfl_xor_sync(0xFFFFFFFFu, m_run[e], o);
+            const float l_o = __shfl_xor_sync(0xFFFFFFFFu, l_run[e], o);
+            const float m_new = fmaxf(m_run[e], m_o);
+            if (m_new > -INFINITY)
+                l_run[e] = l_run[e] * ex2_approx(m_run[e] - m_new) + l_o * ex2_approx(m_o - m_new);
+            m_run[e] = m_new;
+        }
+        lse2[e] = m_run[e] + log2f(l_run[e]);
+    }
+
+    // ---- sweep 2: gradients ---------------------------------------------------------------------------
+    float dq[KS][4];
+#pragma unroll
+    for (int mt = 0; mt < KS; ++mt) dq[mt][0] = dq[mt][1] = dq[mt][2] = dq[mt][3] = 0.f;
+    for (int j0 = 0; j0 < ke; j0 += 16) {
+        const int32_t pos16 = S[min(j0 + (lane & 15), ke - 1)];
+        fetch_tile(kbase, k_s32, pos16);
+        fetch_tile(vbase, v_s32, pos16);
+        cp_async_commit();
+        cp_async_wait<0>();
+        __syncwarp();
+        float s[4], dp[4], p[4], ds[4];
+        tile_times(k_s32, qb, s);
+        tile_times(v_s32, dob, dp);
+        const bool v0 = j0 + gid < ke, v1 = j0 + gid + 8 < ke;
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            p[e] = v0 ? ex2_approx(s[e] * c2 - lse2[e]) : 0.f;
+            p[2 + e] = v1 ? ex2_approx(s[2 + e] * c2 - lse2[e]) : 0.f;
+            ds[e] = p[e] * (dp[e] - delta[e]);
+            ds[2 + e] = p[2 + e] * (dp[2 + e] - delta[e]);
+        }
+        const uint32_t ds_lo = pack_bf16(ds[0], ds[1]), ds_hi = pack_bf16(ds[2], ds[3]);
+        const uint32_t p_lo = pack_bf16(p[0], p[1]), p_hi = pack_bf16(p[2], p[3]);
+        // dQ^T[d, head] += K^T[d, key] dS^T[key, head]
+        {
+            const uint32_t b0 = movmatrix_t(ds_lo), b1 = movmatrix_t(ds_hi);
+            const int mi = lane >> 3;
+            const uint32_t addr = k_s32 + ((lane & 7) + (mi >> 1) * 8) * ROW + (mi & 1) * 16;
+#pragma unroll
+            for (int mt = 0; mt < KS; ++mt) {
+                uint32_t a0, a1, a2, a3;
+                ldmatrix_x4_trans(a0, a1, a2, a3, addr + mt * 32);
+                mma_bf16_16816(dq[mt], a0, a1, a2, a3, b0, b1);
+            }
+        }
+        // dK[key, d] += scale * dS^T[key, head] Q[head, d];   dV'[key, d] += P^T[key, head] do[head, d]
+        {
+            const int32_t key0 = __shfl_sync(0xFFFFFFFFu, pos16, gid), key1 = __shfl_sync(0xFFFFFFFFu, pos16, gid + 8);
+            float* const dk0 = a.dK32 + (((size_t)b * a.Lk + key0) * a.n_kv + g) * DH + 2 * tig;
+            float* const dk1 = a.dK32 + (((size_t)b * a.Lk + key1) * a.n_kv + g) * DH + 2 * tig;
+            float* const dv0 = a.dV32 + (((size_t)b * a.Lk + key0) * a.n_kv + g) * DH + 2 * tig;
+            float* const dv1 = a.dV32 + (((size_t)b * a.Lk + key1) * a.n_kv + g) * DH + 2 * tig;
+            const uint32_t boff = (lane & 7) * ROW + (lane >> 3) * 16;
+#pragma unroll
+            for (int n4 = 0; n4 < DH / 32; ++n4) {       // four 8-wide column tiles of d per step
+                uint32_t bq[4], bd[4];
+                ldmatrix_x4_trans(bq[0], bq[1], bq[2], bq[3], q_s32 + boff + n4 * 64);
+                ldmatrix_x4_trans(bd[0], bd[1], bd[2], bd[3], d_s32 + boff + n4 * 64);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    float ck[4], cv[4];
+                    mma_bf16_1688(ck, ds_lo, ds_hi, bq[i]);
+                    mma_bf16_1688(cv, p_lo, p_hi, bd[i]);
+                    const int col = (n4 * 4 + i) * 8;
+                    if (v0) {
+                        red_add_v2(dk0 + col, ck[0] * a.scale, ck[1] * a.scale);
+                        red_add_v2(dv0 + col, cv[0], cv[1]);
+                    }
+                    if (v1) {
+                        red_add_v2(dk1 + col, ck[2] * a.scale, ck[3] * a.scale);
+                        red_add_v2(dv1 + col, cv[2], cv[3]);
+                    }
+                }
+            }
+        }
+        __syncwarp();                                     // the tiles are rewritten by the next iteration
+    }
+
+    // ---- dQ: rows of the fragment are d, columns the heads 2 tig, 2 tig + 1 ---------------------------
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+        const int hl = 2 * tig + e;
+        if (hl < G) {
+            __nv_bfloat16* const dst = a.dQ + (qrow * a.n_h + (g * G + hl)) * DH;
+#pragma unroll
+            for (int mt = 0; mt < KS; ++mt) {
+                dst[mt * 16 + gid] = __float2bfloat16(dq[mt][e] * a.scale);
+                dst[mt * 16 + gid + 8] = __float2bfloat16(dq[mt][2 + e] * a.scale);
+            }
+        }
+    }
+}
+
+// dK = bf16(dK32);  dV = bf16(dV'32 * sigmoid(g2));  dg2 = bf16(dV'32 * V * sigmoid'(g2))
+__global__ void __launch_bounds__(256) gsa_attn_bwd_finish_kernel(const float* __restrict__ dK32,
+                                                                  const float* __restrict__ dV32,
+                                                                  const __nv_bfloat16* __restrict__ V,
+                                                                  const __nv_bfloat16* __restrict__ g2,
+                                                                  __nv_bfloat16* __restrict__ dK,
+                                                                  __nv_bfloat16* __restrict__ dV,
+                                                                  __nv_bfloat16* __restrict__ dg2, int64_t n) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x * 4;
+    for (int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4; i < n; i += stride) {
+        const float4 k4 = *reinterpret_cast<const float4*>(dK32 + i);
+        const float4 v4 = *reinterpret_cast<const float4*>(dV32 + i);
+        const uint2 vr = *reinterpret_cast<const uint2*>(V + i);
+        const uint2 gr = *reinterpret_cast<const uint2*>(g2 + i);
+        const float dk[4] = {k4.x, k4.y, k4.z, k4.w}, dvg[4] = {v4.x, v4.y, v4.z, v4.w};
+        const __nv_bfloat16* vv = reinterpret_cast<const __nv_bfloat16*>(&vr);
+        const __nv_bfloat16* gg = reinterpret_cast<const __nv_bfloat16*>(&gr);
+        __align__(8) __nv_bfloat16 ok[4], ov[4], og[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float sg = 1.0f / (1.0f + __expf(-__bfloat162float(gg[e])));
+            ok[e] = __float2bfloat16(dk[e]);
+            ov[e] = __float2bfloat16(dvg[e] * sg);
+            og[e] = __float2bfloat16(dvg[e] * __bfloat162float(vv[e]) * sg * (1.0f - sg));
+        }
+        *reinterpret_cast<uint2*>(dK + i) = *reinterpret_cast<const uint2*>(ok);
+        *reinterpret_cast<uint2*>(dV + i) = *reinterpret_cast<const uint2*>(ov);
+        *reinterpret_cast<uint2*>(dg2 + i) = *reinterpret_cast<const uint2*>(og);
+    }
+}
+
+template <int DH, int G>
+cudaError_t launch_bwd_t(const BwdArgs& a, cudaStream_t st) {
+    constexpr int ROW = (DH + 8) * 2;
+    constexpr int WARP_SMEM = 2 * 16 * ROW + 2 * 8 * ROW + 64;
+    const int smem = kBwdWarps * WARP_SMEM;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(gsa_sparse_attn_bwd_kernel<DH, G>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    const int64_t items = (int64_t)a.rr.rows() * a.n_kv;
+    const int64_t ctas = (items + kBwdWarps - 1) / kBwdWarps;
+    gsa_sparse_attn_bwd_kernel<DH, G><<<(unsigned)ctas, kBwdWarps * 32, smem, st>>>(a);
+    ++g_launches;
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+bool attn_bwd_supported(const gsa_params_t& p) {
+    const int G = p.n_h / p.n_kv;
+    return (p.d_h == 128 || p.d_h == 64) && (G == 1 || G == 2 || G == 4 || G == 8);
+}
+
+cudaError_t launch_sparse_attn_bwd(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* Q,
+                                   const __nv_bfloat16* K, const __nv_bfloat16* Vg, const __nv_bfloat16* g1,
+                                   const __nv_bfloat16* out, const __nv_bfloat16* dout, const int32_t* idx,
+                                   const int32_t* kt, IdxLayout il, __nv_bfloat16* dQ, __nv_bfloat16* dg1,
+                                   float* dK32, float* dV32, cudaStream_t st) {
+    if (rr.rows() <= 0) return cudaSuccess;
+    BwdArgs a;
+    a.Q = Q; a.K = K; a.Vg = Vg; a.g1 = g1; a.out = out; a.dout = dout; a.idx = idx; a.kt = kt;
+    a.dQ = dQ; a.dg1 = dg1; a.dK32 = dK32; a.dV32 = dV32; a.rr = rr; a.il = il;
+    a.Lq = p.Lq; a.Lk = p.Lk; a.n_h = p.n_h; a.n_kv = p.n_kv; a.k_max = p.k_max;
+    a.scale = p.sm_scale > 0.f ? p.sm_scale : 1.0f / sqrtf((float)p.d_h);
+    const int G = p.n_h / p.n_kv;
+#define GSA_BWD_CASE(DH_, G_) if (p.d_h == DH_ && G == G_) return launch_bwd_t<DH_, G_>(a, st)
+    GSA_BWD_CASE(128, 1); GSA_BWD_CASE(128, 2); GSA_BWD_CASE(128, 4); GSA_BWD_CASE(128, 8);
+    GSA_BWD_CASE(64, 1); GSA_BWD_CASE(64, 2); GSA_BWD_CASE(64, 4); GSA_BWD_CASE(64, 8);
+#undef GSA_BWD_CASE
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_attn_bwd_finish(const float* dK32, const float* dV32, const __nv_bfloat16* V,
+                                   const __nv_bfloat16* g2, __nv_bfloat16* dK, __nv_bfloat16* dV,
+                                   __nv_bfloat16* dg2, int64_t n_elems, cudaStream_t st) {
+    if (n_elems <= 0) return cudaSuccess;
+    const int64_t want = (n_elems / 4 + 255) / 256;
+    const int blocks = (int)(want < 148 * 16 ? want : 148 * 16);
+    gsa_attn_bwd_finish_kernel<<<blocks, 256, 0, st>>>(dK32, dV32, V, g2, dK, dV, dg2, n_elems);
+    ++g_launches;
+    return cudaGetLastError();
+}
+
+}  // namespace gsa

@@ -46,6 +46,21 @@ cudaError_t launch_select(const gsa_params_t& p, RowRange rr, const float* score
 cudaError_t launch_value_gate(const __nv_bfloat16* V, const __nv_bfloat16* g2, __nv_bfloat16* Vg,
                               int64_t n_elems, cudaStream_t st);
 
+// Backward of sparse gated attention (gsa_attn_bwd.cu): dQ, dg1 for the rows of rr; dK, dV' summed in fp32
+// into dK32 / dV32 (which the caller zeroed); launch_attn_bwd_finish turns those into bf16 dK, dV, dg2.
+bool attn_bwd_supported(const gsa_params_t& p);
+cudaError_t launch_sparse_attn_bwd(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* Q,
+                                   const __nv_bfloat16* K, const __nv_bfloat16* Vg, const __nv_bfloat16* g1,
+                                   const __nv_bfloat16* out, const __nv_bfloat16* dout, const int32_t* idx,
+                                   const int32_t* kt, IdxLayout il, __nv_bfloat16* dQ, __nv_bfloat16* dg1,
+                                   float* dK32, float* dV32, cudaStream_t st);
+cudaError_t launch_attn_bwd_finish(const float* dK32, const float* dV32, const __nv_bfloat16* V,
+                                   const __nv_bfloat16* g2, __nv_bfloat16* dK, __nv_bfloat16* dV,
+                                   __nv_bfloat16* dg2, int64_t n_elems, cudaStream_t st);
+// Running mean of the score variance (gsa_vbar.cu)
+cudaError_t launch_vbar_update(const float* var, int64_t n, float momentum, float* v_bar, float* mean_var,
+                               cudaStream_t st);
+
 // Optional progress report of launch_sparse_attn: output rows become final range by range (a query
 // row is final once the key range holding its last visible key has been processed).  events[i], which
 // the caller created, is recorded when rows t_lo[i] <= t < t_hi[i] of every batch element are final.

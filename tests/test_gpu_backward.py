@@ -1,0 +1,157 @@
+"""GPU parity of the training-side entry points against the fp64 CPU oracle, through the C ABI:
+gsa_sparse_gated_attn_bwd (Eq. 9-12 and Eq. 10 differentiated, index sets fixed) and gsa_vbar_update
+(running mean of the score variance, Eq. 8).
+
+Tolerance of the gradients: the kernel rounds P, dS, dout*sigmoid(g1) and V' to bf16 (2^-9 each) before
+the tensor-core products and every result to bf16 once; sums run in fp32.  As for the forward outputs
+the bound is 2.5e-2 of the tensor's largest magnitude (not of the row's: where the exact derivative
+cancels to zero, as dQ does for a row with a single key, the roundings of the two cancelling terms
+remain), and the error over a whole tensor must stay below 1 % in the Frobenius norm.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2601_15305_b200 import binding as gsa
+from paper_2601_15305_b200.inputs import CONFIGS, make_inputs
+
+import gpu_util as U
+
+pytestmark = pytest.mark.gpu
+
+GRAD_REL_TO_MAX_TOL = 2.5e-2
+GRAD_FROBENIUS_TOL = 1e-2
+
+
+def _index_sets(cfg, q0, q1, seed, k_lo=None, k_hi=None):
+    """Valid ascending random index sets for rows [q0, q1) of every batch element: [B, R, k_max], [B, R]."""
+    g = torch.Generator().manual_seed(seed)
+    R = q1 - q0
+    idx = torch.full((cfg.B, R, cfg.k_max), -1, dtype=torch.int32)
+    kt = torch.empty((cfg.B, R), dtype=torch.int32)
+    for b in range(cfg.B):
+        for r in range(R):
+            n = cfg.Lk - cfg.Lq + q0 + r + 1
+            k = min(n, int(torch.randint(k_lo or cfg.k_min, (k_hi or cfg.k_max) + 1, (1,), generator=g)))
+            idx[b, r, :k] = torch.randperm(n, generator=g)[:k].sort().values.to(torch.int32)
+            kt[b, r] = k
+    return idx, kt
+
+
+def _run_bwd(cfg, d, idx, kt, dout, q0, q1, **over):
+    p = gsa.make_params(cfg, q_begin=q0, q_end=q1, **over)
+    out = U.run_attn(cfg, d, idx, kt, q_begin=q0, q_end=q1, **over)
+    nan = float("nan")
+    dQ, dg1 = torch.full_like(d["Q"], nan), torch.full_like(d["Q"], nan)
+    dK, dV, dg2 = (torch.full_like(d["K"], nan) for _ in range(3))
+    ws = torch.empty(gsa.gsa_attn_bwd_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+    ws.fill_(0xFF)                               # the call must not rely on a cleared workspace
+    n0 = gsa.gsa_launch_count()
+    gsa.gsa_sparse_gated_attn_bwd(p, d["Q"], d["K"], d["V"], d["g1"], d["g2"], idx, kt, out, dout,
+                                  dQ, dK, dV, dg1, dg2, ws)
+    torch.cuda.synchronize()
+    assert gsa.gsa_device_status(ws) == 0
+    assert gsa.gsa_launch_count() - n0 == 3      # value gate, backward kernel, post-pass
+    return dict(dQ=dQ, dg1=dg1, dK=dK, dV=dV, dg2=dg2)
+
+
+def _compare(cfg, x, got, idx, kt, dout, q0, q1, **okw):
+    R = q1 - q0
+    rows_b = np.repeat(np.arange(cfg.B), R)
+    rows_t = np.tile(np.arange(q0, q1), cfg.B)
+    p = U.oracle_params(cfg, **okw)
+    want = oracle.attn_bwd(p, x["Q"], x["K"], x["V"], x["g1"], x["g2"], idx.reshape(cfg.B * R, -1).numpy(),
+                           kt.reshape(-1).numpy(), dout[:, q0:q1].reshape(cfg.B * R, cfg.n_h, cfg.d_h),
+                           rows_t, rows_b)
+    for name in ("dQ", "dg1"):
+        g = got[name][:, q0:q1].float().cpu().numpy().reshape(cfg.B * R, cfg.n_h, cfg.d_h)
+        w = want[name]
+        assert np.isfinite(g).all(), name
+        assert (np.abs(g - w) <= GRAD_REL_TO_MAX_TOL * np.abs(w).max() + 1e-7).all(), (name, np.abs(g - w).max(), np.abs(w).max())
+        assert np.linalg.norm(g - w) <= GRAD_FROBENIUS_TOL * np.linalg.norm(w), name
+        # rows outside the range are left alone (NaN-poisoned)
+        if q0 > 0:
+            assert torch.isnan(got[name][:, :q0].float()).all()
+    for name in ("dK", "dV", "dg2"):
+        g = got[name].float().cpu().numpy()
+        w = want[name]
+        assert np.isfinite(g).all(), name
+        assert np.abs(w).max() > 0
+        assert (np.abs(g - w) <= GRAD_REL_TO_MAX_TOL * np.abs(w).max() + 1e-7).all(), (name, np.abs(g - w).max(), np.abs(w).max())
+        assert np.linalg.norm(g - w) <= GRAD_FROBENIUS_TOL * np.linalg.norm(w), (name, np.linalg.norm(g - w) / np.linalg.norm(w))
+        # keys nobody selected get exactly zero
+        untouched = np.ones(cfg.B * cfg.Lk, bool)
+        for b in range(cfg.B):
+            for r in range(R):
+                untouched[b * cfg.Lk + idx[b, r, : int(kt[b, r])].numpy()] = False
+        assert (g.reshape(cfg.B * cfg.Lk, -1)[untouched] == 0).all(), name
+    return want
+
+
+def test_attn_backward_tiny_all_rows():
+    """Every row of the tiny workload (d_h = 64, four heads on one KV head), budgets from 1 key upwards."""
+    cfg = CONFIGS["tiny"]
+    x = make_inputs(cfg)
+    d = U.to_dev(x)
+    idx, kt = _index_sets(cfg, 0, cfg.Lq, seed=31, k_lo=1)
+    dout = (torch.randn(d["Q"].shape, generator=torch.Generator().manual_seed(32)) * 0.5).to(torch.bfloat16)
+    got = _run_bwd(cfg, d, idx.cuda(), kt.cuda(), dout.cuda(), 0, cfg.Lq)
+    _compare(cfg, x, got, idx, kt, dout, 0, cfg.Lq)
+
+
+def test_attn_backward_l8k_shape_row_range_and_batch():
+    """The benchmark's layer shape (d_h = 128, 16 heads on 8 KV heads) on a batch of two, rows [300, 396)
+    only; ragged budgets (tiles of 16 keys with a tail), custom softmax scale."""
+    cfg = CONFIGS["l8k"].with_(name="bwd", B=2, Lq=396, Lk=1500, k_base=300, k_min=17, k_max=419, seed=33)
+    x = make_inputs(cfg)
+    d = U.to_dev(x)
+    q0, q1 = 300, 396
+    idx, kt = _index_sets(cfg, q0, q1, seed=34)
+    dout = (torch.randn(d["Q"].shape, generator=torch.Generator().manual_seed(35)) * 0.25).to(torch.bfloat16)
+    got = _run_bwd(cfg, d, idx.cuda(), kt.cuda(), dout.cuda(), q0, q1, sm_scale=0.11)
+    _compare(cfg, x, got, idx, kt, dout, q0, q1, sm_scale=0.11)
+
+
+def test_attn_backward_decode_shape_and_wide_groups():
+    """One query row per sequence against a longer cache; eight heads per KV head."""
+    cfg = CONFIGS["l8k"].with_(name="bwd_dec", B=3, Lq=1, Lk=700, n_h=16, n_kv=2, k_base=100, k_min=30, k_max=256, seed=36)
+    x = make_inputs(cfg)
+    d = U.to_dev(x)
+    idx, kt = _index_sets(cfg, 0, 1, seed=37)
+    dout = torch.randn(d["Q"].shape, generator=torch.Generator().manual_seed(38)).to(torch.bfloat16)
+    got = _run_bwd(cfg, d, idx.cuda(), kt.cuda(), dout.cuda(), 0, 1)
+    _compare(cfg, x, got, idx, kt, dout, 0, 1)
+
+
+def test_attn_backward_argument_errors_do_not_launch():
+    cfg = CONFIGS["tiny"]
+    d = U.to_dev(make_inputs(cfg))
+    idx, kt = _index_sets(cfg, 0, cfg.Lq, seed=39)
+    p = gsa.make_params(cfg)
+    z = torch.zeros_like
+    small = torch.zeros(1024, dtype=torch.uint8, device="cuda")
+    n0 = gsa.gsa_launch_count()
+    with pytest.raises(gsa.GsaError, match="workspace"):
+        gsa.gsa_sparse_gated_attn_bwd(p, d["Q"], d["K"], d["V"], d["g1"], d["g2"], idx.cuda(), kt.cuda(), z(d["Q"]),
+                                      z(d["Q"]), z(d["Q"]), z(d["K"]), z(d["K"]), z(d["Q"]), z(d["K"]), small)
+    assert gsa.gsa_launch_count() == n0
+
+
+def test_vbar_update_matches_oracle():
+    g = torch.Generator().manual_seed(40)
+    var = (torch.rand(131072 + 77, generator=g) * 4e-3).float()
+    for momentum, v0 in ((0.99, 2.0e-3), (0.0, 1.0), (1.0, 0.125), (0.5, 3.3e-3)):
+        vb = torch.tensor([v0], dtype=torch.float32, device="cuda")
+        mv = torch.zeros(1, dtype=torch.float32, device="cuda")
+        gsa.gsa_vbar_update(var.cuda(), momentum, vb, mv)
+        new, mean = oracle.vbar_update(float(np.float32(v0)), momentum, var.numpy())
+        assert abs(mv.item() - mean) <= 2e-7 * abs(mean)            # one rounding to fp32
+        assert abs(vb.item() - new) <= 2e-7 * abs(new)
+    # a second step feeds on the first one's result
+    vb = torch.tensor([1.0], dtype=torch.float32, device="cuda")
+    gsa.gsa_vbar_update(var.cuda(), 0.9, vb)
+    first = vb.item()
+    gsa.gsa_vbar_update(var.cuda(), 0.9, vb)
+    want = oracle.vbar_update(first, 0.9, var.numpy())[0]
+    assert abs(vb.item() - want) <= 2e-7 * want
