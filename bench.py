@@ -173,6 +173,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-projection", action="store_true", help="skip timing the upstream projection GEMM")
+    ap.add_argument("--backward", action="store_true",
+                    help="also time gsa_sparse_gated_attn_bwd on the workload's own index sets (adds a 'backward' object)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "gsa_b200" else args.warmup
     cfg = CONFIGS[args.workload]
@@ -312,6 +314,42 @@ def main():
                       "shape": f"M={M} tokens, K={d_model}, N={n_cols} stacked output columns"}
         del Hs, Wt, po
 
+    # ---- backward of the sparse gated attention stage, on the index sets this workload selects ----
+    backward = None
+    if args.backward:
+        idx_b = torch.empty((cfg.B, cfg.Lq, cfg.k_max), dtype=torch.int32, device="cuda")
+        gsa.gsa_forward(p, d["Q"], d["K"], d["V"], d["qI"], d["kI"], d["w"], None, d["g1"], d["g2"], out, idx_b, kt,
+                        None, args.slab_rows, ws, stream)
+        gen = torch.Generator(device="cuda").manual_seed(6)
+        dout = torch.randn(d["Q"].shape, generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        gq = {k: torch.empty_like(d["Q"]) for k in ("dQ", "dg1")}
+        gk = {k: torch.empty_like(d["K"]) for k in ("dK", "dV", "dg2")}
+        ws_b = torch.empty(gsa.gsa_attn_bwd_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+        run_b = lambda: gsa.gsa_sparse_gated_attn_bwd(p, d["Q"], d["K"], d["V"], d["g1"], d["g2"], idx_b, kt, out, dout,
+                                                      gq["dQ"], gk["dK"], gk["dV"], gq["dg1"], gk["dg2"], ws_b, stream)
+        run_b()
+        torch.cuda.synchronize()
+        assert gsa.gsa_device_status(ws_b) == 0
+        be0, be1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_b = 2
+        be0.record(stream)
+        for _ in range(n_b):
+            run_b()
+        be1.record(stream)
+        torch.cuda.synchronize()
+        b_ms = be0.elapsed_time(be1) / n_b
+        # algorithmic bytes: the query-major kernel gathers K twice and V' once per selected (query, key) pair
+        # and KV head (d_h * 2 bytes each); the key-major kernel gathers Q and dout * sigmoid(g1) of every
+        # head once per pair (n_h * d_h * 2 bytes each); plus the index sets and their inverse (4 + 4 bytes)
+        gather = float(kt_sum) * (3 * cfg.n_kv * cfg.d_h * 2 + 2 * cfg.n_h * cfg.d_h * 2 + 8)
+        backward = {"kernels": "gsa_sparse_attn_bwd_kernel + gsa_sparse_attn_bwd_keys_kernel", "ms": b_ms,
+                    "bound": "hbm", "algorithmic_bytes": gather, "achieved_gbs": gather / (b_ms * 1e-3) / 1e9,
+                    "peak_gbs": peaks["hbm_gbs"], "frac": gather / (b_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                    "tokens_per_s": cfg.B * cfg.Lq / (b_ms * 1e-3), "vs_forward": b_ms / (ms_total / args.steps),
+                    "note": "value gate pre-pass, query-major kernel (dQ, dg1), index-set inversion, key-major "
+                            "kernel (dK, dV, dg2); no floating-point atomics"}
+        del idx_b, dout, gq, gk, ws_b
+
     # ---- end to end through the host-buffer entry point ------------------------------------
     e2e = None
     if not args.no_e2e:
@@ -356,7 +394,7 @@ def main():
                 "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                 "config": workload_config(cfg), "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
                 "roofline": roofline, "cpu_baseline": cpu_baseline, "stages": stages,
-                "upstream_projection": projection}
+                "upstream_projection": projection, "backward": backward}
         print(json.dumps(line))
     if world > 1:
         import torch.distributed as dist

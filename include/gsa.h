@@ -136,7 +136,8 @@ int gsa_output_projection(const gsa_params_t *p, int32_t d_model, const void *at
  *   dQ, dg1  [B, Lq, n_h, d_h] bf16: rows of the range are written, other rows are left alone
  *   dK, dV, dg2  [B, Lk, n_kv, d_h] bf16: every element is written; sums over the rows of the range,
  *          accumulated in fp32 (in an order that depends on scheduling) and rounded once
- *   ws     workspace of gsa_attn_bwd_workspace_bytes(p) bytes: status word, V', fp32 dK and dV'
+ *   ws     workspace of gsa_attn_bwd_workspace_bytes(p) bytes (depends on q_begin / q_end): status word,
+ *          V', dout * sigmoid(g1), softmax statistics, and the index sets inverted (key -> query rows)
  * Returns GSA_ERR_WORKSPACE if ws is too small; nothing is launched on an argument error.
  */
 int gsa_attn_bwd_workspace_bytes(const gsa_params_t *p, size_t *bytes);

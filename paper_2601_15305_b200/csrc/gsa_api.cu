@@ -209,17 +209,29 @@ static size_t attn_ws_bytes(const gsa_params_t& p, bool with_prepass) {
     return n;
 }
 
-// workspace of the backward call: [status][V' bf16][dK fp32][dV' fp32]
-static size_t attn_bwd_ws_bytes(const gsa_params_t& p) {
-    const size_t n = (size_t)p.B * p.Lk * p.n_kv * p.d_h;
-    return kStatusBytes + align_up(n * 2, 256) + 2 * align_up(n * 4, 256);
+// workspace of the backward call: [status][V' bf16][do bf16][lse2 fp32][delta fp32][inverted index sets]
+struct BwdPlan {
+    size_t vg_off, dos_off, lse_off, delta_off, inv_off, total;
+};
+static BwdPlan plan_bwd_ws(const gsa_params_t& p, int32_t rows_per_batch) {
+    BwdPlan w;
+    size_t off = kStatusBytes;
+    w.vg_off = off;    off += align_up((size_t)p.B * p.Lk * p.n_kv * p.d_h * 2, 256);
+    w.dos_off = off;   off += align_up((size_t)p.B * p.Lq * p.n_h * p.d_h * 2, 256);
+    w.lse_off = off;   off += align_up((size_t)p.B * p.Lq * p.n_h * 4, 256);
+    w.delta_off = off; off += align_up((size_t)p.B * p.Lq * p.n_h * 4, 256);
+    w.inv_off = off;   off += attn_bwd_invert_bytes(p, rows_per_batch);
+    w.total = off;
+    return w;
 }
 
 int gsa_attn_bwd_workspace_bytes(const gsa_params_t* p, size_t* bytes) {
     int rc = check_params(p);
     if (rc) return rc;
+    RowRange rr;
+    if ((rc = row_range(p, &rr))) return rc;
     if (!bytes) return GSA_ERR_INVALID_ARG;
-    *bytes = attn_bwd_ws_bytes(*p);
+    *bytes = plan_bwd_ws(*p, rr.R).total;
     return GSA_OK;
 }
 
@@ -232,27 +244,31 @@ int gsa_sparse_gated_attn_bwd(const gsa_params_t* p, const void* Q, const void* 
     RowRange rr;
     if ((rc = row_range(p, &rr))) return rc;
     if (!attn_bwd_supported(*p)) return GSA_ERR_UNSUPPORTED_SHAPE;
+    if ((int64_t)p->B * p->Lk >= (1ll << 31) || (int64_t)p->B * rr.R * p->k_max >= (1ll << 31))
+        return GSA_ERR_UNSUPPORTED_SHAPE;
     const void* ptrs[] = {Q, K, V, g1_logits, g2_logits, idx, out, dout, dQ, dK, dV, dg1, dg2};
     for (const void* q : ptrs) if (!q || !aligned16(q)) return GSA_ERR_INVALID_ARG;
     if (!kt) return GSA_ERR_INVALID_ARG;
-    if (!ws || !aligned16(ws) || ws_bytes < attn_bwd_ws_bytes(*p)) return GSA_ERR_WORKSPACE;
+    const BwdPlan wp = plan_bwd_ws(*p, rr.R);
+    if (!ws || !aligned16(ws) || ws_bytes < wp.total) return GSA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
-    const size_t n = (size_t)p->B * p->Lk * p->n_kv * p->d_h;
     char* wsb = (char*)ws;
-    bf16* Vg = (bf16*)(wsb + kStatusBytes);
-    float* dK32 = (float*)(wsb + kStatusBytes + align_up(n * 2, 256));
-    float* dV32 = (float*)((char*)dK32 + align_up(n * 4, 256));
+    bf16* Vg = (bf16*)(wsb + wp.vg_off);
+    bf16* dOs = (bf16*)(wsb + wp.dos_off);
+    float* lse2 = (float*)(wsb + wp.lse_off);
+    float* delta = (float*)(wsb + wp.delta_off);
     cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, st);
-    if (e == cudaSuccess) e = cudaMemsetAsync(dK32, 0, 2 * align_up(n * 4, 256), st);
-    if (e == cudaSuccess) e = launch_value_gate((const bf16*)V, (const bf16*)g2_logits, Vg, (int64_t)n, st);
+    if (e == cudaSuccess)
+        e = launch_value_gate((const bf16*)V, (const bf16*)g2_logits, Vg, (int64_t)p->B * p->Lk * p->n_kv * p->d_h, st);
     IdxLayout il{0, rr.q_begin, rr.R};
     if (e == cudaSuccess)
         e = launch_sparse_attn_bwd(*p, rr, (const bf16*)Q, (const bf16*)K, Vg, (const bf16*)g1_logits,
                                    (const bf16*)out, (const bf16*)dout, idx, kt, il, (bf16*)dQ, (bf16*)dg1,
-                                   dK32, dV32, st);
+                                   dOs, lse2, delta, st);
     if (e == cudaSuccess)
-        e = launch_attn_bwd_finish(dK32, dV32, (const bf16*)V, (const bf16*)g2_logits, (bf16*)dK, (bf16*)dV,
-                                   (bf16*)dg2, (int64_t)n, st);
+        e = launch_sparse_attn_bwd_keys(*p, rr, (const bf16*)Q, dOs, (const bf16*)K, (const bf16*)V, Vg,
+                                        (const bf16*)g2_logits, lse2, delta, idx, kt, il, wsb + wp.inv_off,
+                                        (bf16*)dK, (bf16*)dV, (bf16*)dg2, st);
     return cuda_rc(e);
 }
 

@@ -10,16 +10,16 @@
 // so the saved forward output is all the state the backward needs; the softmax statistics are
 // recomputed from K in a first sweep over S_t.
 //
-// One warp per (query row, KV head).  Per 16 selected keys the K and V' rows are copied (16-byte
-// asynchronous copies) into a private shared-memory tile and every product runs on the tensor cores
-// (bf16 mma.sync, fp32 accumulation) with the keys as M:
-//   S^T[key, head]  = K  . Q^T       dP^T[key, head] = V' . do^T             (A: tile via ldmatrix)
-//   dQ^T[d, head]  += K^T . dS^T                                             (A: tile via ldmatrix.trans)
-//   dK[key, d]      = dS^T . Q       dV'[key, d]     = P^T . do              (m16n8k8: heads are K)
-// dK and dV' are sums over every query that selected the key: they are accumulated in fp32 with
-// vector reductions (red.global.add.v2.f32) into workspace arrays, and a streaming post-pass applies
-// the value gate's derivative and rounds to bf16.  The kernel is bound by those reductions:
-// 2 * n_kv * d_h fp32 additions in L2 per selected (query, key) pair.
+// Two kernels, neither with floating-point atomics:
+//  * this file, query-major: one warp per (query row, KV head).  Per 16 selected keys the K and V' rows
+//    are copied (16-byte asynchronous copies) into a private shared-memory tile and every product runs on
+//    the tensor cores (bf16 mma.sync, fp32 accumulation) with the keys as M:
+//        S^T[key, head] = K . Q^T      dP^T[key, head] = V' . do^T            (A: tile via ldmatrix)
+//        dQ^T[d, head] += K^T . dS^T                                          (A: tile via ldmatrix.trans)
+//    It writes dQ and dg1 and leaves do (bf16), the softmax statistics and delta per (row, head) in the
+//    workspace for
+//  * gsa_attn_bwd_keys.cu, key-major: dK and dV' are sums over every query that selected the key, so the
+//    index sets are first inverted (key -> list of query rows) and one warp per key then walks its list.
 #include "gsa_common.cuh"
 
 namespace gsa {
@@ -40,8 +40,9 @@ struct BwdArgs {
     const int32_t* kt;
     __nv_bfloat16* dQ;
     __nv_bfloat16* dg1;
-    float* dK32;
-    float* dV32;
+    __nv_bfloat16* dOs;           // workspace: do = dout * sigmoid(g1), [B, Lq, n_h, d_h]
+    float* lse2;                  // workspace: log2-domain log-sum-exp of the scaled logits, [B, Lq, n_h]
+    float* delta;                 // workspace: sum_d dout * out, [B, Lq, n_h]
     RowRange rr;
     IdxLayout il;
     int32_t Lq, Lk, n_h, n_kv, k_max;
@@ -58,17 +59,6 @@ __device__ __forceinline__ float ex2_approx(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-// D(16x8, fp32) = A(16x8, bf16, row) * B(8x8, bf16, col)
-__device__ __forceinline__ void mma_bf16_1688(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%7,%8,%9,%10};\n"
-        : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
-        : "r"(a0), "r"(a1), "r"(b0), "f"(0.f), "f"(0.f), "f"(0.f), "f"(0.f));
-}
-__device__ __forceinline__ void red_add_v2(float* addr, float x, float y) {
-    asm volatile("red.global.add.v2.f32 [%0], {%1, %2};" ::"l"(addr), "f"(x), "f"(y) : "memory");
-}
-
 template <int DH, int G>
 __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(const BwdArgs a) {
     constexpr int ROW = (DH + 8) * 2;                  // bytes of a padded tile row (odd multiple of 16)
@@ -120,6 +110,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
                 const float sg = 1.0f / (1.0f + __expf(-__bfloat162float(a.g1[at + e])));
                 qd[e] = a.Q[at + e];
                 dd[e] = __float2bfloat16(dy * sg);
+                a.dOs[at + e] = dd[e];
                 a.dg1[at + e] = __float2bfloat16(dy * y * (1.0f - sg));
                 part = fmaf(dy, y, part);
             }
@@ -129,7 +120,10 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
-        if (lane == 0) s_delta[hl] = part;
+        if (lane == 0) {
+            s_delta[hl] = part;
+            if (hl < G) a.delta[qrow * a.n_h + g * G + hl] = part;
+        }
     }
     __syncwarp();
     const float delta[2] = {s_delta[2 * tig], s_delta[2 * tig + 1]};
@@ -205,6 +199,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
             m_run[e] = m_new;
         }
         lse2[e] = m_run[e] + log2f(l_run[e]);
+        if (gid == 0 && 2 * tig + e < G) a.lse2[qrow * a.n_h + g * G + 2 * tig + e] = lse2[e];
     }
 
     // ---- sweep 2: gradients ---------------------------------------------------------------------------
@@ -230,7 +225,6 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
             ds[2 + e] = p[2 + e] * (dp[2 + e] - delta[e]);
         }
         const uint32_t ds_lo = pack_bf16(ds[0], ds[1]), ds_hi = pack_bf16(ds[2], ds[3]);
-        const uint32_t p_lo = pack_bf16(p[0], p[1]), p_hi = pack_bf16(p[2], p[3]);
         // dQ^T[d, head] += K^T[d, key] dS^T[key, head]
         {
             const uint32_t b0 = movmatrix_t(ds_lo), b1 = movmatrix_t(ds_hi);
@@ -241,36 +235,6 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
                 uint32_t a0, a1, a2, a3;
                 ldmatrix_x4_trans(a0, a1, a2, a3, addr + mt * 32);
                 mma_bf16_16816(dq[mt], a0, a1, a2, a3, b0, b1);
-            }
-        }
-        // dK[key, d] += scale * dS^T[key, head] Q[head, d];   dV'[key, d] += P^T[key, head] do[head, d]
-        {
-            const int32_t key0 = __shfl_sync(0xFFFFFFFFu, pos16, gid), key1 = __shfl_sync(0xFFFFFFFFu, pos16, gid + 8);
-            float* const dk0 = a.dK32 + (((size_t)b * a.Lk + key0) * a.n_kv + g) * DH + 2 * tig;
-            float* const dk1 = a.dK32 + (((size_t)b * a.Lk + key1) * a.n_kv + g) * DH + 2 * tig;
-            float* const dv0 = a.dV32 + (((size_t)b * a.Lk + key0) * a.n_kv + g) * DH + 2 * tig;
-            float* const dv1 = a.dV32 + (((size_t)b * a.Lk + key1) * a.n_kv + g) * DH + 2 * tig;
-            const uint32_t boff = (lane & 7) * ROW + (lane >> 3) * 16;
-#pragma unroll
-            for (int n4 = 0; n4 < DH / 32; ++n4) {       // four 8-wide column tiles of d per step
-                uint32_t bq[4], bd[4];
-                ldmatrix_x4_trans(bq[0], bq[1], bq[2], bq[3], q_s32 + boff + n4 * 64);
-                ldmatrix_x4_trans(bd[0], bd[1], bd[2], bd[3], d_s32 + boff + n4 * 64);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    float ck[4], cv[4];
-                    mma_bf16_1688(ck, ds_lo, ds_hi, bq[i]);
-                    mma_bf16_1688(cv, p_lo, p_hi, bd[i]);
-                    const int col = (n4 * 4 + i) * 8;
-                    if (v0) {
-                        red_add_v2(dk0 + col, ck[0] * a.scale, ck[1] * a.scale);
-                        red_add_v2(dv0 + col, cv[0], cv[1]);
-                    }
-                    if (v1) {
-                        red_add_v2(dk1 + col, ck[2] * a.scale, ck[3] * a.scale);
-                        red_add_v2(dv1 + col, cv[2], cv[3]);
-                    }
-                }
             }
         }
         __syncwarp();                                     // the tiles are rewritten by the next iteration
@@ -288,37 +252,6 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
                 dst[mt * 16 + gid + 8] = __float2bfloat16(dq[mt][2 + e] * a.scale);
             }
         }
-    }
-}
-
-// dK = bf16(dK32);  dV = bf16(dV'32 * sigmoid(g2));  dg2 = bf16(dV'32 * V * sigmoid'(g2))
-__global__ void __launch_bounds__(256) gsa_attn_bwd_finish_kernel(const float* __restrict__ dK32,
-                                                                  const float* __restrict__ dV32,
-                                                                  const __nv_bfloat16* __restrict__ V,
-                                                                  const __nv_bfloat16* __restrict__ g2,
-                                                                  __nv_bfloat16* __restrict__ dK,
-                                                                  __nv_bfloat16* __restrict__ dV,
-                                                                  __nv_bfloat16* __restrict__ dg2, int64_t n) {
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x * 4;
-    for (int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4; i < n; i += stride) {
-        const float4 k4 = *reinterpret_cast<const float4*>(dK32 + i);
-        const float4 v4 = *reinterpret_cast<const float4*>(dV32 + i);
-        const uint2 vr = *reinterpret_cast<const uint2*>(V + i);
-        const uint2 gr = *reinterpret_cast<const uint2*>(g2 + i);
-        const float dk[4] = {k4.x, k4.y, k4.z, k4.w}, dvg[4] = {v4.x, v4.y, v4.z, v4.w};
-        const __nv_bfloat16* vv = reinterpret_cast<const __nv_bfloat16*>(&vr);
-        const __nv_bfloat16* gg = reinterpret_cast<const __nv_bfloat16*>(&gr);
-        __align__(8) __nv_bfloat16 ok[4], ov[4], og[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const float sg = 1.0f / (1.0f + __expf(-__bfloat162float(gg[e])));
-            ok[e] = __float2bfloat16(dk[e]);
-            ov[e] = __float2bfloat16(dvg[e] * sg);
-            og[e] = __float2bfloat16(dvg[e] * __bfloat162float(vv[e]) * sg * (1.0f - sg));
-        }
-        *reinterpret_cast<uint2*>(dK + i) = *reinterpret_cast<const uint2*>(ok);
-        *reinterpret_cast<uint2*>(dV + i) = *reinterpret_cast<const uint2*>(ov);
-        *reinterpret_cast<uint2*>(dg2 + i) = *reinterpret_cast<const uint2*>(og);
     }
 }
 
@@ -352,11 +285,11 @@ cudaError_t launch_sparse_attn_bwd(const gsa_params_t& p, RowRange rr, const __n
                                    const __nv_bfloat16* K, const __nv_bfloat16* Vg, const __nv_bfloat16* g1,
                                    const __nv_bfloat16* out, const __nv_bfloat16* dout, const int32_t* idx,
                                    const int32_t* kt, IdxLayout il, __nv_bfloat16* dQ, __nv_bfloat16* dg1,
-                                   float* dK32, float* dV32, cudaStream_t st) {
+                                   __nv_bfloat16* dOs, float* lse2, float* delta, cudaStream_t st) {
     if (rr.rows() <= 0) return cudaSuccess;
     BwdArgs a;
     a.Q = Q; a.K = K; a.Vg = Vg; a.g1 = g1; a.out = out; a.dout = dout; a.idx = idx; a.kt = kt;
-    a.dQ = dQ; a.dg1 = dg1; a.dK32 = dK32; a.dV32 = dV32; a.rr = rr; a.il = il;
+    a.dQ = dQ; a.dg1 = dg1; a.dOs = dOs; a.lse2 = lse2; a.delta = delta; a.rr = rr; a.il = il;
     a.Lq = p.Lq; a.Lk = p.Lk; a.n_h = p.n_h; a.n_kv = p.n_kv; a.k_max = p.k_max;
     a.scale = p.sm_scale > 0.f ? p.sm_scale : 1.0f / sqrtf((float)p.d_h);
     const int G = p.n_h / p.n_kv;
@@ -365,17 +298,6 @@ cudaError_t launch_sparse_attn_bwd(const gsa_params_t& p, RowRange rr, const __n
     GSA_BWD_CASE(64, 1); GSA_BWD_CASE(64, 2); GSA_BWD_CASE(64, 4); GSA_BWD_CASE(64, 8);
 #undef GSA_BWD_CASE
     return cudaErrorInvalidValue;
-}
-
-cudaError_t launch_attn_bwd_finish(const float* dK32, const float* dV32, const __nv_bfloat16* V,
-                                   const __nv_bfloat16* g2, __nv_bfloat16* dK, __nv_bfloat16* dV,
-                                   __nv_bfloat16* dg2, int64_t n_elems, cudaStream_t st) {
-    if (n_elems <= 0) return cudaSuccess;
-    const int64_t want = (n_elems / 4 + 255) / 256;
-    const int blocks = (int)(want < 148 * 16 ? want : 148 * 16);
-    gsa_attn_bwd_finish_kernel<<<blocks, 256, 0, st>>>(dK32, dV32, V, g2, dK, dV, dg2, n_elems);
-    ++g_launches;
-    return cudaGetLastError();
 }
 
 }  // namespace gsa

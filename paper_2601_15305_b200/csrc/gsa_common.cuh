@@ -46,17 +46,23 @@ cudaError_t launch_select(const gsa_params_t& p, RowRange rr, const float* score
 cudaError_t launch_value_gate(const __nv_bfloat16* V, const __nv_bfloat16* g2, __nv_bfloat16* Vg,
                               int64_t n_elems, cudaStream_t st);
 
-// Backward of sparse gated attention (gsa_attn_bwd.cu): dQ, dg1 for the rows of rr; dK, dV' summed in fp32
-// into dK32 / dV32 (which the caller zeroed); launch_attn_bwd_finish turns those into bf16 dK, dV, dg2.
+// Backward of sparse gated attention.  Query-major half (gsa_attn_bwd.cu): dQ, dg1 for the rows of rr, and
+// per (row, head) do = dout * sigmoid(g1), the softmax statistics lse2 and delta for the key-major half
+// (gsa_attn_bwd_keys.cu), which inverts the index sets inside invert_ws (attn_bwd_invert_bytes) and writes
+// dK, dV, dg2 for every key.
 bool attn_bwd_supported(const gsa_params_t& p);
 cudaError_t launch_sparse_attn_bwd(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* Q,
                                    const __nv_bfloat16* K, const __nv_bfloat16* Vg, const __nv_bfloat16* g1,
                                    const __nv_bfloat16* out, const __nv_bfloat16* dout, const int32_t* idx,
                                    const int32_t* kt, IdxLayout il, __nv_bfloat16* dQ, __nv_bfloat16* dg1,
-                                   float* dK32, float* dV32, cudaStream_t st);
-cudaError_t launch_attn_bwd_finish(const float* dK32, const float* dV32, const __nv_bfloat16* V,
-                                   const __nv_bfloat16* g2, __nv_bfloat16* dK, __nv_bfloat16* dV,
-                                   __nv_bfloat16* dg2, int64_t n_elems, cudaStream_t st);
+                                   __nv_bfloat16* dOs, float* lse2, float* delta, cudaStream_t st);
+size_t attn_bwd_invert_bytes(const gsa_params_t& p, int32_t rows_per_batch);
+cudaError_t launch_sparse_attn_bwd_keys(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* Q,
+                                        const __nv_bfloat16* dOs, const __nv_bfloat16* K, const __nv_bfloat16* V,
+                                        const __nv_bfloat16* Vg, const __nv_bfloat16* g2, const float* lse2,
+                                        const float* delta, const int32_t* idx, const int32_t* kt, IdxLayout il,
+                                        void* invert_ws, __nv_bfloat16* dK, __nv_bfloat16* dV, __nv_bfloat16* dg2,
+                                        cudaStream_t st);
 // Running mean of the score variance (gsa_vbar.cu)
 cudaError_t launch_vbar_update(const float* var, int64_t n, float momentum, float* v_bar, float* mean_var,
                                cudaStream_t st);

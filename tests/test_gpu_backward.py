@@ -52,7 +52,7 @@ def _run_bwd(cfg, d, idx, kt, dout, q0, q1, **over):
                                   dQ, dK, dV, dg1, dg2, ws)
     torch.cuda.synchronize()
     assert gsa.gsa_device_status(ws) == 0
-    assert gsa.gsa_launch_count() - n0 == 3      # value gate, backward kernel, post-pass
+    assert gsa.gsa_launch_count() - n0 == 8      # value gate, query-major kernel, count + 3 scan steps + fill, key-major kernel
     return dict(dQ=dQ, dg1=dg1, dK=dK, dV=dV, dg2=dg2)
 
 
