@@ -52,7 +52,10 @@ def _run_bwd(cfg, d, idx, kt, dout, q0, q1, **over):
                                   dQ, dK, dV, dg1, dg2, ws)
     torch.cuda.synchronize()
     assert gsa.gsa_device_status(ws) == 0
-    assert gsa.gsa_launch_count() - n0 == 8      # value gate, query-major kernel, count + 3 scan steps + fill, key-major kernel
+    # value gate, query-major kernel, count + 3 scan steps, one fill per range of 8192 query rows, key-major
+    # kernel, and with several ranges the post-pass
+    n_ranges = (q1 - q0 + 8191) // 8192
+    assert gsa.gsa_launch_count() - n0 == 7 + n_ranges + (1 if n_ranges > 1 else 0)
     return dict(dQ=dQ, dg1=dg1, dK=dK, dV=dV, dg2=dg2)
 
 
@@ -122,6 +125,19 @@ def test_attn_backward_decode_shape_and_wide_groups():
     dout = torch.randn(d["Q"].shape, generator=torch.Generator().manual_seed(38)).to(torch.bfloat16)
     got = _run_bwd(cfg, d, idx.cuda(), kt.cuda(), dout.cuda(), 0, 1)
     _compare(cfg, x, got, idx, kt, dout, 0, 1)
+
+
+def test_attn_backward_several_query_ranges():
+    """More than 8192 query rows: the key lists are built and walked range by range and the ranges'
+    partial sums meet in fp32 arrays."""
+    cfg = CONFIGS["tiny"].with_(name="bwd_ranges", B=1, Lq=8192 + 777, Lk=8192 + 777, n_h=4, n_kv=2, d_h=64,
+                                k_base=32, k_min=8, k_max=48, seed=41)
+    x = make_inputs(cfg)
+    d = U.to_dev(x)
+    idx, kt = _index_sets(cfg, 0, cfg.Lq, seed=42)
+    dout = (torch.randn(d["Q"].shape, generator=torch.Generator().manual_seed(43)) * 0.5).to(torch.bfloat16)
+    got = _run_bwd(cfg, d, idx.cuda(), kt.cuda(), dout.cuda(), 0, cfg.Lq)
+    _compare(cfg, x, got, idx, kt, dout, 0, cfg.Lq)
 
 
 def test_attn_backward_argument_errors_do_not_launch():
