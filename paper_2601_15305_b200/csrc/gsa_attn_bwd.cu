@@ -63,7 +63,9 @@ template <int DH, int G>
 __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(const BwdArgs a) {
     constexpr int ROW = (DH + 8) * 2;                  // bytes of a padded tile row (odd multiple of 16)
     constexpr int KTILE = 16 * ROW, QTILE = 8 * ROW;
-    constexpr int WARP_SMEM = 2 * KTILE + 2 * QTILE + 64;
+    constexpr int STAGE = 2 * KTILE;                   // a K tile and a V' tile
+    constexpr int WARP_SMEM = 2 * STAGE;               // two stages; the Q / do tiles borrow stage 1 first
+    static_assert(2 * QTILE + 64 <= STAGE, "the row's own tiles must fit one stage");
     constexpr int KS = DH / 16;                        // k-steps of the S^T / dP^T products, m-tiles of dQ^T
     constexpr int EPL = DH / 32;                       // elements of a head row per lane (row staging)
     constexpr int CPR = DH / 8;                        // 16-byte chunks per tile row
@@ -85,13 +87,10 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
     const int32_t* __restrict__ S = a.idx + irow * a.k_max;
 
     unsigned char* const ws = bwd_smem + warp * WARP_SMEM;
-    unsigned char* const k_tile = ws;
-    unsigned char* const v_tile = ws + KTILE;
-    unsigned char* const q_tile = ws + 2 * KTILE;       // rows = the group's heads (rows >= G are zero)
-    unsigned char* const d_tile = ws + 2 * KTILE + QTILE;
-    float* const s_delta = reinterpret_cast<float*>(ws + 2 * KTILE + 2 * QTILE);   // [8]
-    const uint32_t k_s32 = (uint32_t)__cvta_generic_to_shared(k_tile);
-    const uint32_t v_s32 = (uint32_t)__cvta_generic_to_shared(v_tile);
+    unsigned char* const q_tile = ws + STAGE;           // rows = the group's heads (rows >= G are zero)
+    unsigned char* const d_tile = ws + STAGE + QTILE;
+    float* const s_delta = reinterpret_cast<float*>(ws + STAGE + 2 * QTILE);   // [8]
+    const uint32_t st_s32 = (uint32_t)__cvta_generic_to_shared(ws);   // stage i: K tile at i * STAGE, V' tile after it
     const uint32_t q_s32 = (uint32_t)__cvta_generic_to_shared(q_tile);
     const uint32_t d_s32 = (uint32_t)__cvta_generic_to_shared(d_tile);
 
@@ -136,6 +135,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
         ldmatrix_x4(qb[4 * k2], qb[4 * k2 + 1], qb[4 * k2 + 2], qb[4 * k2 + 3], q_s32 + off);
         ldmatrix_x4(dob[4 * k2], dob[4 * k2 + 1], dob[4 * k2 + 2], dob[4 * k2 + 3], d_s32 + off);
     }
+    __syncwarp();                                      // stage 1 is free for tiles from here on
 
     const float c2 = a.scale * kLog2e;
     const size_t kv_row = (size_t)a.n_kv * DH;           // elements between consecutive keys
@@ -166,14 +166,22 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
 
     // ---- sweep 1: softmax statistics per head (log2 domain) ----------------------------------------
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-    for (int j0 = 0; j0 < ke; j0 += 16) {
-        const int32_t pos16 = S[min(j0 + (lane & 15), ke - 1)];
-        fetch_tile(kbase, k_s32, pos16);
-        cp_async_commit();
-        cp_async_wait<0>();
+    // tiles are fetched one iteration ahead
+    auto fetch = [&](int j, int stage, bool with_v) {
+        if (j < ke) {
+            const int32_t pos16 = S[min(j + (lane & 15), ke - 1)];
+            fetch_tile(kbase, st_s32 + stage * STAGE, pos16);
+            if (with_v) fetch_tile(vbase, st_s32 + stage * STAGE + KTILE, pos16);
+        }
+        cp_async_commit();                                // (possibly empty: keeps the group count uniform)
+    };
+    fetch(0, 0, false);
+    for (int j0 = 0, stage = 0; j0 < ke; j0 += 16, stage ^= 1) {
+        fetch(j0 + 16, stage ^ 1, false);
+        cp_async_wait<1>();
         __syncwarp();
         float s[4];
-        tile_times(k_s32, qb, s);
+        tile_times(st_s32 + stage * STAGE, qb, s);
         const bool v0 = j0 + gid < ke, v1 = j0 + gid + 8 < ke;
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
@@ -184,8 +192,9 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
                 m_run[e] = m_new;
             }
         }
-        __syncwarp();
+        __syncwarp();                                     // this stage is refilled by the next iteration
     }
+    cp_async_wait<0>();
     float lse2[2];
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
@@ -206,13 +215,12 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
     float dq[KS][4];
 #pragma unroll
     for (int mt = 0; mt < KS; ++mt) dq[mt][0] = dq[mt][1] = dq[mt][2] = dq[mt][3] = 0.f;
-    for (int j0 = 0; j0 < ke; j0 += 16) {
-        const int32_t pos16 = S[min(j0 + (lane & 15), ke - 1)];
-        fetch_tile(kbase, k_s32, pos16);
-        fetch_tile(vbase, v_s32, pos16);
-        cp_async_commit();
-        cp_async_wait<0>();
+    fetch(0, 0, true);
+    for (int j0 = 0, stage = 0; j0 < ke; j0 += 16, stage ^= 1) {
+        fetch(j0 + 16, stage ^ 1, true);
+        cp_async_wait<1>();
         __syncwarp();
+        const uint32_t k_s32 = st_s32 + stage * STAGE, v_s32 = k_s32 + KTILE;
         float s[4], dp[4], p[4], ds[4];
         tile_times(k_s32, qb, s);
         tile_times(v_s32, dob, dp);
@@ -237,8 +245,9 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
                 mma_bf16_16816(dq[mt], a0, a1, a2, a3, b0, b1);
             }
         }
-        __syncwarp();                                     // the tiles are rewritten by the next iteration
+        __syncwarp();                                     // this stage is refilled by the next iteration
     }
+    cp_async_wait<0>();
 
     // ---- dQ: rows of the fragment are d, columns the heads 2 tig, 2 tig + 1 ---------------------------
 #pragma unroll
@@ -258,7 +267,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
 template <int DH, int G>
 cudaError_t launch_bwd_t(const BwdArgs& a, cudaStream_t st) {
     constexpr int ROW = (DH + 8) * 2;
-    constexpr int WARP_SMEM = 2 * 16 * ROW + 2 * 8 * ROW + 64;
+    constexpr int WARP_SMEM = 4 * 16 * ROW;
     const int smem = kBwdWarps * WARP_SMEM;
     static bool attr_done = false;
     if (!attr_done) {

@@ -159,7 +159,8 @@ struct KeyArgs {
     __nv_bfloat16* dg2;
     int64_t n_keys;               // B * Lk
     int32_t n_h, n_kv, G;
-    int32_t HB;                   // heads per tile row block: min(n_h, 16)
+    int32_t HB;                   // heads per tile row block: min(n_h, 16), a power of two
+    int32_t hb_shift;             // log2(HB)
     int32_t NHB;                  // head blocks: n_h / HB
     float scale;
 };
@@ -252,8 +253,8 @@ __global__ void __launch_bounds__(kKeyWarps * 32) gsa_sparse_attn_bwd_keys_kerne
         dv[mt][0] = dv[mt][1] = dv[mt][2] = dv[mt][3] = 0.f;
     }
     // tile row r = (query r / HB of the tile, head h_base + r % HB); this lane's rows are gid and gid + 8
-    const int q_of_r0 = gid / a.HB, q_of_r1 = (gid + 8) / a.HB;
-    const int h_r0 = h_base + gid % a.HB, h_r1 = h_base + (gid + 8) % a.HB;
+    const int q_of_r0 = gid >> a.hb_shift, q_of_r1 = (gid + 8) >> a.hb_shift;
+    const int h_r0 = h_base + (gid & (a.HB - 1)), h_r1 = h_base + ((gid + 8) & (a.HB - 1));
     const int col_r0 = h_r0 / a.G - g_base, col_r1 = h_r1 / a.G - g_base;     // the one column that counts
 
     // tiles are fetched one iteration ahead, together with the statistics of this lane's two rows
@@ -268,8 +269,8 @@ __global__ void __launch_bounds__(kKeyWarps * 32) gsa_sparse_attn_bwd_keys_kerne
             for (int i = 0; i < 16 * CPR / 32; ++i) {
                 const int chunk = i * 32 + lane;
                 const int r = chunk / CPR, c = chunk % CPR;
-                const int32_t qrow = __shfl_sync(0xFFFFFFFFu, t16, r / a.HB);
-                const size_t at = ((size_t)qrow * a.n_h + h_base + r % a.HB) * DH + c * 8;
+                const int32_t qrow = __shfl_sync(0xFFFFFFFFu, t16, r >> a.hb_shift);
+                const size_t at = ((size_t)qrow * a.n_h + h_base + (r & (a.HB - 1))) * DH + c * 8;
                 cp_async16(q_dst + r * ROW + c * 16, a.Q + at);
                 cp_async16(d_dst + r * ROW + c * 16, a.dOs + at);
             }
@@ -471,6 +472,8 @@ cudaError_t launch_sparse_attn_bwd_keys(const gsa_params_t& p, RowRange rr, cons
     a.n_keys = n_keys; a.n_h = p.n_h; a.n_kv = p.n_kv; a.G = p.n_h / p.n_kv;
     a.HB = p.n_h < 16 ? p.n_h : 16;
     a.NHB = p.n_h / a.HB;
+    a.hb_shift = 0;
+    while ((1 << a.hb_shift) < a.HB) ++a.hb_shift;
     a.scale = p.sm_scale > 0.f ? p.sm_scale : 1.0f / sqrtf((float)p.d_h);
     if (p.d_h != 128 && p.d_h != 64) return cudaErrorInvalidValue;
     if (n_ranges == 1)
