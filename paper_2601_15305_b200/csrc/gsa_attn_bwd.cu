@@ -269,12 +269,10 @@ cudaError_t launch_bwd_t(const BwdArgs& a, cudaStream_t st) {
     constexpr int ROW = (DH + 8) * 2;
     constexpr int WARP_SMEM = 4 * 16 * ROW;
     const int smem = kBwdWarps * WARP_SMEM;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(gsa_sparse_attn_bwd_kernel<DH, G>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    // (set on every call: the attribute belongs to the current device)
+    {
+        cudaError_t e = cudaFuncSetAttribute(gsa_sparse_attn_bwd_kernel<DH, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
-        attr_done = true;
     }
     const int64_t items = (int64_t)a.rr.rows() * a.n_kv;
     const int64_t ctas = (items + kBwdWarps - 1) / kBwdWarps;

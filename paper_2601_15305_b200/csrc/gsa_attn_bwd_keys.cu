@@ -383,12 +383,10 @@ cudaError_t launch_keys_t(const KeyArgs& a, int n_ranges, cudaStream_t st) {
     constexpr int ROW = (DH + 8) * 2;
     constexpr int WARP_SMEM = 4 * 16 * ROW;
     const int smem = kKeyWarps * WARP_SMEM;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(gsa_sparse_attn_bwd_keys_kernel<DH, PARTIAL>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    // (set on every call: the attribute belongs to the current device)
+    {
+        cudaError_t e = cudaFuncSetAttribute(gsa_sparse_attn_bwd_keys_kernel<DH, PARTIAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
-        attr_done = true;
     }
     const int64_t items = a.n_keys * a.NHB * n_ranges;
     const int64_t ctas = (items + kKeyWarps - 1) / kKeyWarps;

@@ -573,11 +573,10 @@ cudaError_t launch_select(const gsa_params_t& p, RowRange rr, const float* score
     a.k_base = p.k_base; a.k_min = p.k_min; a.k_max = p.k_max; a.k_mode = p.k_mode; a.v_bar = p.v_bar;
 
     const size_t smem = ((sizeof(SelShared) + 15) / 16) * 16;
-    static bool attr_done = false;
-    if (!attr_done) {
+    // (set on every call: the attribute belongs to the current device)
+    {
         cudaError_t e = cudaFuncSetAttribute(gsa_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        attr_done = true;
     }
     gsa_select_kernel<<<rr.rows(), kSelThreads, smem, st>>>(a);
     ++g_launches;
