@@ -249,3 +249,39 @@ def vbar_update(v_bar: float, momentum: float, var) -> tuple:
     m = ctypes.c_double(0.0)
     new = f(ctypes.c_double(v_bar), ctypes.c_double(momentum), _ptr(v), ctypes.c_int64(v.size), ctypes.byref(m))
     return float(new), float(m.value)
+
+
+def attn_probs_mean(p: OracleParams, Q, K, idx, keff, rows_t, rows_b=None) -> np.ndarray:
+    """Target of the indexer's sparse-phase loss (Eq. 14): the attention distribution of Eq. 11 on S_t,
+    averaged over the heads.  [n, k_max] float64, zeros past keff."""
+    rows_b, rows_t = _rows(p, rows_t, rows_b)
+    Q, K = _f32(Q), _f32(K)
+    idx, keff = _i32(idx), _i32(keff).reshape(-1)
+    n = len(rows_t)
+    assert idx.shape == (n, p.k_max) and keff.shape == (n,)
+    out = np.empty((n, p.k_max), dtype=np.float64)
+    c = p.c()
+    lib().gsa_oracle_attn_probs_mean_rows(ctypes.byref(c), _ptr(Q), _ptr(K), _ptr(rows_b), _ptr(rows_t),
+                                          ctypes.c_int(n), _ptr(idx), _ptr(keff), _ptr(out))
+    return out
+
+
+def indexer_kl(p: OracleParams, qI, kI, w, bI, idx, keff, pbar, rows_t, rows_b=None):
+    """Eq. 14 for the listed rows with the target distribution pbar [n, k_max] given, and its derivatives.
+    Returns dict(loss [n], dqI [n, HI, dI], dw [n, HI], dkI [B, Lk, dI], dbI [HI]), all float64."""
+    rows_b, rows_t = _rows(p, rows_t, rows_b)
+    qI, kI, w, bI = _f32(qI), _f32(kI), _f32(w), _f32(bI)
+    idx, keff = _i32(idx), _i32(keff).reshape(-1)
+    pbar = np.ascontiguousarray(pbar, dtype=np.float64)
+    n = len(rows_t)
+    assert idx.shape == (n, p.k_max) and keff.shape == (n,) and pbar.shape == (n, p.k_max)
+    loss = np.empty(n, dtype=np.float64)
+    dqI = np.empty((n, p.HI, p.dI), dtype=np.float64)
+    dw = np.empty((n, p.HI), dtype=np.float64)
+    dkI = np.empty((p.B, p.Lk, p.dI), dtype=np.float64)
+    dbI = np.empty(p.HI, dtype=np.float64)
+    c = p.c()
+    lib().gsa_oracle_indexer_kl_rows(ctypes.byref(c), _ptr(qI), _ptr(kI), _ptr(w), _ptr(bI), _ptr(rows_b),
+                                     _ptr(rows_t), ctypes.c_int(n), _ptr(idx), _ptr(keff), _ptr(pbar),
+                                     _ptr(loss), _ptr(dqI), _ptr(dw), _ptr(dkI), _ptr(dbI))
+    return dict(loss=loss, dqI=dqI, dw=dw, dkI=dkI, dbI=dbI)

@@ -35,7 +35,9 @@
  * and gates are saturated, single-key and equal-logit closed forms, g1 = -40 -> 0.
  * Training side (end of this file): the backward of Eq. 9-12 and Eq. 10 is pinned by central differences
  * of the forward above, by library autograd on the forward written as masked dense attention, and by the
- * single-key / shift-invariance closed forms; the running mean of the variance by a worked example.
+ * single-key / shift-invariance closed forms; the running mean of the variance by a worked example; the
+ * indexer's sparse-phase loss (Eq. 14) and its derivatives by library softmax / KL divergence / autograd, a
+ * two-key closed form, the zero of the loss at target = softmax(I), and central differences.
  * Parity unpinned: nothing (every function above has at least one such pin); the
  * absolute values on random data have no printed reference in the paper.
  */
@@ -403,4 +405,112 @@ double gsa_oracle_vbar_update(double v_bar, double momentum, const float *var, i
     const double m = n > 0 ? s / (double)n : 0.0;
     if (mean_var) *mean_var = m;
     return momentum * v_bar + (1.0 - momentum) * m;
+}
+
+/* ---- the indexer's sparse-phase loss (Sec. 5.1, Eq. 14) ------------------------ */
+/* Target of the loss: the attention distribution on S_t.  Eq. 11 gives one distribution per head; the
+ * indexer score has no head index, so the target is their mean over the n_h heads (each sums to 1 over
+ * S_t, hence so does the mean).  pbar: [n_rows, k_max], entries past keff are 0. */
+void gsa_oracle_attn_probs_mean_rows(const gsa_oracle_params *p, const float *Q, const float *K,
+                                     const int32_t *rows_b, const int32_t *rows_t, int n_rows,
+                                     const int32_t *idx, const int32_t *keff, double *pbar)
+{
+    const int d = p->d_h, grp = p->n_h / p->n_kv;
+    const double scale = p->sm_scale > 0.0 ? p->sm_scale : 1.0 / sqrt((double)d);
+    const size_t qrow = (size_t)p->n_h * d, kvb = (size_t)p->Lk * p->n_kv * d;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int r = 0; r < n_rows; ++r) {
+        const int b = rows_b[r], t = rows_t[r], ke = keff[r];
+        const int32_t *S = idx + (size_t)r * p->k_max;
+        double *out = pbar + (size_t)r * p->k_max;
+        double *z = (double *)malloc(sizeof(double) * (size_t)(ke > 0 ? ke : 1));
+        for (int j = 0; j < p->k_max; ++j) out[j] = 0.0;
+        for (int h = 0; h < p->n_h; ++h) {
+            const int g = h / grp;
+            const float *q = Q + ((size_t)b * p->Lq + t) * qrow + (size_t)h * d;
+            double zmax = -INFINITY, den = 0.0;
+            for (int j = 0; j < ke; ++j) {
+                const float *ks = K + b * kvb + ((size_t)S[j] * p->n_kv + g) * d;
+                double dot = 0.0;
+                for (int c = 0; c < d; ++c) dot += (double)q[c] * (double)ks[c];
+                z[j] = dot * scale;
+                if (z[j] > zmax) zmax = z[j];
+            }
+            for (int j = 0; j < ke; ++j) { z[j] = exp(z[j] - zmax); den += z[j]; }
+            for (int j = 0; j < ke; ++j) out[j] += z[j] / den / (double)p->n_h;
+        }
+        free(z);
+    }
+}
+
+/* Eq. 14 for the listed rows, with the target distribution given (a constant: no derivative flows into it):
+ *     loss_t = sum_{j in S_t} pbar_j * (log pbar_j - log q_j),   q = softmax_j(I[t, s_j]),   0 log 0 = 0,
+ * I from Eq. 7 (or Eq. 3 with act = 1).  Derivatives of sum_t loss_t by the chain rule:
+ *     dI_j = q_j * sum_i pbar_i - pbar_j                       (= q_j - pbar_j for a normalised target)
+ *     with x_ij = q^I_i . k^I_{s_j} + b_i and f = sigmoid (or ReLU):
+ *     dw_i = sum_j dI_j f(x_ij),   dx_ij = dI_j w_i f'(x_ij),
+ *     dq^I_i = sum_j dx_ij k^I_{s_j},   dk^I[s_j] += sum_i dx_ij q^I_i,   db_i += sum_j dx_ij.
+ * loss: [n_rows]; dqI: [n_rows, HI, dI]; dw: [n_rows, HI]; dkI: [B, Lk, dI] and dbI: [HI], zeroed here and
+ * summed over the listed rows.  Rows run one after the other (no two threads add into dkI). */
+void gsa_oracle_indexer_kl_rows(const gsa_oracle_params *p, const float *qI, const float *kI,
+                                const float *w, const float *bI, const int32_t *rows_b,
+                                const int32_t *rows_t, int n_rows, const int32_t *idx,
+                                const int32_t *keff, const double *pbar, double *loss, double *dqI,
+                                double *dw, double *dkI, double *dbI)
+{
+    const int H = p->HI, D = p->dI;
+    memset(dkI, 0, sizeof(double) * (size_t)p->B * p->Lk * D);
+    for (int i = 0; i < H; ++i) dbI[i] = 0.0;
+    double *I = (double *)malloc(sizeof(double) * (size_t)(p->k_max > 0 ? p->k_max : 1));
+    double *x = (double *)malloc(sizeof(double) * (size_t)(p->k_max > 0 ? p->k_max : 1) * H);
+    for (int r = 0; r < n_rows; ++r) {
+        const int b = rows_b[r], t = rows_t[r], ke = keff[r];
+        const int32_t *S = idx + (size_t)r * p->k_max;
+        const double *pb = pbar + (size_t)r * p->k_max;
+        const float *q = qI + ((size_t)b * p->Lq + t) * H * D;
+        const float *wt = w + ((size_t)b * p->Lq + t) * H;
+        double imax = -INFINITY, den = 0.0, psum = 0.0;
+        for (int j = 0; j < ke; ++j) {
+            const float *k = kI + ((size_t)b * p->Lk + S[j]) * D;
+            double acc = 0.0;
+            for (int i = 0; i < H; ++i) {
+                double v = bI ? (double)bI[i] : 0.0;
+                for (int c = 0; c < D; ++c) v += (double)q[i * D + c] * (double)k[c];
+                x[(size_t)j * H + i] = v;
+                acc += (double)wt[i] * (p->act == 1 ? (v > 0.0 ? v : 0.0) : sigmoid_d(v));
+            }
+            I[j] = acc;
+            if (acc > imax) imax = acc;
+            psum += pb[j];
+        }
+        for (int j = 0; j < ke; ++j) den += exp(I[j] - imax);
+        const double logden = imax + log(den);
+        double L = 0.0;
+        for (int j = 0; j < ke; ++j)
+            if (pb[j] > 0.0) L += pb[j] * (log(pb[j]) - (I[j] - logden));
+        loss[r] = L;
+        for (int i = 0; i < H; ++i) {
+            dw[(size_t)r * H + i] = 0.0;
+            for (int c = 0; c < D; ++c) dqI[((size_t)r * H + i) * D + c] = 0.0;
+        }
+        for (int j = 0; j < ke; ++j) {
+            const double dI = exp(I[j] - logden) * psum - pb[j];
+            const float *k = kI + ((size_t)b * p->Lk + S[j]) * D;
+            double *dk = dkI + ((size_t)b * p->Lk + S[j]) * D;
+            for (int i = 0; i < H; ++i) {
+                const double v = x[(size_t)j * H + i];
+                double f, fp;
+                if (p->act == 1) { f = v > 0.0 ? v : 0.0; fp = v > 0.0 ? 1.0 : 0.0; }
+                else { f = sigmoid_d(v); fp = f * (1.0 - f); }
+                dw[(size_t)r * H + i] += dI * f;
+                const double dx = dI * (double)wt[i] * fp;
+                dbI[i] += dx;
+                for (int c = 0; c < D; ++c) {
+                    dqI[((size_t)r * H + i) * D + c] += dx * (double)k[c];
+                    dk[c] += dx * (double)q[i * D + c];
+                }
+            }
+        }
+    }
+    free(I); free(x);
 }

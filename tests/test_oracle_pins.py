@@ -539,6 +539,106 @@ def test_vbar_update_closed_form():
     assert oracle.vbar_update(0.5, 1.0, np.array([9.0, 1.0], np.float32))[0] == 0.5
 
 
+# ------------------------------------------------------------------ Eq. 14: the indexer's sparse-phase loss
+def _kl_problem(seed=0, act=0, **kw):
+    p = small_params(**{**dict(B=2, Lq=5, Lk=9, n_h=4, n_kv=2, d_h=8, HI=3, dI=4, k_max=5, act=act), **kw})
+    g = torch.Generator().manual_seed(seed)
+    r = lambda *s: torch.randn(*s, generator=g).to(torch.bfloat16)
+    x = dict(Q=r(p.B, p.Lq, p.n_h, p.d_h), K=r(p.B, p.Lk, p.n_kv, p.d_h), qI=r(p.B, p.Lq, p.HI, p.dI),
+             kI=r(p.B, p.Lk, p.dI), w=torch.rand(p.B, p.Lq, p.HI, generator=g).float() * 0.9 + 0.05,
+             bI=torch.tensor([0.25, -0.5, 0.125][: p.HI]))
+    rows_b, rows_t, idx, keff = _rand_index_sets(p, seed + 1)
+    return p, x, rows_b, rows_t, idx, keff
+
+
+def test_attn_probs_mean_is_library_softmax_averaged_over_heads():
+    p, x, rows_b, rows_t, idx, keff = _kl_problem(11)
+    got = oracle.attn_probs_mean(p, x["Q"], x["K"], idx, keff, rows_t, rows_b)
+    grp = p.n_h // p.n_kv
+    for r, (b, t) in enumerate(zip(rows_b, rows_t)):
+        S = torch.from_numpy(idx[r, : keff[r]]).long()
+        acc = torch.zeros(keff[r], dtype=torch.float64)
+        for h in range(p.n_h):
+            z = (x["K"][b, S, h // grp].double() @ x["Q"][b, t, h].double()) / math.sqrt(p.d_h)
+            acc += torch.softmax(z, dim=0)
+        np.testing.assert_allclose(got[r, : keff[r]], (acc / p.n_h).numpy(), rtol=1e-12, atol=1e-15)
+        assert (got[r, keff[r]:] == 0).all()
+        assert abs(got[r].sum() - 1.0) < 1e-12
+
+
+@pytest.mark.parametrize("act", [0, 1])
+def test_indexer_kl_loss_and_gradients_match_library_autograd(act):
+    """Eq. 7 (or Eq. 3) on the selected keys, log-softmax and KL divergence written with torch's library
+    routines in fp64 and differentiated by autograd."""
+    p, x, rows_b, rows_t, idx, keff = _kl_problem(12, act=act)
+    pbar = oracle.attn_probs_mean(p, x["Q"], x["K"], idx, keff, rows_t, rows_b)
+    got = oracle.indexer_kl(p, x["qI"], x["kI"], x["w"], x["bI"], idx, keff, pbar, rows_t, rows_b)
+    t64 = {k: x[k].double().clone().requires_grad_(True) for k in ("qI", "kI", "w", "bI")}
+    total = 0.0
+    for r, (b, t) in enumerate(zip(rows_b, rows_t)):
+        S = torch.from_numpy(idx[r, : keff[r]]).long()
+        z = t64["kI"][b, S] @ t64["qI"][b, t].T + t64["bI"]                      # [k, HI]
+        f = torch.relu(z) if act else torch.sigmoid(z)
+        I = f @ t64["w"][b, t]
+        tgt = torch.from_numpy(pbar[r, : keff[r]])
+        L = torch.nn.functional.kl_div(torch.log_softmax(I, dim=0), tgt, reduction="sum")
+        np.testing.assert_allclose(got["loss"][r], L.item(), rtol=1e-10, atol=1e-13)
+        assert got["loss"][r] >= -1e-15
+        total = total + L
+    total.backward()
+    np.testing.assert_allclose(got["dqI"], t64["qI"].grad.numpy()[rows_b, rows_t], rtol=1e-9, atol=1e-13)
+    np.testing.assert_allclose(got["dw"], t64["w"].grad.numpy()[rows_b, rows_t], rtol=1e-9, atol=1e-13)
+    np.testing.assert_allclose(got["dkI"], t64["kI"].grad.numpy(), rtol=1e-9, atol=1e-13)
+    np.testing.assert_allclose(got["dbI"], t64["bI"].grad.numpy(), rtol=1e-9, atol=1e-13)
+
+
+def test_indexer_kl_closed_forms_and_central_differences():
+    """Equal indexer keys give equal scores, so q is uniform: with the target (1/4, 3/4) the loss is
+    1/4 ln(1/2) + 3/4 ln(3/2) and the derivative with respect to the two scores is (1/2 - 1/4, 1/2 - 3/4).
+    A target equal to softmax(I) gives loss 0 and zero derivatives.  Then central
+    differences of the loss itself for sampled elements of q^I, k^I and w."""
+    p = small_params(B=1, Lq=3, Lk=3, HI=2, dI=4, k_max=2)
+    qI = torch.randn(1, 3, 2, 4, generator=torch.Generator().manual_seed(1)).to(torch.bfloat16)
+    kI = torch.ones(1, 3, 4).to(torch.bfloat16) * 0.5
+    w = torch.tensor([[[0.5, 0.25]] * 3])
+    idx = np.array([[0, 2]], np.int32)
+    got = oracle.indexer_kl(p, qI, kI, w, None, idx, [2], np.array([[0.25, 0.75]]), rows_t=[2])
+    assert abs(got["loss"][0] - (0.25 * math.log(0.5) + 0.75 * math.log(1.5))) < 1e-14
+    # dI = (1/4, -1/4): the two keys are equal, so dq^I (a sum over keys of dI * ... * k^I) cancels
+    assert np.abs(got["dqI"]).max() < 1e-15 and np.abs(got["dw"]).max() < 1e-15
+    assert np.abs(got["dkI"][0, 0] + got["dkI"][0, 2]).max() < 1e-15 and np.abs(got["dkI"][0, 0]).max() > 1e-4
+    assert (got["dkI"][0, 1] == 0).all()
+
+    pr, x, rows_b, rows_t, idx, keff = _kl_problem(13)
+    pbar = oracle.attn_probs_mean(pr, x["Q"], x["K"], idx, keff, rows_t, rows_b)
+    # target = the indexer's own distribution -> nothing to learn
+    sc = oracle.scores(pr, x["qI"], x["kI"], x["w"], x["bI"], rows_t, rows_b)
+    own = np.zeros_like(pbar)
+    for r in range(len(rows_t)):
+        e = np.exp(sc[r, idx[r, : keff[r]]])
+        own[r, : keff[r]] = e / e.sum()
+    z = oracle.indexer_kl(pr, x["qI"], x["kI"], x["w"], x["bI"], idx, keff, own, rows_t, rows_b)
+    assert np.abs(z["loss"]).max() < 1e-14 and np.abs(z["dqI"]).max() < 1e-14 and np.abs(z["dkI"]).max() < 1e-14
+
+    got = oracle.indexer_kl(pr, x["qI"], x["kI"], x["w"], x["bI"], idx, keff, pbar, rows_t, rows_b)
+    full = dict(qI=np.zeros(x["qI"].shape), w=np.zeros(x["w"].shape), kI=got["dkI"])
+    full["qI"][rows_b, rows_t] = got["dqI"]
+    full["w"][rows_b, rows_t] = got["dw"]
+    loss = lambda xx: float(oracle.indexer_kl(pr, xx["qI"], xx["kI"], xx["w"], xx["bI"], idx, keff, pbar,
+                                              rows_t, rows_b)["loss"].sum())
+    eps = 2.0 ** -9
+    rng = np.random.default_rng(3)
+    for name, gr in full.items():
+        base = x[name].float().numpy()
+        for f in rng.choice(base.size, size=25, replace=False):
+            at = np.unravel_index(f, base.shape)
+            hi, lo = base.copy(), base.copy()
+            hi[at] += eps
+            lo[at] -= eps
+            fd = (loss({**x, name: hi}) - loss({**x, name: lo})) / (2 * eps)
+            assert abs(fd - gr[at]) <= 1e-4 * np.abs(gr).max() + 1e-10, (name, at, fd, gr[at])
+
+
 def test_paper_printed_cost_model():
     """Appendix A prints d^I H^I/(d n_h) ~ 0.002 and a 12.8x speed-up for its parameters."""
     vals = {}
