@@ -147,6 +147,38 @@ int gsa_sparse_gated_attn_bwd(const gsa_params_t *p, const void *Q, const void *
                               void *dV, void *dg1, void *dg2, void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * The indexer's sparse-phase loss (Sec. 5.1, Eq. 14) for rows [q_begin, q_end):
+ *     loss_t = sum_{j in S_t} pbar[t, j] * (log pbar[t, j] - log q_j),     q = softmax_j I[t, s_j],
+ * I from Eq. 7 (or Eq. 3 with act = 1), with 0 log 0 = 0.  The target is a constant of the loss.
+ *
+ * gsa_attn_probs_mean writes the target: Eq. 11 gives one attention distribution over S_t per head and the
+ * indexer score has no head index, so pbar[t, j] is their mean over the n_h heads (the paper says "the
+ * softmax attention" without naming the reduction over heads).
+ *   Q, K, idx, kt   as given to gsa_sparse_gated_attn_fwd
+ *   pbar   [B, R, k_max] fp32: entry j belongs to key idx[.., j]; entries past kt are 0
+ *   ws     workspace, ws_bytes >= 256 (device status word)
+ *
+ * gsa_indexer_kl_bwd computes the loss per row and the derivatives of the sum of the rows' losses:
+ *     dI_j = q_j * sum_i pbar_i - pbar_j,    with x_ij = q^I_i . k^I_{s_j} + b_i and f = sigmoid (or ReLU):
+ *     dw_i = sum_j dI_j f(x_ij),   dx_ij = dI_j w_i f'(x_ij),   dq^I_i = sum_j dx_ij k^I_{s_j},
+ *     dk^I[s] = sum over (t, i, j: s_j = s) of dx_ij q^I_i,      db_i = sum over (t, j) of dx_ij.
+ *   qI, kI, w, bI   as given to gsa_indexer_scores (bI may be NULL); w is the weight after its sigmoid,
+ *                   dw the derivative with respect to that value
+ *   pbar   [B, R, k_max] fp32 (any non-negative target works; it need not sum to 1)
+ *   loss   [B, R] fp32
+ *   dqI    [B, Lq, HI, dI] bf16 and dw [B, Lq, HI] fp32: rows of the range are written
+ *   dkI    [B, Lk, dI] bf16: every element is written (fp32 sums, order depends on scheduling, rounded once)
+ *   dbI    [HI] fp32 or NULL (fp32 atomics: order depends on scheduling)
+ *   ws     workspace of gsa_indexer_kl_workspace_bytes(p) bytes: status word and the fp32 sums of dk^I
+ */
+int gsa_attn_probs_mean(const gsa_params_t *p, const void *Q, const void *K, const int32_t *idx,
+                        const int32_t *kt, float *pbar, void *ws, size_t ws_bytes, void *stream);
+int gsa_indexer_kl_workspace_bytes(const gsa_params_t *p, size_t *bytes);
+int gsa_indexer_kl_bwd(const gsa_params_t *p, const void *qI, const void *kI, const float *w, const float *bI,
+                       const int32_t *idx, const int32_t *kt, const float *pbar, float *loss, void *dqI,
+                       void *dkI, float *dw, float *dbI, void *ws, size_t ws_bytes, void *stream);
+
+/*
  * Running mean of the score variance: the normaliser v_bar of Eq. 8 is an exponential moving average of
  * the score variance across the batch.  The paper gives neither momentum nor start value: both are the
  * caller's.

@@ -23,6 +23,7 @@ EXPORTS = (
     "gsa_sparse_gated_attn_fwd_static", "gsa_attn_workspace_bytes", "gsa_debug_set_attn_range_keys",
     "gsa_select_fallback_rows", "gsa_project", "gsa_project_columns", "gsa_output_projection",
     "gsa_attn_bwd_workspace_bytes", "gsa_sparse_gated_attn_bwd", "gsa_vbar_update",
+    "gsa_attn_probs_mean", "gsa_indexer_kl_workspace_bytes", "gsa_indexer_kl_bwd",
 )
 
 STATIC_SCRATCH_BYTES = 32 << 20     # GSA_STATIC_SCRATCH_BYTES of include/gsa.h
@@ -164,6 +165,26 @@ def gsa_sparse_gated_attn_bwd(p, Q, K, V, g1, g2, idx, kt, out, dout, dQ, dK, dV
                                            _dp(dg1, BF16), _dp(dg2, BF16), _dp(ws),
                                            ctypes.c_size_t(ws.numel() * ws.element_size()), _stream(stream)),
            "gsa_sparse_gated_attn_bwd")
+
+
+def gsa_attn_probs_mean(p, Q, K, idx, kt, pbar, ws, stream=None) -> None:
+    _check(lib().gsa_attn_probs_mean(ctypes.byref(p), _dp(Q, BF16), _dp(K, BF16), _dp(idx, I32), _dp(kt, I32),
+                                     _dp(pbar, F32), _dp(ws), ctypes.c_size_t(ws.numel() * ws.element_size()),
+                                     _stream(stream)), "gsa_attn_probs_mean")
+
+
+def gsa_indexer_kl_workspace_bytes(p) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().gsa_indexer_kl_workspace_bytes(ctypes.byref(p), ctypes.byref(n)), "gsa_indexer_kl_workspace_bytes")
+    return int(n.value)
+
+
+def gsa_indexer_kl_bwd(p, qI, kI, w, bI, idx, kt, pbar, loss, dqI, dkI, dw, dbI, ws, stream=None) -> None:
+    _check(lib().gsa_indexer_kl_bwd(ctypes.byref(p), _dp(qI, BF16), _dp(kI, BF16), _dp(w, F32), _dp(bI, F32),
+                                    _dp(idx, I32), _dp(kt, I32), _dp(pbar, F32), _dp(loss, F32), _dp(dqI, BF16),
+                                    _dp(dkI, BF16), _dp(dw, F32), _dp(dbI, F32), _dp(ws),
+                                    ctypes.c_size_t(ws.numel() * ws.element_size()), _stream(stream)),
+           "gsa_indexer_kl_bwd")
 
 
 def gsa_vbar_update(var, momentum: float, v_bar, mean_var=None, stream=None) -> None:

@@ -272,6 +272,53 @@ int gsa_sparse_gated_attn_bwd(const gsa_params_t* p, const void* Q, const void* 
     return cuda_rc(e);
 }
 
+int gsa_attn_probs_mean(const gsa_params_t* p, const void* Q, const void* K, const int32_t* idx,
+                        const int32_t* kt, float* pbar, void* ws, size_t ws_bytes, void* stream) {
+    int rc = check_params(p);
+    if (rc) return rc;
+    RowRange rr;
+    if ((rc = row_range(p, &rr))) return rc;
+    if (!attn_bwd_supported(*p)) return GSA_ERR_UNSUPPORTED_SHAPE;
+    if (!Q || !K || !idx || !kt || !pbar || !aligned16(Q) || !aligned16(K) || !aligned16(idx) || !aligned16(pbar))
+        return GSA_ERR_INVALID_ARG;
+    if (!ws || !aligned16(ws) || ws_bytes < (size_t)kStatusBytes) return GSA_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, st);
+    IdxLayout il{0, rr.q_begin, rr.R};
+    if (e == cudaSuccess) e = launch_attn_probs_mean(*p, rr, (const bf16*)Q, (const bf16*)K, idx, kt, il, pbar, st);
+    return cuda_rc(e);
+}
+
+int gsa_indexer_kl_workspace_bytes(const gsa_params_t* p, size_t* bytes) {
+    int rc = check_params(p);
+    if (rc) return rc;
+    if (!bytes) return GSA_ERR_INVALID_ARG;
+    *bytes = kStatusBytes + align_up((size_t)p->B * p->Lk * p->dI * 4, 256);
+    return GSA_OK;
+}
+
+int gsa_indexer_kl_bwd(const gsa_params_t* p, const void* qI, const void* kI, const float* w, const float* bI,
+                       const int32_t* idx, const int32_t* kt, const float* pbar, float* loss, void* dqI,
+                       void* dkI, float* dw, float* dbI, void* ws, size_t ws_bytes, void* stream) {
+    int rc = check_params(p);
+    if (rc) return rc;
+    RowRange rr;
+    if ((rc = row_range(p, &rr))) return rc;
+    const void* ptrs[] = {qI, kI, w, idx, pbar, dqI, dkI};
+    for (const void* q : ptrs) if (!q || !aligned16(q)) return GSA_ERR_INVALID_ARG;
+    if (!kt || !loss || !dw) return GSA_ERR_INVALID_ARG;
+    size_t need = 0;
+    gsa_indexer_kl_workspace_bytes(p, &need);
+    if (!ws || !aligned16(ws) || ws_bytes < need) return GSA_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, st);
+    IdxLayout il{0, rr.q_begin, rr.R};
+    if (e == cudaSuccess)
+        e = launch_indexer_kl(*p, rr, (const bf16*)qI, (const bf16*)kI, w, bI, idx, kt, il, pbar, loss, (bf16*)dqI,
+                              (bf16*)dkI, dw, dbI, (float*)((char*)ws + kStatusBytes), st);
+    return cuda_rc(e);
+}
+
 int gsa_vbar_update(const float* var, int64_t n, float momentum, float* v_bar, float* mean_var, void* stream) {
     if (!var || !v_bar || n < 1 || !(momentum >= 0.f && momentum <= 1.f)) return GSA_ERR_INVALID_ARG;
     return cuda_rc(launch_vbar_update(var, n, momentum, v_bar, mean_var, (cudaStream_t)stream));

@@ -63,6 +63,17 @@ cudaError_t launch_sparse_attn_bwd_keys(const gsa_params_t& p, RowRange rr, cons
                                         const float* delta, const int32_t* idx, const int32_t* kt, IdxLayout il,
                                         void* invert_ws, __nv_bfloat16* dK, __nv_bfloat16* dV, __nv_bfloat16* dg2,
                                         cudaStream_t st);
+// The indexer's sparse-phase loss (gsa_indexer_loss.cu): its target (mean over the heads of the attention
+// distribution on S_t; pbar is zeroed inside) and the loss with its derivatives (dkI32: B * Lk * dI floats
+// of scratch, zeroed inside; dbI may be null).
+cudaError_t launch_attn_probs_mean(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* Q,
+                                   const __nv_bfloat16* K, const int32_t* idx, const int32_t* kt, IdxLayout il,
+                                   float* pbar, cudaStream_t st);
+cudaError_t launch_indexer_kl(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* qI,
+                              const __nv_bfloat16* kI, const float* w, const float* bI, const int32_t* idx,
+                              const int32_t* kt, IdxLayout il, const float* pbar, float* loss,
+                              __nv_bfloat16* dqI, __nv_bfloat16* dkI, float* dw, float* dbI, float* dkI32,
+                              cudaStream_t st);
 // Running mean of the score variance (gsa_vbar.cu)
 cudaError_t launch_vbar_update(const float* var, int64_t n, float momentum, float* v_bar, float* mean_var,
                                cudaStream_t st);

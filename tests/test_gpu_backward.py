@@ -1,6 +1,7 @@
 """GPU parity of the training-side entry points against the fp64 CPU oracle, through the C ABI:
-gsa_sparse_gated_attn_bwd (Eq. 9-12 and Eq. 10 differentiated, index sets fixed) and gsa_vbar_update
-(running mean of the score variance, Eq. 8).
+gsa_sparse_gated_attn_bwd (Eq. 9-12 and Eq. 10 differentiated, index sets fixed), gsa_vbar_update
+(running mean of the score variance, Eq. 8), and the indexer's sparse-phase loss (Eq. 14):
+gsa_attn_probs_mean (its target) and gsa_indexer_kl_bwd (loss and derivatives).
 
 Tolerance of the gradients: the kernel rounds P, dS, dout*sigmoid(g1) and V' to bf16 (2^-9 each) before
 the tensor-core products and every result to bf16 once; sums run in fp32.  As for the forward outputs
@@ -171,3 +172,85 @@ def test_vbar_update_matches_oracle():
     gsa.gsa_vbar_update(var.cuda(), 0.9, vb)
     want = oracle.vbar_update(first, 0.9, var.numpy())[0]
     assert abs(vb.item() - want) <= 2e-7 * want
+
+
+# ------------------------------------------------------------------------- the indexer's loss (Eq. 14)
+def _run_probs(cfg, d, idx, kt, q0, q1, **over):
+    p = gsa.make_params(cfg, q_begin=q0, q_end=q1, **over)
+    pbar = torch.full((cfg.B, q1 - q0, cfg.k_max), float("nan"), dtype=torch.float32, device="cuda")
+    ws = torch.zeros(1024, dtype=torch.uint8, device="cuda")
+    gsa.gsa_attn_probs_mean(p, d["Q"], d["K"], idx, kt, pbar, ws)
+    torch.cuda.synchronize()
+    assert gsa.gsa_device_status(ws) == 0
+    return pbar
+
+
+def _run_kl(cfg, d, bI, idx, kt, pbar, q0, q1, **over):
+    p = gsa.make_params(cfg, q_begin=q0, q_end=q1, **over)
+    nan = float("nan")
+    loss = torch.full((cfg.B, q1 - q0), nan, dtype=torch.float32, device="cuda")
+    dqI = torch.full_like(d["qI"], nan)
+    dkI = torch.full_like(d["kI"], nan)
+    dw = torch.full_like(d["w"], nan)
+    dbI = torch.full((cfg.HI,), nan, dtype=torch.float32, device="cuda")
+    ws = torch.empty(gsa.gsa_indexer_kl_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+    ws.fill_(0xFF)
+    gsa.gsa_indexer_kl_bwd(p, d["qI"], d["kI"], d["w"], bI, idx, kt, pbar, loss, dqI, dkI, dw, dbI, ws)
+    torch.cuda.synchronize()
+    assert gsa.gsa_device_status(ws) == 0
+    return dict(loss=loss, dqI=dqI, dkI=dkI, dw=dw, dbI=dbI)
+
+
+def _check_loss_path(cfg, q0, q1, seed, bias=False, act=0, **over):
+    """Both entry points against the oracle.  The loss kernel is fed the oracle's target rounded to fp32, so
+    its own comparison does not inherit the target kernel's rounding."""
+    x = make_inputs(cfg)
+    d = U.to_dev(x)
+    idx, kt = _index_sets(cfg, q0, q1, seed=seed)
+    R = q1 - q0
+    rows_b, rows_t = np.repeat(np.arange(cfg.B), R), np.tile(np.arange(q0, q1), cfg.B)
+    p = U.oracle_params(cfg, act=act, **over)
+    idx2, kt1 = idx.reshape(cfg.B * R, -1).numpy(), kt.reshape(-1).numpy()
+
+    want_p = oracle.attn_probs_mean(p, x["Q"], x["K"], idx2, kt1, rows_t, rows_b)
+    got_p = _run_probs(cfg, d, idx.cuda(), kt.cuda(), q0, q1, **over).cpu().numpy().reshape(cfg.B * R, -1)
+    # probabilities: fp32 sums of 2^(.) from bf16 products; 2e-3 relative plus a floor for the tiny ones
+    assert np.isfinite(got_p).all()
+    assert (np.abs(got_p - want_p) <= 2e-3 * want_p + 1e-7).all(), np.abs(got_p - want_p).max()
+    assert np.abs(got_p.sum(axis=1) - 1.0).max() <= 1e-4
+    for r in range(cfg.B * R):
+        assert (got_p[r, kt1[r]:] == 0).all()
+
+    bI = torch.tensor([0.3, -0.2, 0.1, 0.0, -0.4, 0.25, 0.05, -0.1][: cfg.HI]) if bias else None
+    pb32 = want_p.astype(np.float32)
+    want = oracle.indexer_kl(p, x["qI"], x["kI"], x["w"], bI, idx2, kt1, pb32.astype(np.float64), rows_t, rows_b)
+    got = _run_kl(cfg, d, None if bI is None else bI.cuda(), idx.cuda(), kt.cuda(),
+                  torch.from_numpy(pb32).reshape(cfg.B, R, -1).cuda(), q0, q1, act=act, **over)
+    gl = got["loss"].cpu().numpy().reshape(-1)
+    # the loss is a difference of O(log k) terms held in fp32
+    assert (np.abs(gl - want["loss"]) <= 2e-3 * np.abs(want["loss"]) + 2e-5).all(), np.abs(gl - want["loss"]).max()
+    cmp = dict(dqI=(got["dqI"][:, q0:q1].float().cpu().numpy().reshape(cfg.B * R, cfg.HI, cfg.dI), want["dqI"]),
+               dw=(got["dw"][:, q0:q1].cpu().numpy().reshape(cfg.B * R, cfg.HI), want["dw"]),
+               dkI=(got["dkI"].float().cpu().numpy(), want["dkI"]),
+               dbI=(got["dbI"].cpu().numpy(), want["dbI"]))
+    for name, (g, w) in cmp.items():
+        assert np.isfinite(g).all(), name
+        assert np.abs(w).max() > 0, name
+        assert (np.abs(g - w) <= GRAD_REL_TO_MAX_TOL * np.abs(w).max() + 1e-7).all(), (name, np.abs(g - w).max(), np.abs(w).max())
+        assert np.linalg.norm(g - w) <= GRAD_FROBENIUS_TOL * np.linalg.norm(w), (name, np.linalg.norm(g - w) / np.linalg.norm(w))
+    if q0 > 0:
+        assert torch.isnan(got["dqI"][:, :q0].float()).all() and torch.isnan(got["dw"][:, :q0]).all()
+
+
+def test_indexer_kl_tiny_all_rows():
+    _check_loss_path(CONFIGS["tiny"], 0, CONFIGS["tiny"].Lq, seed=51)
+
+
+def test_indexer_kl_layer_shape_row_range_batch_bias():
+    cfg = CONFIGS["l8k"].with_(name="kl", B=2, Lq=396, Lk=1500, k_base=300, k_min=17, k_max=419, seed=52)
+    _check_loss_path(cfg, 300, 396, seed=53, bias=True)
+
+
+def test_indexer_kl_relu_indexer():
+    cfg = CONFIGS["l8k"].with_(name="kl_relu", B=1, Lq=200, Lk=900, HI=4, dI=32, k_base=100, k_min=20, k_max=160, seed=54)
+    _check_loss_path(cfg, 0, 200, seed=55, bias=True, act=1)
