@@ -325,8 +325,10 @@ def main():
         gq = {k: torch.empty_like(d["Q"]) for k in ("dQ", "dg1")}
         gk = {k: torch.empty_like(d["K"]) for k in ("dK", "dV", "dg2")}
         ws_b = torch.empty(gsa.gsa_attn_bwd_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+        pbar = torch.empty((cfg.B, cfg.Lq, cfg.k_max), dtype=torch.float32, device="cuda")
         run_b = lambda: gsa.gsa_sparse_gated_attn_bwd(p, d["Q"], d["K"], d["V"], d["g1"], d["g2"], idx_b, kt, out, dout,
-                                                      gq["dQ"], gk["dK"], gk["dV"], gq["dg1"], gk["dg2"], ws_b, stream)
+                                                      gq["dQ"], gk["dK"], gk["dV"], gq["dg1"], gk["dg2"], ws_b, stream,
+                                                      pbar=pbar)
         run_b()
         torch.cuda.synchronize()
         assert gsa.gsa_device_status(ws_b) == 0
@@ -346,9 +348,35 @@ def main():
                     "bound": "hbm", "algorithmic_bytes": gather, "achieved_gbs": gather / (b_ms * 1e-3) / 1e9,
                     "peak_gbs": peaks["hbm_gbs"], "frac": gather / (b_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                     "tokens_per_s": cfg.B * cfg.Lq / (b_ms * 1e-3), "vs_forward": b_ms / (ms_total / args.steps),
-                    "note": "value gate pre-pass, query-major kernel (dQ, dg1), index-set inversion, key-major "
-                            "kernel (dK, dV, dg2); no floating-point atomics"}
-        del idx_b, dout, gq, gk, ws_b
+                    "note": "value gate pre-pass, query-major kernel (dQ, dg1, and the indexer loss's target as a "
+                            "by-product), index-set inversion, key-major kernel (dK, dV, dg2)"}
+        del dout, gq, gk, ws_b
+        # the indexer's sparse-phase loss (Eq. 14) on the same index sets: its target, then loss + derivatives
+        loss_rows = torch.empty((cfg.B, cfg.Lq), dtype=torch.float32, device="cuda")
+        dqI, dkI, dw = torch.empty_like(d["qI"]), torch.empty_like(d["kI"]), torch.empty_like(d["w"])
+        dbI = torch.empty((cfg.HI,), dtype=torch.float32, device="cuda")
+        ws_s = torch.zeros(1024, dtype=torch.uint8, device="cuda")
+        ws_k = torch.empty(gsa.gsa_indexer_kl_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+        run_t = lambda: gsa.gsa_attn_probs_mean(p, d["Q"], d["K"], idx_b, kt, pbar, ws_s, stream)
+        run_k = lambda: gsa.gsa_indexer_kl_bwd(p, d["qI"], d["kI"], d["w"], None, idx_b, kt, pbar, loss_rows, dqI, dkI,
+                                               dw, dbI, ws_k, stream)
+        run_t(); run_k()
+        torch.cuda.synchronize()
+        assert gsa.gsa_device_status(ws_s) == 0 and gsa.gsa_device_status(ws_k) == 0
+        le = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        le[0].record(stream)
+        for _ in range(n_b):
+            run_t()
+        le[1].record(stream)
+        for _ in range(n_b):
+            run_k()
+        le[2].record(stream)
+        torch.cuda.synchronize()
+        backward["indexer_loss"] = {"target_ms": le[0].elapsed_time(le[1]) / n_b, "loss_and_grads_ms": le[1].elapsed_time(le[2]) / n_b,
+                                    "mean_loss": float(loss_rows.double().mean().item()),
+                                    "note": "target_ms: gsa_attn_probs_mean on its own (the backward call above already "
+                                            "emits the same target); gsa_indexer_kl_bwd gathers k^I, dk^I by fp32 vector reductions"}
+        del idx_b, pbar, loss_rows, dqI, dkI, dw, ws_k
 
     # ---- end to end through the host-buffer entry point ------------------------------------
     e2e = None

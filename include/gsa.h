@@ -136,6 +136,8 @@ int gsa_output_projection(const gsa_params_t *p, int32_t d_model, const void *at
  *   dQ, dg1  [B, Lq, n_h, d_h] bf16: rows of the range are written, other rows are left alone
  *   dK, dV, dg2  [B, Lk, n_kv, d_h] bf16: every element is written; sums over the rows of the range,
  *          accumulated in fp32 (in an order that depends on scheduling) and rounded once
+ *   pbar   [B, R, k_max] fp32 or NULL: the target of the indexer's loss (what gsa_attn_probs_mean writes,
+ *          see below), which this call's second sweep has at hand: one call instead of two
  *   ws     workspace of gsa_attn_bwd_workspace_bytes(p) bytes (depends on q_begin / q_end): status word,
  *          V', dout * sigmoid(g1), softmax statistics, and the index sets inverted (key -> query rows)
  * Returns GSA_ERR_WORKSPACE if ws is too small; nothing is launched on an argument error.
@@ -144,7 +146,8 @@ int gsa_attn_bwd_workspace_bytes(const gsa_params_t *p, size_t *bytes);
 int gsa_sparse_gated_attn_bwd(const gsa_params_t *p, const void *Q, const void *K, const void *V,
                               const void *g1_logits, const void *g2_logits, const int32_t *idx,
                               const int32_t *kt, const void *out, const void *dout, void *dQ, void *dK,
-                              void *dV, void *dg1, void *dg2, void *ws, size_t ws_bytes, void *stream);
+                              void *dV, void *dg1, void *dg2, float *pbar, void *ws, size_t ws_bytes,
+                              void *stream);
 
 /*
  * The indexer's sparse-phase loss (Sec. 5.1, Eq. 14) for rows [q_begin, q_end):

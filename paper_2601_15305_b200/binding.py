@@ -158,11 +158,12 @@ def gsa_attn_bwd_workspace_bytes(p) -> int:
     return int(n.value)
 
 
-def gsa_sparse_gated_attn_bwd(p, Q, K, V, g1, g2, idx, kt, out, dout, dQ, dK, dV, dg1, dg2, ws, stream=None) -> None:
+def gsa_sparse_gated_attn_bwd(p, Q, K, V, g1, g2, idx, kt, out, dout, dQ, dK, dV, dg1, dg2, ws, stream=None,
+                              pbar=None) -> None:
     _check(lib().gsa_sparse_gated_attn_bwd(ctypes.byref(p), _dp(Q, BF16), _dp(K, BF16), _dp(V, BF16), _dp(g1, BF16),
                                            _dp(g2, BF16), _dp(idx, I32), _dp(kt, I32), _dp(out, BF16),
                                            _dp(dout, BF16), _dp(dQ, BF16), _dp(dK, BF16), _dp(dV, BF16),
-                                           _dp(dg1, BF16), _dp(dg2, BF16), _dp(ws),
+                                           _dp(dg1, BF16), _dp(dg2, BF16), _dp(pbar, F32), _dp(ws),
                                            ctypes.c_size_t(ws.numel() * ws.element_size()), _stream(stream)),
            "gsa_sparse_gated_attn_bwd")
 

@@ -238,7 +238,8 @@ int gsa_attn_bwd_workspace_bytes(const gsa_params_t* p, size_t* bytes) {
 int gsa_sparse_gated_attn_bwd(const gsa_params_t* p, const void* Q, const void* K, const void* V,
                               const void* g1_logits, const void* g2_logits, const int32_t* idx,
                               const int32_t* kt, const void* out, const void* dout, void* dQ, void* dK,
-                              void* dV, void* dg1, void* dg2, void* ws, size_t ws_bytes, void* stream) {
+                              void* dV, void* dg1, void* dg2, float* pbar, void* ws, size_t ws_bytes,
+                              void* stream) {
     int rc = check_params(p);
     if (rc) return rc;
     RowRange rr;
@@ -248,7 +249,7 @@ int gsa_sparse_gated_attn_bwd(const gsa_params_t* p, const void* Q, const void* 
         return GSA_ERR_UNSUPPORTED_SHAPE;
     const void* ptrs[] = {Q, K, V, g1_logits, g2_logits, idx, out, dout, dQ, dK, dV, dg1, dg2};
     for (const void* q : ptrs) if (!q || !aligned16(q)) return GSA_ERR_INVALID_ARG;
-    if (!kt) return GSA_ERR_INVALID_ARG;
+    if (!kt || (pbar && !aligned16(pbar))) return GSA_ERR_INVALID_ARG;
     const BwdPlan wp = plan_bwd_ws(*p, rr.R);
     if (!ws || !aligned16(ws) || ws_bytes < wp.total) return GSA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
@@ -261,10 +262,11 @@ int gsa_sparse_gated_attn_bwd(const gsa_params_t* p, const void* Q, const void* 
     if (e == cudaSuccess)
         e = launch_value_gate((const bf16*)V, (const bf16*)g2_logits, Vg, (int64_t)p->B * p->Lk * p->n_kv * p->d_h, st);
     IdxLayout il{0, rr.q_begin, rr.R};
+    if (e == cudaSuccess && pbar) e = cudaMemsetAsync(pbar, 0, (size_t)rr.rows() * p->k_max * 4, st);
     if (e == cudaSuccess)
         e = launch_sparse_attn_bwd(*p, rr, (const bf16*)Q, (const bf16*)K, Vg, (const bf16*)g1_logits,
                                    (const bf16*)out, (const bf16*)dout, idx, kt, il, (bf16*)dQ, (bf16*)dg1,
-                                   dOs, lse2, delta, st);
+                                   dOs, lse2, delta, pbar, st);
     if (e == cudaSuccess)
         e = launch_sparse_attn_bwd_keys(*p, rr, (const bf16*)Q, dOs, (const bf16*)K, (const bf16*)V, Vg,
                                         (const bf16*)g2_logits, lse2, delta, idx, kt, il, wsb + wp.inv_off,

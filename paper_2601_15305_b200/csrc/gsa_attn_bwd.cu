@@ -43,6 +43,7 @@ struct BwdArgs {
     __nv_bfloat16* dOs;           // workspace: do = dout * sigmoid(g1), [B, Lq, n_h, d_h]
     float* lse2;                  // workspace: log2-domain log-sum-exp of the scaled logits, [B, Lq, n_h]
     float* delta;                 // workspace: sum_d dout * out, [B, Lq, n_h]
+    float* pbar;                  // optional output: mean over the heads of P on S_t, [B, R, k_max], pre-zeroed
     RowRange rr;
     IdxLayout il;
     int32_t Lq, Lk, n_h, n_kv, k_max;
@@ -232,6 +233,22 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
             ds[e] = p[e] * (dp[e] - delta[e]);
             ds[2 + e] = p[2 + e] * (dp[2 + e] - delta[e]);
         }
+        if (a.pbar) {
+            // the target of the indexer's loss (Eq. 14) falls out of this sweep: sum the group's heads per
+            // key (rows gid, gid + 8), one fp32 atomic per key and KV head
+            float r0 = 0.f, r1 = 0.f;
+#pragma unroll
+            for (int e = 0; e < 2; ++e)
+                if (2 * tig + e < G) { r0 += p[e]; r1 += p[2 + e]; }
+            r0 += __shfl_xor_sync(0xFFFFFFFFu, r0, 1); r0 += __shfl_xor_sync(0xFFFFFFFFu, r0, 2);
+            r1 += __shfl_xor_sync(0xFFFFFFFFu, r1, 1); r1 += __shfl_xor_sync(0xFFFFFFFFu, r1, 2);
+            if (tig == 0) {
+                float* const prow = a.pbar + irow * a.k_max;
+                const float inv_heads = 1.0f / (float)a.n_h;
+                if (v0) atomicAdd(prow + j0 + gid, r0 * inv_heads);
+                if (v1) atomicAdd(prow + j0 + gid + 8, r1 * inv_heads);
+            }
+        }
         const uint32_t ds_lo = pack_bf16(ds[0], ds[1]), ds_hi = pack_bf16(ds[2], ds[3]);
         // dQ^T[d, head] += K^T[d, key] dS^T[key, head]
         {
@@ -292,11 +309,11 @@ cudaError_t launch_sparse_attn_bwd(const gsa_params_t& p, RowRange rr, const __n
                                    const __nv_bfloat16* K, const __nv_bfloat16* Vg, const __nv_bfloat16* g1,
                                    const __nv_bfloat16* out, const __nv_bfloat16* dout, const int32_t* idx,
                                    const int32_t* kt, IdxLayout il, __nv_bfloat16* dQ, __nv_bfloat16* dg1,
-                                   __nv_bfloat16* dOs, float* lse2, float* delta, cudaStream_t st) {
+                                   __nv_bfloat16* dOs, float* lse2, float* delta, float* pbar, cudaStream_t st) {
     if (rr.rows() <= 0) return cudaSuccess;
     BwdArgs a;
     a.Q = Q; a.K = K; a.Vg = Vg; a.g1 = g1; a.out = out; a.dout = dout; a.idx = idx; a.kt = kt;
-    a.dQ = dQ; a.dg1 = dg1; a.dOs = dOs; a.lse2 = lse2; a.delta = delta; a.rr = rr; a.il = il;
+    a.dQ = dQ; a.dg1 = dg1; a.dOs = dOs; a.lse2 = lse2; a.delta = delta; a.pbar = pbar; a.rr = rr; a.il = il;
     a.Lq = p.Lq; a.Lk = p.Lk; a.n_h = p.n_h; a.n_kv = p.n_kv; a.k_max = p.k_max;
     a.scale = p.sm_scale > 0.f ? p.sm_scale : 1.0f / sqrtf((float)p.d_h);
     const int G = p.n_h / p.n_kv;

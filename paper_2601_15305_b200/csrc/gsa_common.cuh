@@ -55,7 +55,7 @@ cudaError_t launch_sparse_attn_bwd(const gsa_params_t& p, RowRange rr, const __n
                                    const __nv_bfloat16* K, const __nv_bfloat16* Vg, const __nv_bfloat16* g1,
                                    const __nv_bfloat16* out, const __nv_bfloat16* dout, const int32_t* idx,
                                    const int32_t* kt, IdxLayout il, __nv_bfloat16* dQ, __nv_bfloat16* dg1,
-                                   __nv_bfloat16* dOs, float* lse2, float* delta, cudaStream_t st);
+                                   __nv_bfloat16* dOs, float* lse2, float* delta, float* pbar, cudaStream_t st);
 size_t attn_bwd_invert_bytes(const gsa_params_t& p, int32_t rows_per_batch);
 cudaError_t launch_sparse_attn_bwd_keys(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* Q,
                                         const __nv_bfloat16* dOs, const __nv_bfloat16* K, const __nv_bfloat16* V,

@@ -46,18 +46,19 @@ def _run_bwd(cfg, d, idx, kt, dout, q0, q1, **over):
     nan = float("nan")
     dQ, dg1 = torch.full_like(d["Q"], nan), torch.full_like(d["Q"], nan)
     dK, dV, dg2 = (torch.full_like(d["K"], nan) for _ in range(3))
+    pbar = torch.full((cfg.B, q1 - q0, cfg.k_max), nan, dtype=torch.float32, device="cuda")
     ws = torch.empty(gsa.gsa_attn_bwd_workspace_bytes(p), dtype=torch.uint8, device="cuda")
     ws.fill_(0xFF)                               # the call must not rely on a cleared workspace
     n0 = gsa.gsa_launch_count()
     gsa.gsa_sparse_gated_attn_bwd(p, d["Q"], d["K"], d["V"], d["g1"], d["g2"], idx, kt, out, dout,
-                                  dQ, dK, dV, dg1, dg2, ws)
+                                  dQ, dK, dV, dg1, dg2, ws, pbar=pbar)
     torch.cuda.synchronize()
     assert gsa.gsa_device_status(ws) == 0
     # value gate, query-major kernel, count + 3 scan steps, one fill per range of 8192 query rows, key-major
     # kernel, and with several ranges the post-pass
     n_ranges = (q1 - q0 + 8191) // 8192
     assert gsa.gsa_launch_count() - n0 == 7 + n_ranges + (1 if n_ranges > 1 else 0)
-    return dict(dQ=dQ, dg1=dg1, dK=dK, dV=dV, dg2=dg2)
+    return dict(dQ=dQ, dg1=dg1, dK=dK, dV=dV, dg2=dg2, pbar=pbar)
 
 
 def _compare(cfg, x, got, idx, kt, dout, q0, q1, **okw):
@@ -90,6 +91,11 @@ def _compare(cfg, x, got, idx, kt, dout, q0, q1, **okw):
             for r in range(R):
                 untouched[b * cfg.Lk + idx[b, r, : int(kt[b, r])].numpy()] = False
         assert (g.reshape(cfg.B * cfg.Lk, -1)[untouched] == 0).all(), name
+    # the optional by-product: the target of the indexer's loss (same bound as in the test of gsa_attn_probs_mean)
+    want_p = oracle.attn_probs_mean(p, x["Q"], x["K"], idx.reshape(cfg.B * R, -1).numpy(), kt.reshape(-1).numpy(),
+                                    rows_t, rows_b)
+    got_p = got["pbar"].cpu().numpy().reshape(cfg.B * R, -1)
+    assert (np.abs(got_p - want_p) <= 2e-3 * want_p + 1e-7).all(), np.abs(got_p - want_p).max()
     return want
 
 
