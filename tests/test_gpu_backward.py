@@ -134,6 +134,20 @@ def test_attn_backward_decode_shape_and_wide_groups():
     _compare(cfg, x, got, idx, kt, dout, 0, 1)
 
 
+@pytest.mark.parametrize("n_h,n_kv,d_h", [(32, 8, 64), (8, 8, 128), (2, 1, 64), (1, 1, 128), (64, 8, 64)])
+def test_attn_backward_head_layouts(n_h, n_kv, d_h):
+    """Head counts on either side of the 16-row tile of the key-major kernel: several queries per tile
+    (n_h < 16), several head blocks per key (n_h > 16), one head per KV head, eight heads per KV head."""
+    cfg = CONFIGS["tiny"].with_(name=f"bwd_h{n_h}", B=2, Lq=70, Lk=150, n_h=n_h, n_kv=n_kv, d_h=d_h,
+                                k_base=40, k_min=5, k_max=61, seed=60 + n_h)
+    x = make_inputs(cfg)
+    d = U.to_dev(x)
+    idx, kt = _index_sets(cfg, 0, cfg.Lq, seed=61)
+    dout = (torch.randn(d["Q"].shape, generator=torch.Generator().manual_seed(62)) * 0.5).to(torch.bfloat16)
+    got = _run_bwd(cfg, d, idx.cuda(), kt.cuda(), dout.cuda(), 0, cfg.Lq)
+    _compare(cfg, x, got, idx, kt, dout, 0, cfg.Lq)
+
+
 def test_attn_backward_several_query_ranges():
     """More than 8192 query rows: the key lists are built and walked range by range and the ranges'
     partial sums meet in fp32 arrays."""
