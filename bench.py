@@ -166,7 +166,8 @@ def main():
     ap.add_argument("--impl", default="gsa_b200", choices=["gsa_b200", "reference"])
     ap.add_argument("--slab-rows", type=int, default=0)
     ap.add_argument("--act", default="sigmoid", choices=["sigmoid", "relu"], help="indexer activation (Eq. 7 / Eq. 3)")
-    ap.add_argument("--k-mode", type=int, default=0, choices=[0, 1, 2], help="0 Eq. 8, 1 inverse, 2 fixed k = k_base")
+    ap.add_argument("--k-mode", type=int, default=0, choices=[0, 1, 2, 3],
+                    help="0 Eq. 8, 1 inverse, 2 fixed k = k_base, 3 every visible key (needs k_max >= Lk)")
     ap.add_argument("--k-base", type=int, default=0, help="override the base budget (k sweep)")
     ap.add_argument("--lq", type=int, default=0, help="only the last LQ query rows (chunked prefill; smaller ncu captures)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (smaller ncu captures)")

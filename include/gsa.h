@@ -62,7 +62,11 @@ typedef struct gsa_params {
     int32_t k_max;
     int32_t k_mode;     /* 0: Eq. 8 as printed, k ~ Var/Vbar.  1: the direction the paper's
                            prose describes, k ~ Vbar/Var (Var = 0 gives k_max).
-                           2: fixed k = k_base                                               */
+                           2: fixed k = k_base
+                           3: every visible key (needs k_max >= Lk): the dense fallback for
+                              short contexts, where the indexer costs more than it saves
+                              (Sec. 8); gsa_forward then runs no indexer and no selection
+                              (qI, kI, w may be NULL) and the layer is dense gated attention */
     float v_bar;        /* Vbar of Eq. 8: caller-owned running mean of score variance, > 0   */
     float sm_scale;     /* softmax scale of Eq. 11; <= 0 means 1/sqrt(d_h)                   */
     int32_t q_begin;    /* per-stage calls process query rows q_begin <= t < q_end of every  */

@@ -25,7 +25,8 @@
  *   - ties in I are broken towards the lower position; S_t is emitted ascending;
  *   - one S_t per query position, shared by all heads (I has no head index);
  *   - k_mode 0 is Eq. 8 as printed; k_mode 1 is the direction the prose describes
- *     (k_base * Vbar / Var; Var = 0 gives k_max); k_mode 2 is a fixed k = k_base.
+ *     (k_base * Vbar / Var; Var = 0 gives k_max); k_mode 2 is a fixed k = k_base;
+ *     k_mode 3 selects every visible key (the dense fallback for short contexts, Sec. 8).
  *
  * Pins (tests/test_oracle_pins.py): closed-form sigmoid values on one-hot inputs,
  * the reflection identity I(q)+I(-q)=sum_j w_j, the open range (0, sum w), two-valued
@@ -105,7 +106,8 @@ void gsa_oracle_budget(const gsa_oracle_params *p, const double *I_row, int n_t,
     double r;
     if (p->k_mode == 0)      r = (double)p->k_base * var / p->v_bar;
     else if (p->k_mode == 1) r = var > 0.0 ? (double)p->k_base * p->v_bar / var : INFINITY;
-    else                     r = (double)p->k_base;
+    else if (p->k_mode == 2) r = (double)p->k_base;
+    else                     r = INFINITY;            /* k_mode 3: every visible key (k_max >= Lk) */
 
     double f = floor(r);
     int32_t k;

@@ -50,9 +50,10 @@ int check_params(const gsa_params_t* p) {
     if (p->B < 1 || p->Lq < 1 || p->Lk < p->Lq || p->n_h < 1 || p->n_kv < 1) return GSA_ERR_INVALID_ARG;
     if (p->n_h % p->n_kv != 0) return GSA_ERR_INVALID_ARG;
     if (p->k_min < 1 || p->k_min > p->k_max || p->k_base < 1) return GSA_ERR_INVALID_ARG;
-    if (p->k_mode < 0 || p->k_mode > 2) return GSA_ERR_INVALID_ARG;
+    if (p->k_mode < 0 || p->k_mode > 3) return GSA_ERR_INVALID_ARG;
+    if (p->k_mode == 3 && p->k_max < p->Lk) return GSA_ERR_INVALID_ARG;
     if (p->act < 0 || p->act > 1) return GSA_ERR_INVALID_ARG;
-    if (p->k_mode != 2 && !(p->v_bar > 0.f)) return GSA_ERR_INVALID_ARG;
+    if (p->k_mode < 2 && !(p->v_bar > 0.f)) return GSA_ERR_INVALID_ARG;
     if (!one_of(p->d_h, {64, 128}) || !one_of(p->dI, {32, 64}) || !one_of(p->HI, {1, 2, 4, 8}))
         return GSA_ERR_UNSUPPORTED_SHAPE;
     if (!one_of(p->n_h / p->n_kv, {1, 2, 4, 8}) || !one_of(p->n_kv, {1, 2, 4, 8}))
@@ -380,7 +381,9 @@ static int forward_impl(const gsa_params_t* p, const void* Q, const void* K, con
                         AttnProgress* progress) {
     int rc = check_params(p);
     if (rc) return rc;
-    if (!Q || !K || !V || !qI || !kI || !w || !g1_logits || !out || slab_rows < 0) return GSA_ERR_INVALID_ARG;
+    const bool dense = p->k_mode == 3;                 // every visible key: no indexer, no selection
+    if (!Q || !K || !V || !g1_logits || !out || slab_rows < 0) return GSA_ERR_INVALID_ARG;
+    if (!dense && (!qI || !kI || !w)) return GSA_ERR_INVALID_ARG;
     const void* ptrs[] = {Q, K, V, qI, kI, w, g1_logits, g2_logits, out, idx_out, kt_out, var_out};
     for (const void* q : ptrs) if (q && !aligned16(q)) return GSA_ERR_INVALID_ARG;
     const WsPlan wp = plan_ws(*p, slab_rows);
@@ -398,7 +401,10 @@ static int forward_impl(const gsa_params_t* p, const void* Q, const void* K, con
     if (g_prof_ev[0]) cudaEventRecord(g_prof_ev[0], st);
 
     // Eq. 7, 8, 4 slab by slab: score rows live only inside the workspace
-    if (wp.slab_rows >= p->Lq) {
+    if (dense) {
+        RowRange all_rows{0, p->B, 0, p->Lq};
+        if ((e = launch_all_visible(*p, all_rows, idx, kt, var_out, il, st)) != cudaSuccess) return cuda_rc(e);
+    } else if (wp.slab_rows >= p->Lq) {
         const int nb_per = wp.slab_rows / p->Lq;
         for (int b0 = 0; b0 < p->B; b0 += nb_per) {
             RowRange rr{b0, (p->B - b0 < nb_per ? p->B - b0 : nb_per), 0, p->Lq};

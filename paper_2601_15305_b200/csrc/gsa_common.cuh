@@ -78,6 +78,10 @@ cudaError_t launch_indexer_kl(const gsa_params_t& p, RowRange rr, const __nv_bfl
 cudaError_t launch_vbar_update(const float* var, int64_t n, float momentum, float* v_bar, float* mean_var,
                                cudaStream_t st);
 
+// k_mode 3: S_t = every visible key (idx = 0, 1, ..., kt = number of visible keys, var = 0)
+cudaError_t launch_all_visible(const gsa_params_t& p, RowRange rr, int32_t* idx, int32_t* kt, float* var,
+                               IdxLayout il, cudaStream_t st);
+
 // Optional progress report of launch_sparse_attn: output rows become final range by range (a query
 // row is final once the key range holding its last visible key has been processed).  events[i], which
 // the caller created, is recorded when rows t_lo[i] <= t < t_hi[i] of every batch element are final.

@@ -197,7 +197,8 @@ __device__ __forceinline__ int budget_from_var(const SelectArgs& a, double var, 
     double r;
     if (a.k_mode == 0)      r = (double)a.k_base * var / (double)a.v_bar;
     else if (a.k_mode == 1) r = var > 0.0 ? (double)a.k_base * (double)a.v_bar / var : 1e300;
-    else                    r = (double)a.k_base;
+    else if (a.k_mode == 2) r = (double)a.k_base;
+    else                    r = 1e300;                          // k_mode 3: everything visible
     if (r_out) *r_out = r;
     const double fl = floor(r);
     if (!(fl < (double)a.k_max)) return a.k_max;
@@ -560,7 +561,30 @@ __global__ void __launch_bounds__(kSelThreads, 2) gsa_select_kernel(const Select
     for (int i = k + tid; i < a.k_max; i += kSelThreads) out_idx[i] = -1;
 }
 
+// k_mode 3 without scores: S_t is every visible key
+__global__ void __launch_bounds__(256) gsa_all_visible_kernel(RowRange rr, IdxLayout il, int32_t Lq, int32_t Lk,
+                                                              int32_t k_max, int32_t* __restrict__ idx,
+                                                              int32_t* __restrict__ kt, float* __restrict__ var) {
+    const int lr = blockIdx.x;
+    const int b = rr.b0 + lr / rr.R, t = rr.q_begin + lr % rr.R;
+    const int n = Lk - Lq + t + 1;
+    const int64_t row = il.row(b, t);
+    for (int i = threadIdx.x; i < k_max; i += blockDim.x) idx[row * k_max + i] = i < n ? i : -1;
+    if (threadIdx.x == 0) {
+        kt[row] = n;
+        if (var) var[row] = 0.f;
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_all_visible(const gsa_params_t& p, RowRange rr, int32_t* idx, int32_t* kt, float* var,
+                               IdxLayout il, cudaStream_t st) {
+    if (rr.rows() <= 0) return cudaSuccess;
+    gsa_all_visible_kernel<<<rr.rows(), 256, 0, st>>>(rr, il, p.Lq, p.Lk, p.k_max, idx, kt, var);
+    ++g_launches;
+    return cudaGetLastError();
+}
 
 cudaError_t launch_select(const gsa_params_t& p, RowRange rr, const float* scores,
                           int64_t row_stride, int32_t* idx, int32_t* kt, float* var, IdxLayout il,

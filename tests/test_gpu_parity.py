@@ -373,6 +373,38 @@ def test_forward_large_budget_equals_dense_gated_attention():
     U.check_out(out[0].float().cpu().numpy(), o["out"])
 
 
+def test_forward_dense_fallback_mode_needs_no_indexer_inputs():
+    """k_mode 3: every visible key, no indexer and no selection launches, indexer inputs may be absent."""
+    cfg = CONFIGS["tiny"].with_(name="dense", B=2, Lq=150, Lk=333, k_base=8, k_min=4, k_max=336)
+    x = make_inputs(cfg)
+    d = U.to_dev(x)
+    p = gsa.make_params(cfg, k_mode=3)
+    out = torch.full_like(d["Q"], float("nan"))
+    idx = torch.full((cfg.B, cfg.Lq, cfg.k_max), -7, dtype=torch.int32, device="cuda")
+    kt = torch.full((cfg.B, cfg.Lq), -7, dtype=torch.int32, device="cuda")
+    ws = torch.empty(gsa.gsa_workspace_bytes(p, 0), dtype=torch.uint8, device="cuda")
+    ws.fill_(0xFF)
+    n0 = gsa.gsa_launch_count()
+    gsa.gsa_forward(p, d["Q"], d["K"], d["V"], None, None, None, None, d["g1"], d["g2"], out, idx, kt, None, 0, ws)
+    torch.cuda.synchronize()
+    assert gsa.gsa_device_status(ws) == 0
+    n_vis = cfg.Lk - cfg.Lq + np.arange(cfg.Lq) + 1
+    assert (kt.cpu().numpy() == n_vis[None]).all()
+    for t in (0, 77, 149):
+        assert idx[1, t, : n_vis[t]].tolist() == list(range(n_vis[t])) and (idx[1, t, n_vis[t]:] == -1).all()
+    rows_t = np.tile(np.arange(cfg.Lq), cfg.B)
+    rows_b = np.repeat(np.arange(cfg.B), cfg.Lq)
+    o = oracle.forward(U.oracle_params(cfg, k_mode=3), **x, rows_t=rows_t, rows_b=rows_b)
+    U.check_out(out.float().cpu().numpy().reshape(cfg.B * cfg.Lq, cfg.n_h, cfg.d_h), o["out"])
+    # k_max below Lk cannot hold every key: refused before any launch
+    n1 = gsa.gsa_launch_count()
+    with pytest.raises(gsa.GsaError):
+        gsa.gsa_forward(gsa.make_params(cfg.with_(k_max=256), k_mode=3), d["Q"], d["K"], d["V"], None, None, None, None,
+                        d["g1"], d["g2"], out, None, kt, None, 0, ws)
+    assert gsa.gsa_launch_count() == n1
+    assert n1 - n0 <= 6          # all-visible, value gate, range cuts, attention, finalize
+
+
 def test_forward_batched_chunked_prefill():
     """B = 3, Lk > Lq, ragged sizes, k_max not a multiple of the 16-key tile."""
     cfg = CONFIGS["l8k"].with_(name="chunk", B=3, Lq=150, Lk=1111, k_base=300, k_min=50, k_max=777, seed=13,

@@ -361,6 +361,24 @@ def test_forward_large_budget_is_dense_gated_attention():
             np.testing.assert_allclose(r["out"][i, h], ref.numpy(), rtol=1e-12, atol=1e-15)
 
 
+def test_dense_fallback_mode_selects_every_visible_key():
+    """k_mode 3 (the short-context dense fallback, Sec. 8): whatever the scores, S_t is 0..t and the layer is
+    dense gated attention, checked against library softmax attention."""
+    cfg = CONFIGS["tiny"].with_(Lq=40, Lk=64, k_base=4, k_min=2, k_max=64)
+    x = make_inputs(cfg)
+    p = OracleParams.from_config(cfg, k_mode=3)
+    rows = [0, 7, 39]
+    r = oracle.forward(p, **x, rows_t=rows)
+    Vg = x["V"][0].double() * torch.sigmoid(x["g2"][0].double())
+    for i, t in enumerate(rows):
+        n = p.visible(t)
+        assert r["keff"][i] == n and r["idx"][i, :n].tolist() == list(range(n)) and (r["idx"][i, n:] == -1).all()
+        for h in range(cfg.n_h):
+            ref = _textbook_attention(x["Q"][0, t, h].double()[None], x["K"][0, :n, 0].double(), Vg[:n, 0],
+                                      1.0 / math.sqrt(cfg.d_h))[0] * torch.sigmoid(x["g1"][0, t, h].double())
+            np.testing.assert_allclose(r["out"][i, h], ref.numpy(), rtol=1e-12, atol=1e-15)
+
+
 def test_forward_is_composition_of_stages():
     cfg = CONFIGS["tiny"]
     x = make_inputs(cfg)
