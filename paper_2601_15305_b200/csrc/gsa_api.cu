@@ -210,9 +210,9 @@ static size_t attn_ws_bytes(const gsa_params_t& p, bool with_prepass) {
     return n;
 }
 
-// workspace of the backward call: [status][V' bf16][do bf16][lse2 fp32][delta fp32][inverted index sets]
+// workspace of the backward call: [status][V' bf16][do bf16][lse2 fp32][delta fp32][key-range scratch][inverted index sets]
 struct BwdPlan {
-    size_t vg_off, dos_off, lse_off, delta_off, inv_off, total;
+    size_t vg_off, dos_off, lse_off, delta_off, range_off, inv_off, total;
 };
 static BwdPlan plan_bwd_ws(const gsa_params_t& p, int32_t rows_per_batch) {
     BwdPlan w;
@@ -221,6 +221,7 @@ static BwdPlan plan_bwd_ws(const gsa_params_t& p, int32_t rows_per_batch) {
     w.dos_off = off;   off += align_up((size_t)p.B * p.Lq * p.n_h * p.d_h * 2, 256);
     w.lse_off = off;   off += align_up((size_t)p.B * p.Lq * p.n_h * 4, 256);
     w.delta_off = off; off += align_up((size_t)p.B * p.Lq * p.n_h * 4, 256);
+    w.range_off = off; off += attn_bwd_range_bytes(p);
     w.inv_off = off;   off += attn_bwd_invert_bytes(p, rows_per_batch);
     w.total = off;
     return w;
@@ -267,7 +268,7 @@ int gsa_sparse_gated_attn_bwd(const gsa_params_t* p, const void* Q, const void* 
     if (e == cudaSuccess)
         e = launch_sparse_attn_bwd(*p, rr, (const bf16*)Q, (const bf16*)K, Vg, (const bf16*)g1_logits,
                                    (const bf16*)out, (const bf16*)dout, idx, kt, il, (bf16*)dQ, (bf16*)dg1,
-                                   dOs, lse2, delta, pbar, st);
+                                   dOs, lse2, delta, pbar, wsb + wp.range_off, st);
     if (e == cudaSuccess)
         e = launch_sparse_attn_bwd_keys(*p, rr, (const bf16*)Q, dOs, (const bf16*)K, (const bf16*)V, Vg,
                                         (const bf16*)g2_logits, lse2, delta, idx, kt, il, wsb + wp.inv_off,

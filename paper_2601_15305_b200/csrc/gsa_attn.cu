@@ -607,6 +607,7 @@ size_t attn_scratch_bytes(const gsa_params_t& p) {
 }
 
 void set_attn_range_keys(int keys) { g_range_keys = keys >= 1024 ? keys : kRangeKeysDefault; }
+int attn_range_keys() { return g_range_keys; }
 
 cudaError_t launch_value_gate(const __nv_bfloat16* V, const __nv_bfloat16* g2, __nv_bfloat16* Vg,
                               int64_t n_elems, cudaStream_t st) {

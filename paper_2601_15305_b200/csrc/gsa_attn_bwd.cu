@@ -17,7 +17,11 @@
 //        S^T[key, head] = K . Q^T      dP^T[key, head] = V' . do^T            (A: tile via ldmatrix)
 //        dQ^T[d, head] += K^T . dS^T                                          (A: tile via ldmatrix.trans)
 //    It writes dQ and dg1 and leaves do (bf16), the softmax statistics and delta per (row, head) in the
-//    workspace for
+//    workspace for the other kernel.  When the keys span several L2-sized ranges (as in the forward pass:
+//    random 256-byte rows come much faster out of L2 than out of HBM) the work items are (key range, row,
+//    KV head), range-major, in two launches: the first leaves each range's softmax statistics, the second
+//    combines them, does the gradient sweep over its range's part of S_t (ascending index sets make that a
+//    contiguous sub-list) and adds its part of dQ into an fp32 array that a streaming pass rounds;
 //  * gsa_attn_bwd_keys.cu, key-major: dK and dV' are sums over every query that selected the key, so the
 //    index sets are first inverted (key -> list of query rows) and one warp per key then walks its list.
 #include "gsa_common.cuh"
@@ -44,6 +48,10 @@ struct BwdArgs {
     float* lse2;                  // workspace: log2-domain log-sum-exp of the scaled logits, [B, Lq, n_h]
     float* delta;                 // workspace: sum_d dout * out, [B, Lq, n_h]
     float* pbar;                  // optional output: mean over the heads of P on S_t, [B, R, k_max], pre-zeroed
+    float2* part_ml;              // key ranges: per range (max, sum) of the scaled logits, [n_ranges][B * Lq * n_h]
+    float* dq32;                  // key ranges: dQ summed over the ranges, [B, Lq, n_h, d_h], pre-zeroed
+    int32_t range_keys, n_ranges;
+    int64_t total_rows;           // B * Lq
     RowRange rr;
     IdxLayout il;
     int32_t Lq, Lk, n_h, n_kv, k_max;
@@ -60,7 +68,27 @@ __device__ __forceinline__ float ex2_approx(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-template <int DH, int G>
+// first position j of the ascending list S[0 .. n) with S[j] >= x; the whole warp calls it (32 probes a round)
+__device__ __forceinline__ int warp_lower_bound(const int32_t* __restrict__ S, int n, int x, int lane) {
+    int lo = 0, len = n;
+    while (len > 0) {
+        const int step = (len + 31) >> 5;
+        const int pos = lo + (lane + 1) * step - 1;
+        const bool lt = pos < lo + len && S[pos] < x;
+        const int c = __popc(__ballot_sync(0xFFFFFFFFu, lt));          // the first c probes are below x
+        const int end = lo + len;
+        lo += c * step;
+        len = min(step - 1, end - lo);
+        if (len < 0) len = 0;
+    }
+    return lo;
+}
+
+// MODE 0: one item = (row, KV head), both sweeps over the whole index set.
+// MODE 1: one item = (key range, row, KV head): statistics sweep over the range's part of S_t -> part_ml.
+// MODE 2: one item = (key range, row, KV head): statistics combined from part_ml, gradient sweep over the
+//         range's part, dQ added into dq32; the items of range 0 also write dg1, do, delta and lse2.
+template <int DH, int G, int MODE>
 __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(const BwdArgs a) {
     constexpr int ROW = (DH + 8) * 2;                  // bytes of a padded tile row (odd multiple of 16)
     constexpr int KTILE = 16 * ROW, QTILE = 8 * ROW;
@@ -75,17 +103,31 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int gid = lane >> 2, tig = lane & 3;
     const int64_t item = (int64_t)blockIdx.x * kBwdWarps + warp;
-    const int64_t n_items = (int64_t)a.rr.rows() * a.n_kv;
-    if (item >= n_items) return;                       // (no block-wide barrier below)
+    const int64_t per_range = (int64_t)a.rr.rows() * a.n_kv;
+    if (item >= per_range * (MODE == 0 ? 1 : a.n_ranges)) return;     // (no block-wide barrier below)
+    const int range = MODE == 0 ? 0 : (int)(item / per_range);       // range-major: the warps in flight share a range
+    const int64_t rem = item % per_range;
     // long rows first: late rows have the most keys
-    const int lr = a.rr.rows() - 1 - (int)(item / a.n_kv);
-    const int g = (int)(item % a.n_kv);
+    const int lr = a.rr.rows() - 1 - (int)(rem / a.n_kv);
+    const int g = (int)(rem % a.n_kv);
     const int b = a.rr.b0 + lr / a.rr.R;
     const int t = a.rr.q_begin + lr % a.rr.R;
     const int64_t qrow = (int64_t)b * a.Lq + t;
     const int64_t irow = a.il.row(b, t);
-    const int ke = a.kt[irow];
+    const int ke_all = a.kt[irow];
     const int32_t* __restrict__ S = a.idx + irow * a.k_max;
+    // this item's part of the index set: positions [j_lo, ke)
+    int j_lo = 0, ke = ke_all;
+    if (MODE != 0) {
+        j_lo = warp_lower_bound(S, ke_all, range * a.range_keys, lane);
+        ke = warp_lower_bound(S, ke_all, (range + 1) * a.range_keys, lane);
+    }
+    const bool writes_row = MODE == 0 || (MODE == 2 && range == 0);   // dg1, do, delta, lse2 are written once
+    if (MODE == 1 && j_lo >= ke) {                     // nothing of the row in this range
+        if (lane < G) a.part_ml[((size_t)range * a.total_rows + qrow) * a.n_h + g * G + lane] = make_float2(-INFINITY, 0.f);
+        return;
+    }
+    if (MODE == 2 && j_lo >= ke && !writes_row) return;
 
     unsigned char* const ws = bwd_smem + warp * WARP_SMEM;
     unsigned char* const q_tile = ws + STAGE;           // rows = the group's heads (rows >= G are zero)
@@ -105,14 +147,20 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
             const int64_t at = (qrow * a.n_h + (g * G + hl)) * DH + lane * EPL;
 #pragma unroll
             for (int e = 0; e < EPL; ++e) {
-                const float dy = __bfloat162float(a.dout[at + e]);
-                const float y = __bfloat162float(a.out[at + e]);
-                const float sg = 1.0f / (1.0f + __expf(-__bfloat162float(a.g1[at + e])));
                 qd[e] = a.Q[at + e];
-                dd[e] = __float2bfloat16(dy * sg);
-                a.dOs[at + e] = dd[e];
-                a.dg1[at + e] = __float2bfloat16(dy * y * (1.0f - sg));
-                part = fmaf(dy, y, part);
+                if (MODE != 1) {                       // (the statistics launch needs Q only)
+                    const float dy = __bfloat162float(a.dout[at + e]);
+                    const float y = __bfloat162float(a.out[at + e]);
+                    const float sg = 1.0f / (1.0f + __expf(-__bfloat162float(a.g1[at + e])));
+                    dd[e] = __float2bfloat16(dy * sg);
+                    if (writes_row) {
+                        a.dOs[at + e] = dd[e];
+                        a.dg1[at + e] = __float2bfloat16(dy * y * (1.0f - sg));
+                    }
+                    part = fmaf(dy, y, part);
+                } else {
+                    dd[e] = __float2bfloat16(0.f);
+                }
             }
         } else {
 #pragma unroll
@@ -122,7 +170,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
         for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
         if (lane == 0) {
             s_delta[hl] = part;
-            if (hl < G) a.delta[qrow * a.n_h + g * G + hl] = part;
+            if (hl < G && writes_row) a.delta[qrow * a.n_h + g * G + hl] = part;
         }
     }
     __syncwarp();
@@ -176,8 +224,9 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
         }
         cp_async_commit();                                // (possibly empty: keeps the group count uniform)
     };
-    fetch(0, 0, false);
-    for (int j0 = 0, stage = 0; j0 < ke; j0 += 16, stage ^= 1) {
+    if (MODE != 2) {
+    fetch(j_lo, 0, false);
+    for (int j0 = j_lo, stage = 0; j0 < ke; j0 += 16, stage ^= 1) {
         fetch(j0 + 16, stage ^ 1, false);
         cp_async_wait<1>();
         __syncwarp();
@@ -196,7 +245,6 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
         __syncwarp();                                     // this stage is refilled by the next iteration
     }
     cp_async_wait<0>();
-    float lse2[2];
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
 #pragma unroll
@@ -208,16 +256,42 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
                 l_run[e] = l_run[e] * ex2_approx(m_run[e] - m_new) + l_o * ex2_approx(m_o - m_new);
             m_run[e] = m_new;
         }
-        lse2[e] = m_run[e] + log2f(l_run[e]);
-        if (gid == 0 && 2 * tig + e < G) a.lse2[qrow * a.n_h + g * G + 2 * tig + e] = lse2[e];
     }
+    }
+    if (MODE == 1) {                                   // this range's statistics; the gradient launch combines them
+#pragma unroll
+        for (int e = 0; e < 2; ++e)
+            if (gid == 0 && 2 * tig + e < G)
+                a.part_ml[((size_t)range * a.total_rows + qrow) * a.n_h + g * G + 2 * tig + e] = make_float2(m_run[e], l_run[e]);
+        return;
+    }
+    if (MODE == 2) {
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const int h = g * G + min(2 * tig + e, G - 1);    // (columns >= G are padding: any finite value will do)
+            for (int r = 0; r < a.n_ranges; ++r) {
+                const float2 ml = a.part_ml[((size_t)r * a.total_rows + qrow) * a.n_h + h];
+                const float m_new = fmaxf(m_run[e], ml.x);
+                if (m_new > -INFINITY)
+                    l_run[e] = l_run[e] * ex2_approx(m_run[e] - m_new) + ml.y * ex2_approx(ml.x - m_new);
+                m_run[e] = m_new;
+            }
+        }
+    }
+    float lse2[2];
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+        lse2[e] = m_run[e] + log2f(l_run[e]);
+        if (writes_row && gid == 0 && 2 * tig + e < G) a.lse2[qrow * a.n_h + g * G + 2 * tig + e] = lse2[e];
+    }
+    if (MODE == 2 && j_lo >= ke) return;               // (an item of range 0 that only had the row's values to write)
 
     // ---- sweep 2: gradients ---------------------------------------------------------------------------
     float dq[KS][4];
 #pragma unroll
     for (int mt = 0; mt < KS; ++mt) dq[mt][0] = dq[mt][1] = dq[mt][2] = dq[mt][3] = 0.f;
-    fetch(0, 0, true);
-    for (int j0 = 0, stage = 0; j0 < ke; j0 += 16, stage ^= 1) {
+    fetch(j_lo, 0, true);
+    for (int j0 = j_lo, stage = 0; j0 < ke; j0 += 16, stage ^= 1) {
         fetch(j0 + 16, stage ^ 1, true);
         cp_async_wait<1>();
         __syncwarp();
@@ -271,34 +345,88 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
     for (int e = 0; e < 2; ++e) {
         const int hl = 2 * tig + e;
         if (hl < G) {
-            __nv_bfloat16* const dst = a.dQ + (qrow * a.n_h + (g * G + hl)) * DH;
+            if (MODE == 2) {                           // this range's part: eight lanes fill one 32-byte sector
+                float* const dst = a.dq32 + (qrow * a.n_h + (g * G + hl)) * DH;
 #pragma unroll
-            for (int mt = 0; mt < KS; ++mt) {
-                dst[mt * 16 + gid] = __float2bfloat16(dq[mt][e] * a.scale);
-                dst[mt * 16 + gid + 8] = __float2bfloat16(dq[mt][2 + e] * a.scale);
+                for (int mt = 0; mt < KS; ++mt) {
+                    atomicAdd(dst + mt * 16 + gid, dq[mt][e] * a.scale);
+                    atomicAdd(dst + mt * 16 + gid + 8, dq[mt][2 + e] * a.scale);
+                }
+            } else {
+                __nv_bfloat16* const dst = a.dQ + (qrow * a.n_h + (g * G + hl)) * DH;
+#pragma unroll
+                for (int mt = 0; mt < KS; ++mt) {
+                    dst[mt * 16 + gid] = __float2bfloat16(dq[mt][e] * a.scale);
+                    dst[mt * 16 + gid + 8] = __float2bfloat16(dq[mt][2 + e] * a.scale);
+                }
             }
         }
     }
 }
 
-template <int DH, int G>
-cudaError_t launch_bwd_t(const BwdArgs& a, cudaStream_t st) {
+// dQ rows of the range from the fp32 sums
+__global__ void __launch_bounds__(256) gsa_bwd_dq_finish_kernel(const float* __restrict__ dq32,
+                                                                __nv_bfloat16* __restrict__ dQ, RowRange rr,
+                                                                int32_t Lq, int64_t row_elems) {
+    const int lr = blockIdx.x;
+    const int64_t qrow = (int64_t)(rr.b0 + lr / rr.R) * Lq + rr.q_begin + lr % rr.R;
+    for (int64_t i = threadIdx.x * 4; i < row_elems; i += blockDim.x * 4) {
+        const float4 v = *reinterpret_cast<const float4*>(dq32 + qrow * row_elems + i);
+        __align__(8) __nv_bfloat16 o[4] = {__float2bfloat16(v.x), __float2bfloat16(v.y), __float2bfloat16(v.z),
+                                           __float2bfloat16(v.w)};
+        *reinterpret_cast<uint2*>(dQ + qrow * row_elems + i) = *reinterpret_cast<const uint2*>(o);
+    }
+}
+
+template <int DH, int G, int MODE>
+cudaError_t launch_bwd_mode(const BwdArgs& a, cudaStream_t st) {
     constexpr int ROW = (DH + 8) * 2;
     constexpr int WARP_SMEM = 4 * 16 * ROW;
     const int smem = kBwdWarps * WARP_SMEM;
+    auto kern = gsa_sparse_attn_bwd_kernel<DH, G, MODE>;
     // (set on every call: the attribute belongs to the current device)
-    {
-        cudaError_t e = cudaFuncSetAttribute(gsa_sparse_attn_bwd_kernel<DH, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e != cudaSuccess) return e;
-    }
-    const int64_t items = (int64_t)a.rr.rows() * a.n_kv;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    const int64_t items = (int64_t)a.rr.rows() * a.n_kv * (MODE == 0 ? 1 : a.n_ranges);
     const int64_t ctas = (items + kBwdWarps - 1) / kBwdWarps;
-    gsa_sparse_attn_bwd_kernel<DH, G><<<(unsigned)ctas, kBwdWarps * 32, smem, st>>>(a);
+    kern<<<(unsigned)ctas, kBwdWarps * 32, smem, st>>>(a);
     ++g_launches;
     return cudaGetLastError();
 }
 
+template <int DH, int G>
+cudaError_t launch_bwd_t(const BwdArgs& a, cudaStream_t st) {
+    if (a.n_ranges <= 1) return launch_bwd_mode<DH, G, 0>(a, st);
+    cudaError_t e = cudaMemsetAsync(a.dq32, 0, (size_t)a.total_rows * a.n_h * DH * 4, st);
+    if (e == cudaSuccess) e = launch_bwd_mode<DH, G, 1>(a, st);
+    if (e == cudaSuccess) e = launch_bwd_mode<DH, G, 2>(a, st);
+    if (e != cudaSuccess) return e;
+    gsa_bwd_dq_finish_kernel<<<a.rr.rows(), 256, 0, st>>>(a.dq32, a.dQ, a.rr, a.Lq, (int64_t)a.n_h * DH);
+    ++g_launches;
+    return cudaGetLastError();
+}
+
+// key ranges of the query-major half: the forward pass's range size; one range when the keys fit one
+struct BwdRanges { int range_keys, n_ranges; };
+BwdRanges plan_bwd_ranges(const gsa_params_t& p) {
+    BwdRanges r;
+    r.range_keys = attn_range_keys();
+    r.n_ranges = (p.Lk + r.range_keys - 1) / r.range_keys;
+    if (r.n_ranges > 48) {
+        r.range_keys = ((p.Lk + 47) / 48 + 1023) / 1024 * 1024;
+        r.n_ranges = (p.Lk + r.range_keys - 1) / r.range_keys;
+    }
+    return r;
+}
+
 }  // namespace
+
+size_t attn_bwd_range_bytes(const gsa_params_t& p) {
+    const BwdRanges br = plan_bwd_ranges(p);
+    if (br.n_ranges <= 1) return 0;
+    const size_t rows = (size_t)p.B * p.Lq;
+    return ((size_t)br.n_ranges * rows * p.n_h * 8 + 255) / 256 * 256 + (rows * p.n_h * p.d_h * 4 + 255) / 256 * 256;
+}
 
 bool attn_bwd_supported(const gsa_params_t& p) {
     const int G = p.n_h / p.n_kv;
@@ -309,9 +437,14 @@ cudaError_t launch_sparse_attn_bwd(const gsa_params_t& p, RowRange rr, const __n
                                    const __nv_bfloat16* K, const __nv_bfloat16* Vg, const __nv_bfloat16* g1,
                                    const __nv_bfloat16* out, const __nv_bfloat16* dout, const int32_t* idx,
                                    const int32_t* kt, IdxLayout il, __nv_bfloat16* dQ, __nv_bfloat16* dg1,
-                                   __nv_bfloat16* dOs, float* lse2, float* delta, float* pbar, cudaStream_t st) {
+                                   __nv_bfloat16* dOs, float* lse2, float* delta, float* pbar, void* range_ws,
+                                   cudaStream_t st) {
     if (rr.rows() <= 0) return cudaSuccess;
     BwdArgs a;
+    const BwdRanges br = plan_bwd_ranges(p);
+    a.range_keys = br.range_keys; a.n_ranges = br.n_ranges; a.total_rows = (int64_t)p.B * p.Lq;
+    a.part_ml = (float2*)range_ws;
+    a.dq32 = (float*)((char*)range_ws + ((size_t)br.n_ranges * a.total_rows * p.n_h * 8 + 255) / 256 * 256);
     a.Q = Q; a.K = K; a.Vg = Vg; a.g1 = g1; a.out = out; a.dout = dout; a.idx = idx; a.kt = kt;
     a.dQ = dQ; a.dg1 = dg1; a.dOs = dOs; a.lse2 = lse2; a.delta = delta; a.pbar = pbar; a.rr = rr; a.il = il;
     a.Lq = p.Lq; a.Lk = p.Lk; a.n_h = p.n_h; a.n_kv = p.n_kv; a.k_max = p.k_max;

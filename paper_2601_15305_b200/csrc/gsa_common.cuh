@@ -55,7 +55,9 @@ cudaError_t launch_sparse_attn_bwd(const gsa_params_t& p, RowRange rr, const __n
                                    const __nv_bfloat16* K, const __nv_bfloat16* Vg, const __nv_bfloat16* g1,
                                    const __nv_bfloat16* out, const __nv_bfloat16* dout, const int32_t* idx,
                                    const int32_t* kt, IdxLayout il, __nv_bfloat16* dQ, __nv_bfloat16* dg1,
-                                   __nv_bfloat16* dOs, float* lse2, float* delta, float* pbar, cudaStream_t st);
+                                   __nv_bfloat16* dOs, float* lse2, float* delta, float* pbar, void* range_ws,
+                                   cudaStream_t st);
+size_t attn_bwd_range_bytes(const gsa_params_t& p);      // scratch of the query-major half when Lk spans several key ranges
 size_t attn_bwd_invert_bytes(const gsa_params_t& p, int32_t rows_per_batch);
 cudaError_t launch_sparse_attn_bwd_keys(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* Q,
                                         const __nv_bfloat16* dOs, const __nv_bfloat16* K, const __nv_bfloat16* V,
@@ -103,6 +105,7 @@ cudaError_t launch_sparse_attn(const gsa_params_t& p, RowRange rr, const __nv_bf
 size_t attn_scratch_bytes(const gsa_params_t& p);
 // keys per L2-resident key range of the sparse-attention gather (tuning knob)
 void set_attn_range_keys(int keys);
+int attn_range_keys();
 
 // device address, on the current device, of the library's built-in scratch array (status word at
 // its start, then the gated values of the allocation-free entry point)

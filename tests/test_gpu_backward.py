@@ -40,7 +40,7 @@ def _index_sets(cfg, q0, q1, seed, k_lo=None, k_hi=None):
     return idx, kt
 
 
-def _run_bwd(cfg, d, idx, kt, dout, q0, q1, **over):
+def _run_bwd(cfg, d, idx, kt, dout, q0, q1, key_range=16384, **over):
     p = gsa.make_params(cfg, q_begin=q0, q_end=q1, **over)
     out = U.run_attn(cfg, d, idx, kt, q_begin=q0, q_end=q1, **over)
     nan = float("nan")
@@ -57,7 +57,9 @@ def _run_bwd(cfg, d, idx, kt, dout, q0, q1, **over):
     # value gate, query-major kernel, count + 3 scan steps, one fill per range of 8192 query rows, key-major
     # kernel, and with several ranges the post-pass
     n_ranges = (q1 - q0 + 8191) // 8192
-    assert gsa.gsa_launch_count() - n0 == 7 + n_ranges + (1 if n_ranges > 1 else 0)
+    key_ranges = (cfg.Lk + key_range - 1) // key_range          # of the query-major half (as in the forward pass)
+    extra = 2 if key_ranges > 1 else 0                          # statistics launch + dQ rounding pass
+    assert gsa.gsa_launch_count() - n0 == 7 + n_ranges + (1 if n_ranges > 1 else 0) + extra
     return dict(dQ=dQ, dg1=dg1, dK=dK, dV=dV, dg2=dg2, pbar=pbar)
 
 
@@ -146,6 +148,25 @@ def test_attn_backward_head_layouts(n_h, n_kv, d_h):
     dout = (torch.randn(d["Q"].shape, generator=torch.Generator().manual_seed(62)) * 0.5).to(torch.bfloat16)
     got = _run_bwd(cfg, d, idx.cuda(), kt.cuda(), dout.cuda(), 0, cfg.Lq)
     _compare(cfg, x, got, idx, kt, dout, 0, cfg.Lq)
+
+
+def test_attn_backward_several_key_ranges():
+    """Keys spanning several L2 ranges (forced small here): the query-major half runs per (range, row, KV head),
+    combines the ranges' softmax statistics and sums their parts of dQ.  Rows whose visible keys end inside a
+    range, rows with nothing in some range, a batch of two."""
+    cfg = CONFIGS["l8k"].with_(name="bwd_kr", B=2, Lq=300, Lk=3500, k_base=200, k_min=9, k_max=333, seed=44)
+    x = make_inputs(cfg)
+    d = U.to_dev(x)
+    q0, q1 = 100, 300
+    idx, kt = _index_sets(cfg, q0, q1, seed=45)
+    idx[0, 5, : int(kt[0, 5])] = torch.arange(int(kt[0, 5]), dtype=torch.int32) + 1030     # one row inside one range
+    dout = (torch.randn(d["Q"].shape, generator=torch.Generator().manual_seed(46)) * 0.25).to(torch.bfloat16)
+    gsa.gsa_debug_set_attn_range_keys(1024)
+    try:
+        got = _run_bwd(cfg, d, idx.cuda(), kt.cuda(), dout.cuda(), q0, q1, key_range=1024)
+    finally:
+        gsa.gsa_debug_set_attn_range_keys(0)
+    _compare(cfg, x, got, idx, kt, dout, q0, q1)
 
 
 def test_attn_backward_several_query_ranges():
