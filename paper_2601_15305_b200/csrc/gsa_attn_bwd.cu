@@ -203,14 +203,20 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
     };
     // S^T (or dP^T) of the staged tile: rows gid, gid + 8 = keys, columns 2 tig, 2 tig + 1 = heads
     auto tile_times = [&](uint32_t tile_s32, const uint32_t (&bf)[2 * KS], float (&acc)[4]) {
+        // two accumulators (even / odd k-steps): half the length of the dependent MMA chain
+        float acc2[4] = {0.f, 0.f, 0.f, 0.f};
         acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
         const uint32_t addr = tile_s32 + (lane & 15) * ROW + (lane >> 4) * 16;
 #pragma unroll
-        for (int ks = 0; ks < KS; ++ks) {
-            uint32_t a0, a1, a2, a3;
+        for (int ks = 0; ks < KS; ks += 2) {
+            uint32_t a0, a1, a2, a3, c0, c1, c2r, c3;
             ldmatrix_x4(a0, a1, a2, a3, addr + ks * 32);
+            ldmatrix_x4(c0, c1, c2r, c3, addr + (ks + 1) * 32);
             mma_bf16_16816(acc, a0, a1, a2, a3, bf[2 * ks], bf[2 * ks + 1]);
+            mma_bf16_16816(acc2, c0, c1, c2r, c3, bf[2 * ks + 2], bf[2 * ks + 3]);
         }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[i] += acc2[i];
     };
 
     // ---- sweep 1: softmax statistics per head (log2 domain) ----------------------------------------

@@ -235,14 +235,20 @@ __global__ void __launch_bounds__(kKeyWarps * 32) gsa_sparse_attn_bwd_keys_kerne
     __syncwarp();                                      // stage 1 is free for tiles from here on
 
     auto tile_times = [&](uint32_t tile_s32, const uint32_t (&bf)[2 * KS], float (&acc)[4]) {
+        // two accumulators (even / odd k-steps): half the length of the dependent MMA chain
+        float acc2[4] = {0.f, 0.f, 0.f, 0.f};
         acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
         const uint32_t addr = tile_s32 + (lane & 15) * ROW + (lane >> 4) * 16;
 #pragma unroll
-        for (int ks = 0; ks < KS; ++ks) {
-            uint32_t a0, a1, a2, a3;
+        for (int ks = 0; ks < KS; ks += 2) {
+            uint32_t a0, a1, a2, a3, c0, c1, c2r, c3;
             ldmatrix_x4(a0, a1, a2, a3, addr + ks * 32);
+            ldmatrix_x4(c0, c1, c2r, c3, addr + (ks + 1) * 32);
             mma_bf16_16816(acc, a0, a1, a2, a3, bf[2 * ks], bf[2 * ks + 1]);
+            mma_bf16_16816(acc2, c0, c1, c2r, c3, bf[2 * ks + 2], bf[2 * ks + 3]);
         }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[i] += acc2[i];
     };
 
     const float c2 = a.scale * kLog2eK;
