@@ -142,6 +142,8 @@ int gsa_output_projection(const gsa_params_t *p, int32_t d_model, const void *at
  *          accumulated in fp32 (in an order that depends on scheduling) and rounded once
  *   pbar   [B, R, k_max] fp32 or NULL: the target of the indexer's loss (what gsa_attn_probs_mean writes,
  *          see below), which this call's second sweep has at hand: one call instead of two
+ *   lse    [B, Lq, n_h] fp32 or NULL: what gsa_sparse_gated_attn_fwd_lse saved for the same inputs; with it
+ *          the sweep over S_t that recomputes the softmax statistics is skipped
  *   ws     workspace of gsa_attn_bwd_workspace_bytes(p) bytes (depends on q_begin / q_end): status word,
  *          V', dout * sigmoid(g1), softmax statistics, and the index sets inverted (key -> query rows)
  * Returns GSA_ERR_WORKSPACE if ws is too small; nothing is launched on an argument error.
@@ -150,8 +152,8 @@ int gsa_attn_bwd_workspace_bytes(const gsa_params_t *p, size_t *bytes);
 int gsa_sparse_gated_attn_bwd(const gsa_params_t *p, const void *Q, const void *K, const void *V,
                               const void *g1_logits, const void *g2_logits, const int32_t *idx,
                               const int32_t *kt, const void *out, const void *dout, void *dQ, void *dK,
-                              void *dV, void *dg1, void *dg2, float *pbar, void *ws, size_t ws_bytes,
-                              void *stream);
+                              void *dV, void *dg1, void *dg2, float *pbar, const float *lse, void *ws,
+                              size_t ws_bytes, void *stream);
 
 /*
  * The indexer's sparse-phase loss (Sec. 5.1, Eq. 14) for rows [q_begin, q_end):
@@ -234,6 +236,16 @@ int gsa_sparse_gated_attn_fwd(const gsa_params_t *p, const void *Q, const void *
                               const void *g1_logits, const void *g2_logits, const int32_t *idx,
                               const int32_t *kt, void *out, void *ws, size_t ws_bytes,
                               void *stream);
+
+/*
+ * The same call for training: also saves the softmax statistics the backward pass needs,
+ *     lse[b, t, h] = log sum_{j in S_t} exp(sm_scale * q_h . k_j)      (natural logarithm, fp32),
+ * for rows [q_begin, q_end) of [B, Lq, n_h]; gsa_sparse_gated_attn_bwd takes them back.
+ */
+int gsa_sparse_gated_attn_fwd_lse(const gsa_params_t *p, const void *Q, const void *K, const void *V,
+                                  const void *g1_logits, const void *g2_logits, const int32_t *idx,
+                                  const int32_t *kt, void *out, float *lse, void *ws, size_t ws_bytes,
+                                  void *stream);
 
 /*
  * gsa_sparse_gated_attn_fwd for callers that cannot allocate device memory.  (The paper has no

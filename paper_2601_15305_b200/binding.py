@@ -23,7 +23,7 @@ EXPORTS = (
     "gsa_sparse_gated_attn_fwd_static", "gsa_attn_workspace_bytes", "gsa_debug_set_attn_range_keys",
     "gsa_select_fallback_rows", "gsa_project", "gsa_project_columns", "gsa_output_projection",
     "gsa_attn_bwd_workspace_bytes", "gsa_sparse_gated_attn_bwd", "gsa_vbar_update",
-    "gsa_attn_probs_mean", "gsa_indexer_kl_workspace_bytes", "gsa_indexer_kl_bwd",
+    "gsa_attn_probs_mean", "gsa_indexer_kl_workspace_bytes", "gsa_indexer_kl_bwd", "gsa_sparse_gated_attn_fwd_lse",
 )
 
 STATIC_SCRATCH_BYTES = 32 << 20     # GSA_STATIC_SCRATCH_BYTES of include/gsa.h
@@ -159,11 +159,11 @@ def gsa_attn_bwd_workspace_bytes(p) -> int:
 
 
 def gsa_sparse_gated_attn_bwd(p, Q, K, V, g1, g2, idx, kt, out, dout, dQ, dK, dV, dg1, dg2, ws, stream=None,
-                              pbar=None) -> None:
+                              pbar=None, lse=None) -> None:
     _check(lib().gsa_sparse_gated_attn_bwd(ctypes.byref(p), _dp(Q, BF16), _dp(K, BF16), _dp(V, BF16), _dp(g1, BF16),
                                            _dp(g2, BF16), _dp(idx, I32), _dp(kt, I32), _dp(out, BF16),
                                            _dp(dout, BF16), _dp(dQ, BF16), _dp(dK, BF16), _dp(dV, BF16),
-                                           _dp(dg1, BF16), _dp(dg2, BF16), _dp(pbar, F32), _dp(ws),
+                                           _dp(dg1, BF16), _dp(dg2, BF16), _dp(pbar, F32), _dp(lse, F32), _dp(ws),
                                            ctypes.c_size_t(ws.numel() * ws.element_size()), _stream(stream)),
            "gsa_sparse_gated_attn_bwd")
 
@@ -192,6 +192,14 @@ def gsa_vbar_update(var, momentum: float, v_bar, mean_var=None, stream=None) -> 
     """v_bar (one fp32 on the device) <- momentum * v_bar + (1 - momentum) * mean(var)."""
     _check(lib().gsa_vbar_update(_dp(var, F32), ctypes.c_int64(var.numel()), ctypes.c_float(momentum),
                                  _dp(v_bar, F32), _dp(mean_var, F32), _stream(stream)), "gsa_vbar_update")
+
+
+def gsa_sparse_gated_attn_fwd_lse(p, Q, K, V, g1, g2, idx, kt, out, lse, ws, stream=None) -> None:
+    _check(lib().gsa_sparse_gated_attn_fwd_lse(ctypes.byref(p), _dp(Q, BF16), _dp(K, BF16), _dp(V, BF16),
+                                               _dp(g1, BF16), _dp(g2, BF16), _dp(idx, I32), _dp(kt, I32),
+                                               _dp(out, BF16), _dp(lse, F32), _dp(ws),
+                                               ctypes.c_size_t(ws.numel() * ws.element_size()), _stream(stream)),
+           "gsa_sparse_gated_attn_fwd_lse")
 
 
 def gsa_sparse_gated_attn_fwd_static(p, Q, K, V, g1, g2, idx, kt, out, stream=None) -> None:

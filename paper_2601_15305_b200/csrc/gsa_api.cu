@@ -240,8 +240,8 @@ int gsa_attn_bwd_workspace_bytes(const gsa_params_t* p, size_t* bytes) {
 int gsa_sparse_gated_attn_bwd(const gsa_params_t* p, const void* Q, const void* K, const void* V,
                               const void* g1_logits, const void* g2_logits, const int32_t* idx,
                               const int32_t* kt, const void* out, const void* dout, void* dQ, void* dK,
-                              void* dV, void* dg1, void* dg2, float* pbar, void* ws, size_t ws_bytes,
-                              void* stream) {
+                              void* dV, void* dg1, void* dg2, float* pbar, const float* lse, void* ws,
+                              size_t ws_bytes, void* stream) {
     int rc = check_params(p);
     if (rc) return rc;
     RowRange rr;
@@ -251,7 +251,7 @@ int gsa_sparse_gated_attn_bwd(const gsa_params_t* p, const void* Q, const void* 
         return GSA_ERR_UNSUPPORTED_SHAPE;
     const void* ptrs[] = {Q, K, V, g1_logits, g2_logits, idx, out, dout, dQ, dK, dV, dg1, dg2};
     for (const void* q : ptrs) if (!q || !aligned16(q)) return GSA_ERR_INVALID_ARG;
-    if (!kt || (pbar && !aligned16(pbar))) return GSA_ERR_INVALID_ARG;
+    if (!kt || (pbar && !aligned16(pbar)) || (lse && !aligned16(lse))) return GSA_ERR_INVALID_ARG;
     const BwdPlan wp = plan_bwd_ws(*p, rr.R);
     if (!ws || !aligned16(ws) || ws_bytes < wp.total) return GSA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
@@ -268,7 +268,7 @@ int gsa_sparse_gated_attn_bwd(const gsa_params_t* p, const void* Q, const void* 
     if (e == cudaSuccess)
         e = launch_sparse_attn_bwd(*p, rr, (const bf16*)Q, (const bf16*)K, Vg, (const bf16*)g1_logits,
                                    (const bf16*)out, (const bf16*)dout, idx, kt, il, (bf16*)dQ, (bf16*)dg1,
-                                   dOs, lse2, delta, pbar, wsb + wp.range_off, st);
+                                   dOs, lse2, delta, pbar, lse, wsb + wp.range_off, st);
     if (e == cudaSuccess)
         e = launch_sparse_attn_bwd_keys(*p, rr, (const bf16*)Q, dOs, (const bf16*)K, (const bf16*)V, Vg,
                                         (const bf16*)g2_logits, lse2, delta, idx, kt, il, wsb + wp.inv_off,
@@ -336,9 +336,9 @@ int gsa_attn_workspace_bytes(const gsa_params_t* p, int32_t with_value_gate_prep
     return GSA_OK;
 }
 
-int gsa_sparse_gated_attn_fwd(const gsa_params_t* p, const void* Q, const void* K, const void* V,
-                              const void* g1_logits, const void* g2_logits, const int32_t* idx,
-                              const int32_t* kt, void* out, void* ws, size_t ws_bytes, void* stream) {
+static int attn_fwd_impl(const gsa_params_t* p, const void* Q, const void* K, const void* V,
+                         const void* g1_logits, const void* g2_logits, const int32_t* idx, const int32_t* kt,
+                         void* out, float* lse, void* ws, size_t ws_bytes, void* stream) {
     int rc = check_params(p);
     if (rc) return rc;
     RowRange rr;
@@ -369,7 +369,21 @@ int gsa_sparse_gated_attn_fwd(const gsa_params_t* p, const void* Q, const void* 
         }
     }
     return cuda_rc(launch_sparse_attn(*p, rr, (const bf16*)Q, (const bf16*)K, Vuse, (const bf16*)g1_logits,
-                                      g2use, idx, kt, il, (bf16*)out, scratch, st));
+                                      g2use, idx, kt, il, (bf16*)out, scratch, st, nullptr, lse));
+}
+
+int gsa_sparse_gated_attn_fwd(const gsa_params_t* p, const void* Q, const void* K, const void* V,
+                              const void* g1_logits, const void* g2_logits, const int32_t* idx,
+                              const int32_t* kt, void* out, void* ws, size_t ws_bytes, void* stream) {
+    return attn_fwd_impl(p, Q, K, V, g1_logits, g2_logits, idx, kt, out, nullptr, ws, ws_bytes, stream);
+}
+
+int gsa_sparse_gated_attn_fwd_lse(const gsa_params_t* p, const void* Q, const void* K, const void* V,
+                                  const void* g1_logits, const void* g2_logits, const int32_t* idx,
+                                  const int32_t* kt, void* out, float* lse, void* ws, size_t ws_bytes,
+                                  void* stream) {
+    if (!lse || !aligned16(lse)) return GSA_ERR_INVALID_ARG;
+    return attn_fwd_impl(p, Q, K, V, g1_logits, g2_logits, idx, kt, out, lse, ws, ws_bytes, stream);
 }
 
 // The whole path.  `kv_ready` (may be NULL) is an event the stream waits for before anything reads

@@ -63,6 +63,7 @@ struct AttnArgs {
     int32_t max_parts;        // mode 1: segments (= state slots) per index set
     int32_t range, n_cuts;
     float scale_log2;         // sm_scale * log2(e)
+    float* lse;               // optional output [B, Lq, n_h]: natural log of sum_j exp(sm_scale * q.k_j) over S_t
 };
 
 struct RowId { int32_t b, t; int64_t irow; };
@@ -386,7 +387,8 @@ template <int DH, int G>
 __global__ void __launch_bounds__(1024) gsa_attn_finalize_kernel(const float* __restrict__ state, const int32_t* __restrict__ kt,
                                                                 const __nv_bfloat16* __restrict__ g1, __nv_bfloat16* __restrict__ out,
                                                                 RowRange rr, IdxLayout il, int64_t idx_rows, int Lq, int n_h,
-                                                                int n_kv, int k_max, int mode, int max_parts) {
+                                                                int n_kv, int k_max, int mode, int max_parts,
+                                                                float* __restrict__ lse) {
     constexpr int STATE_F = G * (DH + 2);
     const int rows = rr.rows();
     const int lr0 = blockIdx.x * kFinRows;
@@ -418,6 +420,11 @@ __global__ void __launch_bounds__(1024) gsa_attn_finalize_kernel(const float* __
                 for (int e = 0; e < G; ++e) {
                     const float v = (keff[q] > 0 && l[q][e] > 0.f) ? o[q][e] / l[q][e] * fast_sigmoid(gl[q][e]) : 0.f;
                     out[at0[q] + (size_t)e * DH] = __float2bfloat16_rn(v);
+                    if (lse && d == 0) {               // the running maximum sits in front of the sums (log2 domain)
+                        const RowId r = row_of(rr, il, lr0 + q);
+                        const float m = state[((int64_t)r.irow * n_kv + g) * STATE_F + G * DH + e];
+                        lse[((size_t)r.b * Lq + r.t) * n_h + g * G + e] = (m + log2f(l[q][e])) * 0.6931471805599453f;
+                    }
                 }
             }
         } else {
@@ -450,6 +457,8 @@ __global__ void __launch_bounds__(1024) gsa_attn_finalize_kernel(const float* __
                     const size_t at = (((size_t)r.b * Lq + r.t) * n_h + g * G + e) * DH + d;
                     const float v = den[e] > 0.f ? acc[e] / den[e] * fast_sigmoid(__bfloat162float(g1[at])) : 0.f;
                     out[at] = __float2bfloat16_rn(v);
+                    if (lse && d == 0)
+                        lse[((size_t)r.b * Lq + r.t) * n_h + g * G + e] = (mx[e] + log2f(den[e])) * 0.6931471805599453f;
                 }
             }
         }
@@ -550,7 +559,7 @@ cudaError_t launch_attn_t(AttnArgs a, const gsa_params_t& p, const AttnPlan& pl,
         RowRange fr = rr_all;
         fr.q_begin = t_lo; fr.R = t_hi - t_lo;
         gsa_attn_finalize_kernel<DH, G><<<(unsigned)((fr.rows() + kFinRows - 1) / kFinRows), fin_threads, 0, st>>>(
-            a.state, a.kt, g1, out, fr, a.il, a.idx_rows, p.Lq, p.n_h, p.n_kv, p.k_max, pl.mode, pl.slots);
+            a.state, a.kt, g1, out, fr, a.il, a.idx_rows, p.Lq, p.n_h, p.n_kv, p.k_max, pl.mode, pl.slots, a.lse);
         ++g_launches;
         cudaError_t fe = cudaGetLastError();
         if (fe == cudaSuccess && prog && prog->n < prog->cap && prog->n < 64) {
@@ -625,10 +634,11 @@ cudaError_t launch_sparse_attn(const gsa_params_t& p, RowRange rr, const __nv_bf
                                const __nv_bfloat16* K, const __nv_bfloat16* V,
                                const __nv_bfloat16* g1, const __nv_bfloat16* g2, const int32_t* idx,
                                const int32_t* kt, IdxLayout il, __nv_bfloat16* out, void* scratch,
-                               cudaStream_t st, AttnProgress* progress) {
+                               cudaStream_t st, AttnProgress* progress, float* lse) {
     if (rr.rows() <= 0) return cudaSuccess;
     const AttnPlan pl = plan_attn(p);
     AttnArgs a;
+    a.lse = lse;
     a.Q = Q; a.K = K; a.V = V; a.g2 = g2; a.idx = idx; a.kt = kt;
     a.state = reinterpret_cast<float*>(scratch);
     int32_t* cuts = reinterpret_cast<int32_t*>((char*)scratch + (pl.state_bytes + 255) / 256 * 256);

@@ -48,6 +48,7 @@ struct BwdArgs {
     float* lse2;                  // workspace: log2-domain log-sum-exp of the scaled logits, [B, Lq, n_h]
     float* delta;                 // workspace: sum_d dout * out, [B, Lq, n_h]
     float* pbar;                  // optional output: mean over the heads of P on S_t, [B, R, k_max], pre-zeroed
+    const float* lse_in;          // optional: natural-log softmax statistics saved by the forward pass, [B, Lq, n_h]
     float2* part_ml;              // key ranges: per range (max, sum) of the scaled logits, [n_ranges][B * Lq * n_h]
     float* dq32;                  // key ranges: dQ summed over the ranges, [B, Lq, n_h, d_h], pre-zeroed
     int32_t range_keys, n_ranges;
@@ -230,7 +231,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
         }
         cp_async_commit();                                // (possibly empty: keeps the group count uniform)
     };
-    if (MODE != 2) {
+    if (MODE != 2 && !a.lse_in) {
     fetch(j_lo, 0, false);
     for (int j0 = j_lo, stage = 0; j0 < ke; j0 += 16, stage ^= 1) {
         fetch(j0 + 16, stage ^ 1, false);
@@ -271,7 +272,13 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
                 a.part_ml[((size_t)range * a.total_rows + qrow) * a.n_h + g * G + 2 * tig + e] = make_float2(m_run[e], l_run[e]);
         return;
     }
-    if (MODE == 2) {
+    if (a.lse_in) {                                    // the forward pass saved the statistics: no first sweep
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            m_run[e] = a.lse_in[qrow * a.n_h + g * G + min(2 * tig + e, G - 1)] * kLog2e;
+            l_run[e] = 1.f;
+        }
+    } else if (MODE == 2) {
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
             const int h = g * G + min(2 * tig + e, G - 1);    // (columns >= G are padding: any finite value will do)
@@ -404,7 +411,7 @@ template <int DH, int G>
 cudaError_t launch_bwd_t(const BwdArgs& a, cudaStream_t st) {
     if (a.n_ranges <= 1) return launch_bwd_mode<DH, G, 0>(a, st);
     cudaError_t e = cudaMemsetAsync(a.dq32, 0, (size_t)a.total_rows * a.n_h * DH * 4, st);
-    if (e == cudaSuccess) e = launch_bwd_mode<DH, G, 1>(a, st);
+    if (e == cudaSuccess && !a.lse_in) e = launch_bwd_mode<DH, G, 1>(a, st);
     if (e == cudaSuccess) e = launch_bwd_mode<DH, G, 2>(a, st);
     if (e != cudaSuccess) return e;
     gsa_bwd_dq_finish_kernel<<<a.rr.rows(), 256, 0, st>>>(a.dq32, a.dQ, a.rr, a.Lq, (int64_t)a.n_h * DH);
@@ -443,12 +450,13 @@ cudaError_t launch_sparse_attn_bwd(const gsa_params_t& p, RowRange rr, const __n
                                    const __nv_bfloat16* K, const __nv_bfloat16* Vg, const __nv_bfloat16* g1,
                                    const __nv_bfloat16* out, const __nv_bfloat16* dout, const int32_t* idx,
                                    const int32_t* kt, IdxLayout il, __nv_bfloat16* dQ, __nv_bfloat16* dg1,
-                                   __nv_bfloat16* dOs, float* lse2, float* delta, float* pbar, void* range_ws,
-                                   cudaStream_t st) {
+                                   __nv_bfloat16* dOs, float* lse2, float* delta, float* pbar, const float* lse_in,
+                                   void* range_ws, cudaStream_t st) {
     if (rr.rows() <= 0) return cudaSuccess;
     BwdArgs a;
     const BwdRanges br = plan_bwd_ranges(p);
     a.range_keys = br.range_keys; a.n_ranges = br.n_ranges; a.total_rows = (int64_t)p.B * p.Lq;
+    a.lse_in = lse_in;
     a.part_ml = (float2*)range_ws;
     a.dq32 = (float*)((char*)range_ws + ((size_t)br.n_ranges * a.total_rows * p.n_h * 8 + 255) / 256 * 256);
     a.Q = Q; a.K = K; a.Vg = Vg; a.g1 = g1; a.out = out; a.dout = dout; a.idx = idx; a.kt = kt;

@@ -55,7 +55,8 @@ cudaError_t launch_sparse_attn_bwd(const gsa_params_t& p, RowRange rr, const __n
                                    const __nv_bfloat16* K, const __nv_bfloat16* Vg, const __nv_bfloat16* g1,
                                    const __nv_bfloat16* out, const __nv_bfloat16* dout, const int32_t* idx,
                                    const int32_t* kt, IdxLayout il, __nv_bfloat16* dQ, __nv_bfloat16* dg1,
-                                   __nv_bfloat16* dOs, float* lse2, float* delta, float* pbar, void* range_ws,
+                                   __nv_bfloat16* dOs, float* lse2, float* delta, float* pbar,
+                                   const float* lse_in /*nullable: the forward's saved statistics*/, void* range_ws,
                                    cudaStream_t st);
 size_t attn_bwd_range_bytes(const gsa_params_t& p);      // scratch of the query-major half when Lk spans several key ranges
 size_t attn_bwd_invert_bytes(const gsa_params_t& p, int32_t rows_per_batch);
@@ -99,7 +100,7 @@ cudaError_t launch_sparse_attn(const gsa_params_t& p, RowRange rr, const __nv_bf
                                const __nv_bfloat16* g1, const __nv_bfloat16* g2 /*nullable*/,
                                const int32_t* idx, const int32_t* kt, IdxLayout il,
                                __nv_bfloat16* out, void* scratch, cudaStream_t st,
-                               AttnProgress* progress = nullptr);
+                               AttnProgress* progress = nullptr, float* lse = nullptr);
 
 // bytes of device scratch launch_sparse_attn needs for `p` (softmax state slots, range cuts)
 size_t attn_scratch_bytes(const gsa_params_t& p);

@@ -40,9 +40,16 @@ def _index_sets(cfg, q0, q1, seed, k_lo=None, k_hi=None):
     return idx, kt
 
 
-def _run_bwd(cfg, d, idx, kt, dout, q0, q1, key_range=16384, **over):
+def _run_bwd(cfg, d, idx, kt, dout, q0, q1, key_range=16384, saved_lse=False, **over):
     p = gsa.make_params(cfg, q_begin=q0, q_end=q1, **over)
     out = U.run_attn(cfg, d, idx, kt, q_begin=q0, q_end=q1, **over)
+    lse = None
+    if saved_lse:                                    # the training-time forward call: same output, plus the statistics
+        lse = torch.full((cfg.B, cfg.Lq, cfg.n_h), float("nan"), dtype=torch.float32, device="cuda")
+        out2 = torch.full_like(out, float("nan"))
+        wsf = torch.empty(gsa.gsa_attn_workspace_bytes(p, True), dtype=torch.uint8, device="cuda")
+        gsa.gsa_sparse_gated_attn_fwd_lse(p, d["Q"], d["K"], d["V"], d["g1"], d["g2"], idx, kt, out2, lse, wsf)
+        assert torch.equal(out2[:, q0:q1], out[:, q0:q1])
     nan = float("nan")
     dQ, dg1 = torch.full_like(d["Q"], nan), torch.full_like(d["Q"], nan)
     dK, dV, dg2 = (torch.full_like(d["K"], nan) for _ in range(3))
@@ -51,16 +58,16 @@ def _run_bwd(cfg, d, idx, kt, dout, q0, q1, key_range=16384, **over):
     ws.fill_(0xFF)                               # the call must not rely on a cleared workspace
     n0 = gsa.gsa_launch_count()
     gsa.gsa_sparse_gated_attn_bwd(p, d["Q"], d["K"], d["V"], d["g1"], d["g2"], idx, kt, out, dout,
-                                  dQ, dK, dV, dg1, dg2, ws, pbar=pbar)
+                                  dQ, dK, dV, dg1, dg2, ws, pbar=pbar, lse=lse)
     torch.cuda.synchronize()
     assert gsa.gsa_device_status(ws) == 0
     # value gate, query-major kernel, count + 3 scan steps, one fill per range of 8192 query rows, key-major
     # kernel, and with several ranges the post-pass
     n_ranges = (q1 - q0 + 8191) // 8192
     key_ranges = (cfg.Lk + key_range - 1) // key_range          # of the query-major half (as in the forward pass)
-    extra = 2 if key_ranges > 1 else 0                          # statistics launch + dQ rounding pass
+    extra = (1 if saved_lse else 2) if key_ranges > 1 else 0    # statistics launch (unless saved) + dQ rounding pass
     assert gsa.gsa_launch_count() - n0 == 7 + n_ranges + (1 if n_ranges > 1 else 0) + extra
-    return dict(dQ=dQ, dg1=dg1, dK=dK, dV=dV, dg2=dg2, pbar=pbar)
+    return dict(dQ=dQ, dg1=dg1, dK=dK, dV=dV, dg2=dg2, pbar=pbar, lse=lse)
 
 
 def _compare(cfg, x, got, idx, kt, dout, q0, q1, **okw):
@@ -166,6 +173,33 @@ def test_attn_backward_several_key_ranges():
         got = _run_bwd(cfg, d, idx.cuda(), kt.cuda(), dout.cuda(), q0, q1, key_range=1024)
     finally:
         gsa.gsa_debug_set_attn_range_keys(0)
+    _compare(cfg, x, got, idx, kt, dout, q0, q1)
+
+
+@pytest.mark.parametrize("key_range", [16384, 1024])
+def test_attn_backward_with_statistics_saved_by_the_forward(key_range):
+    """gsa_sparse_gated_attn_fwd_lse writes the same output as the plain call plus lse = log sum exp of the
+    scaled logits over S_t (checked against a library logsumexp); the backward pass given lse skips its
+    first sweep and must give the same gradients (one key range, and several)."""
+    cfg = CONFIGS["l8k"].with_(name="bwd_lse", B=2, Lq=260, Lk=2600, k_base=200, k_min=9, k_max=300, seed=47)
+    x = make_inputs(cfg)
+    d = U.to_dev(x)
+    q0, q1 = 60, 260
+    idx, kt = _index_sets(cfg, q0, q1, seed=48)
+    dout = (torch.randn(d["Q"].shape, generator=torch.Generator().manual_seed(49)) * 0.25).to(torch.bfloat16)
+    gsa.gsa_debug_set_attn_range_keys(key_range)
+    try:
+        got = _run_bwd(cfg, d, idx.cuda(), kt.cuda(), dout.cuda(), q0, q1, key_range=key_range, saved_lse=True)
+    finally:
+        gsa.gsa_debug_set_attn_range_keys(0)
+    grp = cfg.n_h // cfg.n_kv
+    lse = got["lse"].cpu()
+    for b, r in ((0, 0), (1, 77), (1, 199)):
+        S = idx[b, r, : int(kt[b, r])].long()
+        for h in (0, 5, cfg.n_h - 1):
+            z = (x["K"][b, S, h // grp].double() @ x["Q"][b, q0 + r, h].double()) / cfg.d_h ** 0.5
+            assert abs(lse[b, q0 + r, h].item() - torch.logsumexp(z, dim=0).item()) <= 2e-3
+    assert torch.isnan(lse[:, :q0]).all()
     _compare(cfg, x, got, idx, kt, dout, q0, q1)
 
 
