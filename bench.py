@@ -131,7 +131,7 @@ def run_reference(args, cfg):
     oracle.build()
     x = make_inputs(cfg, slice(0, min(cfg.B, 4)) if cfg.decode else None)
     cores = oracle.num_threads()
-    n_rows = 256
+    n_rows = 1024          # about 10 s of the oracle on 16 host cores
     rates = []
     for i in range(args.warmup + args.steps):
         r, dt, n, cores = oracle_sample_rate(cfg.with_(B=x["Q"].shape[0]), x, n_rows)
@@ -424,7 +424,7 @@ def main():
         import oracle
         oracle.build()
         cores = oracle.num_threads()
-        n_rows = 256
+        n_rows = 1024          # about 10 s of the oracle on 16 host cores
         r, dt, n, cores = oracle_sample_rate(cfg.with_(B=x_cpu_sample["Q"].shape[0]), x_cpu_sample, n_rows)
         cpu_baseline = {"value": r, "unit": UNIT, "cores": cores, "kind": "oracle",
                         "sample": f"{n} stratified query rows of {cfg.name} (full visible context each), {dt:.1f} s"}
