@@ -391,8 +391,12 @@ __global__ void __launch_bounds__(1024) gsa_attn_finalize_kernel(const float* __
                                                                 float* __restrict__ lse) {
     constexpr int STATE_F = G * (DH + 2);
     const int rows = rr.rows();
-    const int lr0 = blockIdx.x * kFinRows;
-    for (int i = threadIdx.x; i < n_kv * DH; i += blockDim.x) {
+    // range mode: kFinRows rows per CTA, all (KV head, d) pairs; parts mode (few rows, several state slots to
+    // merge per row): one row and one KV head per CTA, so that a decode batch still fills the GPU
+    const int rows_per_cta = mode == 0 ? kFinRows : 1;
+    const int lr0 = blockIdx.x * rows_per_cta;
+    const int i_begin = gridDim.y > 1 ? blockIdx.y * DH : 0, i_end = gridDim.y > 1 ? i_begin + DH : n_kv * DH;
+    for (int i = i_begin + threadIdx.x; i < i_end; i += blockDim.x) {
         const int d = i % DH;
         const int g = i / DH;
         if (mode == 0) {
@@ -428,7 +432,7 @@ __global__ void __launch_bounds__(1024) gsa_attn_finalize_kernel(const float* __
                 }
             }
         } else {
-            for (int q = 0; q < kFinRows && lr0 + q < rows; ++q) {
+            for (int q = 0; q < rows_per_cta && lr0 + q < rows; ++q) {
                 const RowId r = row_of(rr, il, lr0 + q);
                 const int k_eff = min(kt[r.irow], k_max);
                 const int np = parts_of(k_eff, max_parts);
@@ -558,7 +562,9 @@ cudaError_t launch_attn_t(AttnArgs a, const gsa_params_t& p, const AttnPlan& pl,
         if (t_hi <= t_lo) return cudaSuccess;
         RowRange fr = rr_all;
         fr.q_begin = t_lo; fr.R = t_hi - t_lo;
-        gsa_attn_finalize_kernel<DH, G><<<(unsigned)((fr.rows() + kFinRows - 1) / kFinRows), fin_threads, 0, st>>>(
+        const dim3 fin_grid = pl.mode == 0 ? dim3((unsigned)((fr.rows() + kFinRows - 1) / kFinRows), 1)
+                                           : dim3((unsigned)fr.rows(), (unsigned)a.n_kv);
+        gsa_attn_finalize_kernel<DH, G><<<fin_grid, pl.mode == 0 ? fin_threads : DH, 0, st>>>(
             a.state, a.kt, g1, out, fr, a.il, a.idx_rows, p.Lq, p.n_h, p.n_kv, p.k_max, pl.mode, pl.slots, a.lse);
         ++g_launches;
         cudaError_t fe = cudaGetLastError();
