@@ -389,6 +389,8 @@ def main():
                                     "mean_loss": float(loss_rows.double().mean().item()),
                                     "note": "target_ms: gsa_attn_probs_mean on its own (the backward call above already "
                                             "emits the same target); gsa_indexer_kl_bwd gathers k^I, dk^I by fp32 vector reductions"}
+        backward["train_step_ms"] = ms_total / args.steps + b_ms + backward["indexer_loss"]["loss_and_grads_ms"]
+        backward["train_step_note"] = "forward + attention backward (statistics saved, loss target as by-product) + indexer loss and derivatives"
         del idx_b, pbar, loss_rows, dqI, dkI, dw, ws_k
 
     # ---- end to end through the host-buffer entry point ------------------------------------
