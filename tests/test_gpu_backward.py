@@ -329,3 +329,34 @@ def test_indexer_kl_layer_shape_row_range_batch_bias():
 def test_indexer_kl_relu_indexer():
     cfg = CONFIGS["l8k"].with_(name="kl_relu", B=1, Lq=200, Lk=900, HI=4, dI=32, k_base=100, k_min=20, k_max=160, seed=54)
     _check_loss_path(cfg, 0, 200, seed=55, bias=True, act=1)
+
+
+def test_indexer_warmup_loss_on_all_visible_keys():
+    """Eq. 13 for a short context: the index sets of the dense fallback (k_mode 3: every visible key) fed to the
+    same two entry points."""
+    cfg = CONFIGS["tiny"].with_(name="warmup", B=2, Lq=90, Lk=200, k_base=8, k_min=4, k_max=208, seed=56)
+    x = make_inputs(cfg)
+    d = U.to_dev(x)
+    p = gsa.make_params(cfg, k_mode=3)
+    out = torch.empty_like(d["Q"])
+    idx = torch.empty((cfg.B, cfg.Lq, cfg.k_max), dtype=torch.int32, device="cuda")
+    kt = torch.empty((cfg.B, cfg.Lq), dtype=torch.int32, device="cuda")
+    ws = torch.empty(gsa.gsa_workspace_bytes(p, 0), dtype=torch.uint8, device="cuda")
+    gsa.gsa_forward(p, d["Q"], d["K"], d["V"], None, None, None, None, d["g1"], d["g2"], out, idx, kt, None, 0, ws)
+    torch.cuda.synchronize()
+    idx_c, kt_c = idx.cpu(), kt.cpu()
+    assert (kt_c[0].numpy() == cfg.Lk - cfg.Lq + np.arange(cfg.Lq) + 1).all()
+    R = cfg.Lq
+    rows_b, rows_t = np.repeat(np.arange(cfg.B), R), np.tile(np.arange(R), cfg.B)
+    po = U.oracle_params(cfg)
+    idx2, kt1 = idx_c.reshape(cfg.B * R, -1).numpy(), kt_c.reshape(-1).numpy()
+    want_p = oracle.attn_probs_mean(po, x["Q"], x["K"], idx2, kt1, rows_t, rows_b)
+    got_p = _run_probs(cfg, d, idx, kt, 0, R).cpu().numpy().reshape(cfg.B * R, -1)
+    assert (np.abs(got_p - want_p) <= 2e-3 * want_p + 1e-7).all()
+    pb32 = want_p.astype(np.float32)
+    want = oracle.indexer_kl(po, x["qI"], x["kI"], x["w"], None, idx2, kt1, pb32.astype(np.float64), rows_t, rows_b)
+    got = _run_kl(cfg, d, None, idx, kt, torch.from_numpy(pb32).reshape(cfg.B, R, -1).cuda(), 0, R)
+    gl = got["loss"].cpu().numpy().reshape(-1)
+    assert (np.abs(gl - want["loss"]) <= 2e-3 * np.abs(want["loss"]) + 2e-5).all()
+    g, w = got["dkI"].float().cpu().numpy(), want["dkI"]
+    assert np.linalg.norm(g - w) <= GRAD_FROBENIUS_TOL * np.linalg.norm(w)

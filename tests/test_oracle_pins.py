@@ -610,6 +610,29 @@ def test_indexer_kl_loss_and_gradients_match_library_autograd(act):
     np.testing.assert_allclose(got["dbI"], t64["bI"].grad.numpy(), rtol=1e-9, atol=1e-13)
 
 
+def test_indexer_warmup_loss_is_the_sparse_loss_on_all_visible_keys():
+    """Eq. 13 (warm-up phase): KL(p_t || softmax(I_t)) over every visible key.  With S_t = all visible keys the
+    Eq. 14 routines compute it; checked against the dense computation with library softmax / KL divergence."""
+    p, x, _, _, _, _ = _kl_problem(14, B=1, Lq=6, Lk=9, k_max=9)
+    rows_t = np.arange(p.Lq, dtype=np.int32)
+    idx = np.full((p.Lq, p.k_max), -1, np.int32)
+    keff = np.array([p.visible(t) for t in rows_t], np.int32)
+    for t in rows_t:
+        idx[t, : keff[t]] = np.arange(keff[t])
+    pbar = oracle.attn_probs_mean(p, x["Q"], x["K"], idx, keff, rows_t)
+    got = oracle.indexer_kl(p, x["qI"], x["kI"], x["w"], x["bI"], idx, keff, pbar, rows_t)
+    sc = oracle.scores(p, x["qI"], x["kI"], x["w"], x["bI"], rows_t)
+    grp = p.n_h // p.n_kv
+    for t in rows_t:
+        n = keff[t]
+        dense = torch.zeros(n, dtype=torch.float64)
+        for h in range(p.n_h):
+            z = (x["K"][0, :n, h // grp].double() @ x["Q"][0, t, h].double()) / math.sqrt(p.d_h)
+            dense += torch.softmax(z, dim=0) / p.n_h
+        L = torch.nn.functional.kl_div(torch.log_softmax(torch.from_numpy(sc[t, :n]), dim=0), dense, reduction="sum")
+        np.testing.assert_allclose(got["loss"][t], L.item(), rtol=1e-10, atol=1e-13)
+
+
 def test_indexer_kl_closed_forms_and_central_differences():
     """Equal indexer keys give equal scores, so q is uniform: with the target (1/4, 3/4) the loss is
     1/4 ln(1/2) + 3/4 ln(3/2) and the derivative with respect to the two scores is (1/2 - 1/4, 1/2 - 3/4).
