@@ -7,6 +7,13 @@
  *   gsa_sparse_gated_attn_fwd  value gate G2, sparse softmax attention over
  *                              S_t, output gate G1                         (Eq. 9, 11, 12, 10)
  *   gsa_forward                all of the above for a whole batch          (Sec. 3.2, Eq. 6 pipeline)
+ * The steps either side of the path and its training side:
+ *   gsa_project, gsa_output_projection     the projections that feed / follow the path (text below Eq. 7,
+ *                                          Eq. 9, Eq. 10, Sec. 2.1)
+ *   gsa_sparse_gated_attn_fwd_lse, gsa_sparse_gated_attn_bwd
+ *                                          the attention stage for training and its backward pass
+ *   gsa_attn_probs_mean, gsa_indexer_kl_bwd   the indexer's loss and its derivatives (Sec. 5.1, Eq. 13-14)
+ *   gsa_vbar_update                        the running mean of the score variance of Eq. 8
  *
  * Conventions common to every call
  *   - Every data pointer is DEVICE memory owned by the caller, 16-byte aligned and
@@ -25,7 +32,7 @@
  *     n_t = Lk-Lq+t+1).  Prefill is Lq == Lk; decode is Lq == 1 over an Lk-token cache.
  *
  * Supported shapes: d_h in {64, 128}; dI in {32, 64}; HI in {1, 2, 4, 8};
- * n_h / n_kv in {1, 2, 4, 8}; k_max <= 4096; 1 <= Lq <= Lk < 2^24.
+ * n_h / n_kv in {1, 2, 4, 8}; n_kv in {1, 2, 4, 8}; k_max <= 4096; 1 <= Lq <= Lk < 2^24.
  */
 #ifndef GSA_H_
 #define GSA_H_
