@@ -403,6 +403,10 @@ def test_forward_dense_fallback_mode_needs_no_indexer_inputs():
                         d["g1"], d["g2"], out, None, kt, None, 0, ws)
     assert gsa.gsa_launch_count() == n1
     assert n1 - n0 <= 6          # all-visible, value gate, range cuts, attention, finalize
+    # the per-stage selection call in the same mode: whatever the scores, every visible key, in order
+    sc = torch.rand((cfg.B, cfg.Lq, U.row_stride(cfg)), device="cuda")
+    idx2, kt2, _ = U.run_topk(cfg, sc, k_mode=3)
+    assert torch.equal(idx2, idx) and torch.equal(kt2, kt)
 
 
 def test_forward_batched_chunked_prefill():
