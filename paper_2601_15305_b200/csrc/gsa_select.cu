@@ -100,7 +100,7 @@ __device__ __forceinline__ void block_minmax(SelShared& sh, uint32_t& kmin, uint
     }
     __syncthreads();
     kmin = sh.bc_min; kmax = sh.bc_max;
-    __syncthreads();
+    // (no barrier here: every caller passes another barrier before red_* or bc_* are written again)
 }
 
 // After a histogram has been filled: the bin holding the `want`-th largest entry (1 = largest) and
@@ -132,7 +132,8 @@ __device__ __forceinline__ void find_bin(SelShared& sh, uint32_t want, uint32_t&
     __syncthreads();
     bin = sh.found_bin;
     above = sh.found_above;
-    __syncthreads();
+    // (no barrier here: the histogram is not read after the barrier above, and found_* / warp_tot are next
+    // written only after the caller's next barriers)
 }
 
 // smallest shift with (span >> shift) < kBins
