@@ -12,9 +12,11 @@
 //
 // Two kernels, neither with floating-point atomics:
 //  * this file, query-major: one warp per (query row, KV head).  Per 16 selected keys the K and V' rows
-//    are copied (16-byte asynchronous copies) into a private shared-memory tile and every product runs on
-//    the tensor cores (bf16 mma.sync, fp32 accumulation) with the keys as M:
-//        S^T[key, head] = K . Q^T      dP^T[key, head] = V' . do^T            (A: tile via ldmatrix)
+//    are copied (16-byte asynchronous copies) into a private shared-memory tile, the V' rows go straight
+//    from global memory into MMA fragments, and every product runs on the tensor cores (bf16 mma.sync, fp32
+//    accumulation) with the keys as M:
+//        S^T[key, head] = K . Q^T           (A: tile via ldmatrix)
+//        dP^T[key, head] = V' . do^T        (A: 32-byte loads, contraction index in load order)
 //        dQ^T[d, head] += K^T . dS^T                                          (A: tile via ldmatrix.trans)
 //    It writes dQ and dg1 and leaves do (bf16), the softmax statistics and delta per (row, head) in the
 //    workspace for the other kernel.  When the keys span several L2-sized ranges (as in the forward pass:
@@ -52,6 +54,7 @@ struct BwdArgs {
     float2* part_ml;              // key ranges: per range (max, sum) of the scaled logits, [n_ranges][B * Lq * n_h]
     float* dq32;                  // key ranges: dQ summed over the ranges, [B, Lq, n_h, d_h], pre-zeroed
     int32_t range_keys, n_ranges;
+    const int32_t* cuts;          // key ranges: [B * Lq][n_ranges + 1] first position of each range in the row's index set
     int64_t total_rows;           // B * Lq
     RowRange rr;
     IdxLayout il;
@@ -85,17 +88,36 @@ __device__ __forceinline__ int warp_lower_bound(const int32_t* __restrict__ S, i
     return lo;
 }
 
+// cuts[row][c] = first position of the row's ascending index set that lies in key range c (c = n_ranges: the end)
+__global__ void __launch_bounds__(256) gsa_bwd_range_cuts_kernel(const int32_t* __restrict__ idx, const int32_t* __restrict__ kt,
+                                                                 int32_t* __restrict__ cuts, RowRange rr, IdxLayout il,
+                                                                 int32_t Lq, int32_t k_max, int32_t n_ranges, int32_t range_keys) {
+    const int lane = threadIdx.x & 31;
+    const int64_t lr = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (lr >= rr.rows()) return;
+    const int b = rr.b0 + (int)(lr / rr.R), t = rr.q_begin + (int)(lr % rr.R);
+    const int64_t irow = il.row(b, t);
+    const int ke = kt[irow];
+    const int32_t* __restrict__ S = idx + irow * k_max;
+    int32_t* const out = cuts + ((int64_t)b * Lq + t) * (n_ranges + 1);
+    for (int c = 0; c <= n_ranges; ++c) {
+        const int j = c == 0 ? 0 : (c == n_ranges ? ke : warp_lower_bound(S, ke, c * range_keys, lane));
+        if (lane == 0) out[c] = j;
+    }
+}
+
 // MODE 0: one item = (row, KV head), both sweeps over the whole index set.
 // MODE 1: one item = (key range, row, KV head): statistics sweep over the range's part of S_t -> part_ml.
 // MODE 2: one item = (key range, row, KV head): statistics combined from part_ml, gradient sweep over the
 //         range's part, dQ added into dq32; the items of range 0 also write dg1, do, delta and lse2.
 template <int DH, int G, int MODE>
-__global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(const BwdArgs a) {
+__global__ void __launch_bounds__(kBwdWarps * 32, 4) gsa_sparse_attn_bwd_kernel(const BwdArgs a) {
     constexpr int ROW = (DH + 8) * 2;                  // bytes of a padded tile row (odd multiple of 16)
     constexpr int KTILE = 16 * ROW, QTILE = 8 * ROW;
-    constexpr int STAGE = 2 * KTILE;                   // a K tile and a V' tile
-    constexpr int WARP_SMEM = 2 * STAGE;               // two stages; the Q / do tiles borrow stage 1 first
-    static_assert(2 * QTILE + 64 <= STAGE, "the row's own tiles must fit one stage");
+    constexpr int STAGE = KTILE;                       // a K tile (V' rows go straight into MMA fragments)
+    constexpr int WARP_SMEM = 2 * STAGE;               // two stages; the Q / do tiles borrow them before the sweeps
+    static_assert(2 * QTILE + 64 <= WARP_SMEM, "the row's own tiles must fit the two stages");
+    constexpr int NC = DH / 32;                        // 16-byte pieces of a head row per lane (register-direct rows)
     constexpr int KS = DH / 16;                        // k-steps of the S^T / dP^T products, m-tiles of dQ^T
     constexpr int EPL = DH / 32;                       // elements of a head row per lane (row staging)
     constexpr int CPR = DH / 8;                        // 16-byte chunks per tile row
@@ -120,8 +142,9 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
     // this item's part of the index set: positions [j_lo, ke)
     int j_lo = 0, ke = ke_all;
     if (MODE != 0) {
-        j_lo = warp_lower_bound(S, ke_all, range * a.range_keys, lane);
-        ke = warp_lower_bound(S, ke_all, (range + 1) * a.range_keys, lane);
+        const int32_t* const cut = a.cuts + qrow * (a.n_ranges + 1) + range;
+        j_lo = cut[0];
+        ke = cut[1];
     }
     const bool writes_row = MODE == 0 || (MODE == 2 && range == 0);   // dg1, do, delta, lse2 are written once
     if (MODE == 1 && j_lo >= ke) {                     // nothing of the row in this range
@@ -131,10 +154,10 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
     if (MODE == 2 && j_lo >= ke && !writes_row) return;
 
     unsigned char* const ws = bwd_smem + warp * WARP_SMEM;
-    unsigned char* const q_tile = ws + STAGE;           // rows = the group's heads (rows >= G are zero)
-    unsigned char* const d_tile = ws + STAGE + QTILE;
-    float* const s_delta = reinterpret_cast<float*>(ws + STAGE + 2 * QTILE);   // [8]
-    const uint32_t st_s32 = (uint32_t)__cvta_generic_to_shared(ws);   // stage i: K tile at i * STAGE, V' tile after it
+    unsigned char* const q_tile = ws;                   // rows = the group's heads (rows >= G are zero)
+    unsigned char* const d_tile = ws + QTILE;
+    float* const s_delta = reinterpret_cast<float*>(ws + 2 * QTILE);   // [8]
+    const uint32_t st_s32 = (uint32_t)__cvta_generic_to_shared(ws);   // stage i: K tile at i * STAGE
     const uint32_t q_s32 = (uint32_t)__cvta_generic_to_shared(q_tile);
     const uint32_t d_s32 = (uint32_t)__cvta_generic_to_shared(d_tile);
 
@@ -178,14 +201,20 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
     const float delta[2] = {s_delta[2 * tig], s_delta[2 * tig + 1]};
 
     // B operands of S^T = K Q^T and dP^T = V' do^T: (k = d, n = head), kept for the whole row
-    uint32_t qb[2 * KS], dob[2 * KS];
+    uint32_t qb[2 * KS];
 #pragma unroll
     for (int k2 = 0; k2 < KS / 2; ++k2) {
         const uint32_t off = (lane & 7) * ROW + (lane >> 3) * 16 + k2 * 64;
         ldmatrix_x4(qb[4 * k2], qb[4 * k2 + 1], qb[4 * k2 + 2], qb[4 * k2 + 3], q_s32 + off);
-        ldmatrix_x4(dob[4 * k2], dob[4 * k2 + 1], dob[4 * k2 + 2], dob[4 * k2 + 3], d_s32 + off);
     }
-    __syncwarp();                                      // stage 1 is free for tiles from here on
+    // B operand of dP^T = V' do^T in the order the V' rows are loaded in: lane (gid, tig) brings bytes
+    // [(c/2)*128 + tig*32 + (c%2)*16, +16) of the rows of keys gid and gid + 8 straight from global memory
+    // into the A fragments, so the contraction index is permuted; do of head gid is read the same way
+    uint4 dobd[NC];
+#pragma unroll
+    for (int c = 0; c < NC; ++c)
+        dobd[c] = *reinterpret_cast<const uint4*>(d_tile + gid * ROW + (c >> 1) * 128 + tig * 32 + (c & 1) * 16);
+    __syncwarp();                                      // the stages are free for tiles from here on
 
     const float c2 = a.scale * kLog2e;
     const size_t kv_row = (size_t)a.n_kv * DH;           // elements between consecutive keys
@@ -223,18 +252,37 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
     // ---- sweep 1: softmax statistics per head (log2 domain) ----------------------------------------
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
     // tiles are fetched one iteration ahead
-    auto fetch = [&](int j, int stage, bool with_v) {
+    int32_t pos_fetched = 0;                              // positions of the tile fetched last (lanes 0..15)
+    auto fetch = [&](int j, int stage) {
         if (j < ke) {
-            const int32_t pos16 = S[min(j + (lane & 15), ke - 1)];
-            fetch_tile(kbase, st_s32 + stage * STAGE, pos16);
-            if (with_v) fetch_tile(vbase, st_s32 + stage * STAGE + KTILE, pos16);
+            pos_fetched = S[min(j + (lane & 15), ke - 1)];
+            fetch_tile(kbase, st_s32 + stage * STAGE, pos_fetched);
         }
         cp_async_commit();                                // (possibly empty: keeps the group count uniform)
     };
+    // V' rows of 16 keys as A fragments (see dobd above)
+    uint4 vb[2 * NC];
+    const unsigned char* const vrow0 = reinterpret_cast<const unsigned char*>(vbase) + tig * 32;
+    auto load_v = [&](int32_t pos16) {
+        const uint32_t p0 = __shfl_sync(0xFFFFFFFFu, pos16, gid), p1 = __shfl_sync(0xFFFFFFFFu, pos16, gid + 8);
+        const unsigned char* v0p = vrow0 + (size_t)p0 * kv_row * 2;
+        const unsigned char* v1p = vrow0 + (size_t)p1 * kv_row * 2;
+#pragma unroll
+        for (int c = 0; c < NC; c += 2) {
+            asm volatile("ld.global.nc.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                         : "=r"(vb[c].x), "=r"(vb[c].y), "=r"(vb[c].z), "=r"(vb[c].w), "=r"(vb[c + 1].x),
+                           "=r"(vb[c + 1].y), "=r"(vb[c + 1].z), "=r"(vb[c + 1].w)
+                         : "l"(v0p + (c >> 1) * 128));
+            asm volatile("ld.global.nc.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                         : "=r"(vb[NC + c].x), "=r"(vb[NC + c].y), "=r"(vb[NC + c].z), "=r"(vb[NC + c].w),
+                           "=r"(vb[NC + c + 1].x), "=r"(vb[NC + c + 1].y), "=r"(vb[NC + c + 1].z), "=r"(vb[NC + c + 1].w)
+                         : "l"(v1p + (c >> 1) * 128));
+        }
+    };
     if (MODE != 2 && !a.lse_in) {
-    fetch(j_lo, 0, false);
+    fetch(j_lo, 0);
     for (int j0 = j_lo, stage = 0; j0 < ke; j0 += 16, stage ^= 1) {
-        fetch(j0 + 16, stage ^ 1, false);
+        fetch(j0 + 16, stage ^ 1);
         cp_async_wait<1>();
         __syncwarp();
         float s[4];
@@ -303,15 +351,27 @@ __global__ void __launch_bounds__(kBwdWarps * 32) gsa_sparse_attn_bwd_kernel(con
     float dq[KS][4];
 #pragma unroll
     for (int mt = 0; mt < KS; ++mt) dq[mt][0] = dq[mt][1] = dq[mt][2] = dq[mt][3] = 0.f;
-    fetch(j_lo, 0, true);
+    fetch(j_lo, 0);
+    load_v(pos_fetched);
     for (int j0 = j_lo, stage = 0; j0 < ke; j0 += 16, stage ^= 1) {
-        fetch(j0 + 16, stage ^ 1, true);
+        fetch(j0 + 16, stage ^ 1);
         cp_async_wait<1>();
         __syncwarp();
-        const uint32_t k_s32 = st_s32 + stage * STAGE, v_s32 = k_s32 + KTILE;
+        const uint32_t k_s32 = st_s32 + stage * STAGE;
         float s[4], dp[4], p[4], ds[4];
         tile_times(k_s32, qb, s);
-        tile_times(v_s32, dob, dp);
+        {
+            float dp2[4] = {0.f, 0.f, 0.f, 0.f};
+            dp[0] = dp[1] = dp[2] = dp[3] = 0.f;
+#pragma unroll
+            for (int c = 0; c < NC; ++c) {
+                mma_bf16_16816(dp, vb[c].x, vb[NC + c].x, vb[c].y, vb[NC + c].y, dobd[c].x, dobd[c].y);
+                mma_bf16_16816(dp2, vb[c].z, vb[NC + c].z, vb[c].w, vb[NC + c].w, dobd[c].z, dobd[c].w);
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) dp[i] += dp2[i];
+        }
+        if (j0 + 16 < ke) load_v(pos_fetched);            // the next tile's V' rows, under the rest of this tile's work
         const bool v0 = j0 + gid < ke, v1 = j0 + gid + 8 < ke;
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
@@ -394,7 +454,7 @@ __global__ void __launch_bounds__(256) gsa_bwd_dq_finish_kernel(const float* __r
 template <int DH, int G, int MODE>
 cudaError_t launch_bwd_mode(const BwdArgs& a, cudaStream_t st) {
     constexpr int ROW = (DH + 8) * 2;
-    constexpr int WARP_SMEM = 4 * 16 * ROW;
+    constexpr int WARP_SMEM = 2 * 16 * ROW;
     const int smem = kBwdWarps * WARP_SMEM;
     auto kern = gsa_sparse_attn_bwd_kernel<DH, G, MODE>;
     // (set on every call: the attribute belongs to the current device)
@@ -410,7 +470,11 @@ cudaError_t launch_bwd_mode(const BwdArgs& a, cudaStream_t st) {
 template <int DH, int G>
 cudaError_t launch_bwd_t(const BwdArgs& a, cudaStream_t st) {
     if (a.n_ranges <= 1) return launch_bwd_mode<DH, G, 0>(a, st);
-    cudaError_t e = cudaMemsetAsync(a.dq32, 0, (size_t)a.total_rows * a.n_h * DH * 4, st);
+    gsa_bwd_range_cuts_kernel<<<(unsigned)((a.rr.rows() + 7) / 8), 256, 0, st>>>(a.idx, a.kt, const_cast<int32_t*>(a.cuts), a.rr,
+                                                                                  a.il, a.Lq, a.k_max, a.n_ranges, a.range_keys);
+    ++g_launches;
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaMemsetAsync(a.dq32, 0, (size_t)a.total_rows * a.n_h * DH * 4, st);
     if (e == cudaSuccess && !a.lse_in) e = launch_bwd_mode<DH, G, 1>(a, st);
     if (e == cudaSuccess) e = launch_bwd_mode<DH, G, 2>(a, st);
     if (e != cudaSuccess) return e;
@@ -438,7 +502,8 @@ size_t attn_bwd_range_bytes(const gsa_params_t& p) {
     const BwdRanges br = plan_bwd_ranges(p);
     if (br.n_ranges <= 1) return 0;
     const size_t rows = (size_t)p.B * p.Lq;
-    return ((size_t)br.n_ranges * rows * p.n_h * 8 + 255) / 256 * 256 + (rows * p.n_h * p.d_h * 4 + 255) / 256 * 256;
+    return ((size_t)br.n_ranges * rows * p.n_h * 8 + 255) / 256 * 256 + (rows * p.n_h * p.d_h * 4 + 255) / 256 * 256 +
+           (rows * (br.n_ranges + 1) * 4 + 255) / 256 * 256;
 }
 
 bool attn_bwd_supported(const gsa_params_t& p) {
@@ -459,6 +524,7 @@ cudaError_t launch_sparse_attn_bwd(const gsa_params_t& p, RowRange rr, const __n
     a.lse_in = lse_in;
     a.part_ml = (float2*)range_ws;
     a.dq32 = (float*)((char*)range_ws + ((size_t)br.n_ranges * a.total_rows * p.n_h * 8 + 255) / 256 * 256);
+    a.cuts = (const int32_t*)((char*)a.dq32 + ((size_t)a.total_rows * p.n_h * p.d_h * 4 + 255) / 256 * 256);
     a.Q = Q; a.K = K; a.Vg = Vg; a.g1 = g1; a.out = out; a.dout = dout; a.idx = idx; a.kt = kt;
     a.dQ = dQ; a.dg1 = dg1; a.dOs = dOs; a.lse2 = lse2; a.delta = delta; a.pbar = pbar; a.rr = rr; a.il = il;
     a.Lq = p.Lq; a.Lk = p.Lk; a.n_h = p.n_h; a.n_kv = p.n_kv; a.k_max = p.k_max;

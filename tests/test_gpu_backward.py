@@ -65,7 +65,7 @@ def _run_bwd(cfg, d, idx, kt, dout, q0, q1, key_range=16384, saved_lse=False, **
     # kernel, and with several ranges the post-pass
     n_ranges = (q1 - q0 + 8191) // 8192
     key_ranges = (cfg.Lk + key_range - 1) // key_range          # of the query-major half (as in the forward pass)
-    extra = (1 if saved_lse else 2) if key_ranges > 1 else 0    # statistics launch (unless saved) + dQ rounding pass
+    extra = (2 if saved_lse else 3) if key_ranges > 1 else 0    # range cuts, statistics launch (unless saved), dQ rounding pass
     assert gsa.gsa_launch_count() - n0 == 7 + n_ranges + (1 if n_ranges > 1 else 0) + extra
     return dict(dQ=dQ, dg1=dg1, dK=dK, dV=dV, dg2=dg2, pbar=pbar, lse=lse)
 
