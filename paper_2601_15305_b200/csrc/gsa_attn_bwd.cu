@@ -18,8 +18,8 @@
 //        S^T[key, head] = K . Q^T           (A: tile via ldmatrix)
 //        dP^T[key, head] = V' . do^T        (A: 32-byte loads, contraction index in load order)
 //        dQ^T[d, head] += K^T . dS^T                                          (A: tile via ldmatrix.trans)
-//    It writes dQ and dg1 and leaves do (bf16), the softmax statistics and delta per (row, head) in the
-//    workspace for the other kernel.  When the keys span several L2-sized ranges (as in the forward pass:
+//    A streaming preparation kernel writes dg1, do (bf16) and delta per (row, head) first; this kernel
+//    writes dQ and leaves the softmax statistics in the workspace for the other kernel.  When the keys span several L2-sized ranges (as in the forward pass:
 //    random 256-byte rows come much faster out of L2 than out of HBM) the work items are (key range, row,
 //    KV head), range-major, in two launches: the first leaves each range's softmax statistics, the second
 //    combines them, does the gradient sweep over its range's part of S_t (ascending index sets make that a
@@ -72,6 +72,36 @@ __device__ __forceinline__ float ex2_approx(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// Per (row, head), before the sweeps: do = dout * sigmoid(g1) (bf16), dg1 = dout * out * (1 - sigmoid(g1)),
+// delta = sum_d dout * out.  One warp per (row, head).
+template <int DH>
+__global__ void __launch_bounds__(256) gsa_bwd_prep_kernel(const __nv_bfloat16* __restrict__ g1,
+                                                           const __nv_bfloat16* __restrict__ out,
+                                                           const __nv_bfloat16* __restrict__ dout,
+                                                           __nv_bfloat16* __restrict__ dOs, __nv_bfloat16* __restrict__ dg1,
+                                                           float* __restrict__ delta, RowRange rr, int32_t Lq, int32_t n_h) {
+    constexpr int EPL = DH / 32;
+    const int lane = threadIdx.x & 31;
+    const int64_t w = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (w >= (int64_t)rr.rows() * n_h) return;
+    const int lr = (int)(w / n_h), h = (int)(w % n_h);
+    const int64_t qrow = (int64_t)(rr.b0 + lr / rr.R) * Lq + rr.q_begin + lr % rr.R;
+    const int64_t at = (qrow * n_h + h) * DH + lane * EPL;
+    float part = 0.f;
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) {
+        const float dy = __bfloat162float(dout[at + e]);
+        const float y = __bfloat162float(out[at + e]);
+        const float sg = 1.0f / (1.0f + __expf(-__bfloat162float(g1[at + e])));
+        dOs[at + e] = __float2bfloat16(dy * sg);
+        dg1[at + e] = __float2bfloat16(dy * y * (1.0f - sg));
+        part = fmaf(dy, y, part);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
+    if (lane == 0) delta[qrow * n_h + h] = part;
+}
+
 // first position j of the ascending list S[0 .. n) with S[j] >= x; the whole warp calls it (32 probes a round)
 __device__ __forceinline__ int warp_lower_bound(const int32_t* __restrict__ S, int n, int x, int lane) {
     int lo = 0, len = n;
@@ -116,7 +146,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32, 4) gsa_sparse_attn_bwd_kernel(
     constexpr int KTILE = 16 * ROW, QTILE = 8 * ROW;
     constexpr int STAGE = KTILE;                       // a K tile (V' rows go straight into MMA fragments)
     constexpr int WARP_SMEM = 2 * STAGE;               // two stages; the Q / do tiles borrow them before the sweeps
-    static_assert(2 * QTILE + 64 <= WARP_SMEM, "the row's own tiles must fit the two stages");
+    static_assert(2 * QTILE <= WARP_SMEM, "the row's own tiles must fit the two stages");
     constexpr int NC = DH / 32;                        // 16-byte pieces of a head row per lane (register-direct rows)
     constexpr int KS = DH / 16;                        // k-steps of the S^T / dP^T products, m-tiles of dQ^T
     constexpr int EPL = DH / 32;                       // elements of a head row per lane (row staging)
@@ -146,7 +176,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32, 4) gsa_sparse_attn_bwd_kernel(
         j_lo = cut[0];
         ke = cut[1];
     }
-    const bool writes_row = MODE == 0 || (MODE == 2 && range == 0);   // dg1, do, delta, lse2 are written once
+    const bool writes_row = MODE == 0 || (MODE == 2 && range == 0);   // lse2 is written once per row
     if (MODE == 1 && j_lo >= ke) {                     // nothing of the row in this range
         if (lane < G) a.part_ml[((size_t)range * a.total_rows + qrow) * a.n_h + g * G + lane] = make_float2(-INFINITY, 0.f);
         return;
@@ -156,49 +186,26 @@ __global__ void __launch_bounds__(kBwdWarps * 32, 4) gsa_sparse_attn_bwd_kernel(
     unsigned char* const ws = bwd_smem + warp * WARP_SMEM;
     unsigned char* const q_tile = ws;                   // rows = the group's heads (rows >= G are zero)
     unsigned char* const d_tile = ws + QTILE;
-    float* const s_delta = reinterpret_cast<float*>(ws + 2 * QTILE);   // [8]
     const uint32_t st_s32 = (uint32_t)__cvta_generic_to_shared(ws);   // stage i: K tile at i * STAGE
     const uint32_t q_s32 = (uint32_t)__cvta_generic_to_shared(q_tile);
     const uint32_t d_s32 = (uint32_t)__cvta_generic_to_shared(d_tile);
 
-    // ---- per row: do = dout * sigmoid(g1), dg1, delta; Q and do staged as tiles -------------------
+    // ---- the row's Q and do = dout * sigmoid(g1) (written by the preparation kernel) staged as tiles ---
 #pragma unroll
     for (int hl = 0; hl < 8; ++hl) {
         __nv_bfloat16* qd = reinterpret_cast<__nv_bfloat16*>(q_tile + hl * ROW) + lane * EPL;
         __nv_bfloat16* dd = reinterpret_cast<__nv_bfloat16*>(d_tile + hl * ROW) + lane * EPL;
-        float part = 0.f;
-        if (hl < G) {
-            const int64_t at = (qrow * a.n_h + (g * G + hl)) * DH + lane * EPL;
+        const int64_t at = (qrow * a.n_h + (g * G + hl)) * DH + lane * EPL;
 #pragma unroll
-            for (int e = 0; e < EPL; ++e) {
-                qd[e] = a.Q[at + e];
-                if (MODE != 1) {                       // (the statistics launch needs Q only)
-                    const float dy = __bfloat162float(a.dout[at + e]);
-                    const float y = __bfloat162float(a.out[at + e]);
-                    const float sg = 1.0f / (1.0f + __expf(-__bfloat162float(a.g1[at + e])));
-                    dd[e] = __float2bfloat16(dy * sg);
-                    if (writes_row) {
-                        a.dOs[at + e] = dd[e];
-                        a.dg1[at + e] = __float2bfloat16(dy * y * (1.0f - sg));
-                    }
-                    part = fmaf(dy, y, part);
-                } else {
-                    dd[e] = __float2bfloat16(0.f);
-                }
-            }
-        } else {
-#pragma unroll
-            for (int e = 0; e < EPL; ++e) { qd[e] = __float2bfloat16(0.f); dd[e] = __float2bfloat16(0.f); }
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
-        if (lane == 0) {
-            s_delta[hl] = part;
-            if (hl < G && writes_row) a.delta[qrow * a.n_h + g * G + hl] = part;
+        for (int e = 0; e < EPL; ++e) {
+            qd[e] = hl < G ? a.Q[at + e] : __float2bfloat16(0.f);
+            dd[e] = (hl < G && MODE != 1) ? a.dOs[at + e] : __float2bfloat16(0.f);
         }
     }
     __syncwarp();
-    const float delta[2] = {s_delta[2 * tig], s_delta[2 * tig + 1]};
+    float delta[2];
+#pragma unroll
+    for (int e = 0; e < 2; ++e) delta[e] = (MODE != 1 && 2 * tig + e < G) ? a.delta[qrow * a.n_h + g * G + 2 * tig + e] : 0.f;
 
     // B operands of S^T = K Q^T and dP^T = V' do^T: (k = d, n = head), kept for the whole row
     uint32_t qb[2 * KS];
@@ -469,6 +476,14 @@ cudaError_t launch_bwd_mode(const BwdArgs& a, cudaStream_t st) {
 
 template <int DH, int G>
 cudaError_t launch_bwd_t(const BwdArgs& a, cudaStream_t st) {
+    {
+        const int64_t warps = (int64_t)a.rr.rows() * a.n_h;
+        gsa_bwd_prep_kernel<DH><<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(a.g1, a.out, a.dout, a.dOs, a.dg1, a.delta,
+                                                                            a.rr, a.Lq, a.n_h);
+        ++g_launches;
+        cudaError_t e0 = cudaGetLastError();
+        if (e0 != cudaSuccess) return e0;
+    }
     if (a.n_ranges <= 1) return launch_bwd_mode<DH, G, 0>(a, st);
     gsa_bwd_range_cuts_kernel<<<(unsigned)((a.rr.rows() + 7) / 8), 256, 0, st>>>(a.idx, a.kt, const_cast<int32_t*>(a.cuts), a.rr,
                                                                                   a.il, a.Lq, a.k_max, a.n_ranges, a.range_keys);

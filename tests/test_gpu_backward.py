@@ -61,12 +61,12 @@ def _run_bwd(cfg, d, idx, kt, dout, q0, q1, key_range=16384, saved_lse=False, **
                                   dQ, dK, dV, dg1, dg2, ws, pbar=pbar, lse=lse)
     torch.cuda.synchronize()
     assert gsa.gsa_device_status(ws) == 0
-    # value gate, query-major kernel, count + 3 scan steps, one fill per range of 8192 query rows, key-major
+    # value gate, preparation kernel, query-major kernel, count + 3 scan steps, one fill per range of 8192 query rows, key-major
     # kernel, and with several ranges the post-pass
     n_ranges = (q1 - q0 + 8191) // 8192
     key_ranges = (cfg.Lk + key_range - 1) // key_range          # of the query-major half (as in the forward pass)
     extra = (2 if saved_lse else 3) if key_ranges > 1 else 0    # range cuts, statistics launch (unless saved), dQ rounding pass
-    assert gsa.gsa_launch_count() - n0 == 7 + n_ranges + (1 if n_ranges > 1 else 0) + extra
+    assert gsa.gsa_launch_count() - n0 == 8 + n_ranges + (1 if n_ranges > 1 else 0) + extra
     return dict(dQ=dQ, dg1=dg1, dK=dK, dV=dV, dg2=dg2, pbar=pbar, lse=lse)
 
 
