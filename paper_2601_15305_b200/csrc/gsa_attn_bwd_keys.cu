@@ -16,7 +16,7 @@
 // bits from run to run.
 // Bound: the gather of Q and do, 2 * n_h * d_h * 2 bytes per selected (query, key) pair.  For more than
 // kBwdRangeRows query rows per sequence the rows are cut into ranges whose Q and do (8 KB per row at 16
-// heads of 128) fit the L2: the lists are filled range by range, so each list is grouped by range, and the
+// heads of 128) fit the L2 with room to spare: the lists are filled range by range, so each list is grouped by range, and the
 // work items run range-major, (range, key), so that the warps in flight share one range.  The partial
 // sums of a key's ranges then meet in fp32 arrays (one reduction per range and element, not per pair) and
 // a streaming post-pass applies the gate's derivative and rounds.
@@ -27,7 +27,7 @@ namespace gsa {
 namespace {
 
 constexpr int kKeyWarps = 4;
-constexpr int kBwdRangeRows = 8192;                  // query rows per range: 64 MB of Q and do at 16 x 128
+constexpr int kBwdRangeRows = 4096;                  // query rows per range: 32 MB of Q and do at 16 x 128 (measured best of 2048 .. 8192)
 constexpr int kBwdMaxRanges = 64;
 constexpr int kScanThreads = 1024;
 constexpr int kScanPerThread = 4;

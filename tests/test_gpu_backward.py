@@ -61,9 +61,9 @@ def _run_bwd(cfg, d, idx, kt, dout, q0, q1, key_range=16384, saved_lse=False, **
                                   dQ, dK, dV, dg1, dg2, ws, pbar=pbar, lse=lse)
     torch.cuda.synchronize()
     assert gsa.gsa_device_status(ws) == 0
-    # value gate, preparation kernel, query-major kernel, count + 3 scan steps, one fill per range of 8192 query rows, key-major
+    # value gate, preparation kernel, query-major kernel, count + 3 scan steps, one fill per range of 4096 query rows, key-major
     # kernel, and with several ranges the post-pass
-    n_ranges = (q1 - q0 + 8191) // 8192
+    n_ranges = (q1 - q0 + 4095) // 4096
     key_ranges = (cfg.Lk + key_range - 1) // key_range          # of the query-major half (as in the forward pass)
     extra = (2 if saved_lse else 3) if key_ranges > 1 else 0    # range cuts, statistics launch (unless saved), dQ rounding pass
     assert gsa.gsa_launch_count() - n0 == 8 + n_ranges + (1 if n_ranges > 1 else 0) + extra
@@ -204,7 +204,7 @@ def test_attn_backward_with_statistics_saved_by_the_forward(key_range):
 
 
 def test_attn_backward_several_query_ranges():
-    """More than 8192 query rows: the key lists are built and walked range by range and the ranges'
+    """More than 4096 query rows (here three ranges): the key lists are built and walked range by range and the ranges'
     partial sums meet in fp32 arrays."""
     cfg = CONFIGS["tiny"].with_(name="bwd_ranges", B=1, Lq=8192 + 777, Lk=8192 + 777, n_h=4, n_kv=2, d_h=64,
                                 k_base=32, k_min=8, k_max=48, seed=41)
