@@ -7,7 +7,20 @@
 
 namespace gsa {
 
-int64_t g_launches = 0;
+std::atomic<int64_t> g_launches{0};
+
+int sm_count() {
+    constexpr int kMaxDevices = 64;
+    static std::atomic<int> cache[kMaxDevices];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 148;
+    int n = cache[dev].load(std::memory_order_relaxed);
+    if (n <= 0) {
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cache[dev].store(n, std::memory_order_relaxed);
+    }
+    return n;
+}
 static int32_t g_indexer_path = 0;
 static cudaEvent_t g_prof_ev[3] = {nullptr, nullptr, nullptr};
 
@@ -603,7 +616,7 @@ int gsa_select_fallback_rows(const void* ws, void* stream, int32_t* rows_out) {
     return GSA_OK;
 }
 
-int64_t gsa_launch_count(void) { return g_launches; }
+int64_t gsa_launch_count(void) { return g_launches.load(); }
 
 void gsa_debug_set_indexer_path(int32_t path) { g_indexer_path = path; }
 

@@ -488,17 +488,6 @@ __global__ void __launch_bounds__(256) gsa_value_gate_kernel(const uint4* __rest
     }
 }
 
-int sm_count() {
-    static int n = 0;
-    if (!n) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-            n = 148;
-    }
-    return n;
-}
-
 int g_range_keys = kRangeKeysDefault;
 
 struct AttnPlan {
@@ -628,7 +617,7 @@ cudaError_t launch_value_gate(const __nv_bfloat16* V, const __nv_bfloat16* g2, _
                               int64_t n_elems, cudaStream_t st) {
     const int64_t n_vec = n_elems / 8;
     if (n_vec <= 0) return cudaSuccess;
-    const int blocks = (int)((n_vec + 255) / 256 < 148 * 16 ? (n_vec + 255) / 256 : 148 * 16);
+    const int blocks = (int)((n_vec + 255) / 256 < sm_count() * 16 ? (n_vec + 255) / 256 : sm_count() * 16);
     gsa_value_gate_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(V),
                                                   reinterpret_cast<const uint4*>(g2),
                                                   reinterpret_cast<uint4*>(Vg), n_vec);

@@ -127,7 +127,7 @@ __global__ void __launch_bounds__(256) gsa_bwd_range_cuts_kernel(const int32_t* 
     if (lr >= rr.rows()) return;
     const int b = rr.b0 + (int)(lr / rr.R), t = rr.q_begin + (int)(lr % rr.R);
     const int64_t irow = il.row(b, t);
-    const int ke = kt[irow];
+    const int ke = clamp_budget(kt[irow], k_max);
     const int32_t* __restrict__ S = idx + irow * k_max;
     int32_t* const out = cuts + ((int64_t)b * Lq + t) * (n_ranges + 1);
     for (int c = 0; c <= n_ranges; ++c) {
@@ -167,7 +167,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32, 4) gsa_sparse_attn_bwd_kernel(
     const int t = a.rr.q_begin + lr % a.rr.R;
     const int64_t qrow = (int64_t)b * a.Lq + t;
     const int64_t irow = a.il.row(b, t);
-    const int ke_all = a.kt[irow];
+    const int ke_all = clamp_budget(a.kt[irow], a.k_max);
     const int32_t* __restrict__ S = a.idx + irow * a.k_max;
     // this item's part of the index set: positions [j_lo, ke)
     int j_lo = 0, ke = ke_all;
@@ -262,7 +262,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32, 4) gsa_sparse_attn_bwd_kernel(
     int32_t pos_fetched = 0;                              // positions of the tile fetched last (lanes 0..15)
     auto fetch = [&](int j, int stage) {
         if (j < ke) {
-            pos_fetched = S[min(j + (lane & 15), ke - 1)];
+            pos_fetched = clamp_pos(S[min(j + (lane & 15), ke - 1)], a.Lk);
             fetch_tile(kbase, st_s32 + stage * STAGE, pos_fetched);
         }
         cp_async_commit();                                // (possibly empty: keeps the group count uniform)

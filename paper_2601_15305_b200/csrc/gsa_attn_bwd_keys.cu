@@ -50,9 +50,12 @@ __global__ void __launch_bounds__(256) gsa_bwd_count_kernel(const InvArgs a, int
     if (lr >= a.rr.rows()) return;
     const int b = a.rr.b0 + (int)(lr / a.rr.R), t = a.rr.q_begin + (int)(lr % a.rr.R);
     const int64_t irow = a.il.row(b, t);
-    const int ke = a.kt[irow];
+    const int ke = clamp_budget(a.kt[irow], a.k_max);
     const int32_t* __restrict__ S = a.idx + irow * a.k_max;
-    for (int j = lane; j < ke; j += 32) atomicAdd(cnt + (int64_t)b * a.Lk + S[j], 1);
+    for (int j = lane; j < ke; j += 32) {
+        const int32_t s = S[j];
+        if (key_in_range(s, a.Lk)) atomicAdd(cnt + (int64_t)b * a.Lk + s, 1);
+    }
 }
 
 // one warp per query row: the row's number goes into the list of every selected key
@@ -63,11 +66,13 @@ __global__ void __launch_bounds__(256) gsa_bwd_fill_kernel(const InvArgs a, int3
     if (lr >= a.rr.rows()) return;
     const int b = a.rr.b0 + (int)(lr / a.rr.R), t = a.rr.q_begin + (int)(lr % a.rr.R);
     const int64_t irow = a.il.row(b, t);
-    const int ke = a.kt[irow];
+    const int ke = clamp_budget(a.kt[irow], a.k_max);
     const int32_t* __restrict__ S = a.idx + irow * a.k_max;
     const int32_t qrow = b * a.Lq + t;
     for (int j = lane; j < ke; j += 32) {
-        const int32_t pos = atomicAdd(cur + (int64_t)b * a.Lk + S[j], 1);
+        const int32_t s = S[j];
+        if (!key_in_range(s, a.Lk)) continue;             // (the same entries the count skipped)
+        const int32_t pos = atomicAdd(cur + (int64_t)b * a.Lk + s, 1);
         rows_of_key[pos] = qrow;
     }
 }
@@ -488,7 +493,7 @@ cudaError_t launch_sparse_attn_bwd_keys(const gsa_params_t& p, RowRange rr, cons
     {
         const int64_t n_elems = (int64_t)n_kv_elems;
         const int64_t want = (n_elems / 4 + 255) / 256;
-        const int blocks = (int)(want < 148 * 16 ? want : 148 * 16);
+        const int blocks = (int)(want < sm_count() * 16 ? want : sm_count() * 16);
         gsa_attn_bwd_finish_kernel<<<blocks, 256, 0, st>>>(dK32, dV32, V, g2, dK, dV, dg2, n_elems);
         ++g_launches;
     }

@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "gsa.h"
 
 namespace gsa {
@@ -32,7 +34,10 @@ constexpr int kStatusFallbackWord = 1;   // int32 word: rows on which top-k sele
 enum : int32_t { kDevOk = 0, kDevTimeoutTma = 1, kDevTimeoutMma = 2, kDevTimeoutEpi = 3,
                  kDevTimeoutGather = 4, kDevTimeoutAttn = 5 };
 
-extern int64_t g_launches;          // host-side launch counter
+extern std::atomic<int64_t> g_launches;   // host-side launch counter (any host thread may launch)
+
+// multiprocessors of the current device (cached per device; 148 if the query fails)
+int sm_count();
 
 // ---- stage launchers (host) ----------------------------------------------------------------
 cudaError_t launch_indexer(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* qI,
@@ -125,6 +130,14 @@ cudaError_t launch_gemm_bf16(int M, int K, int N, const __nv_bfloat16* A, const 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return (uint32_t)__cvta_generic_to_shared(p);
 }
+
+// Index sets and budgets come from the caller.  Every kernel that takes them applies the same rule, so that a
+// corrupt set cannot take an access out of its tensor: the budget is clamped to [0, k_max]; a position used
+// as a gather address is clamped into [0, Lk); an entry that would be scattered to (counters, lists) is
+// skipped unless it lies in [0, Lk).
+__device__ __forceinline__ int32_t clamp_budget(int32_t kt, int32_t k_max) { return min(max(kt, 0), k_max); }
+__device__ __forceinline__ int32_t clamp_pos(int32_t s, int32_t Lk) { return min(max(s, 0), Lk - 1); }
+__device__ __forceinline__ bool key_in_range(int32_t s, int32_t Lk) { return (uint32_t)s < (uint32_t)Lk; }
 
 __device__ __forceinline__ float fast_sigmoid(float x) {
     // 1 / (1 + 2^(-x log2 e)); ex2.approx and rcp.approx are accurate to a few ulp

@@ -80,7 +80,7 @@ __global__ void __launch_bounds__(kLossWarps * 32) gsa_attn_probs_mean_kernel(co
     const int b = a.rr.b0 + lr / a.rr.R, t = a.rr.q_begin + lr % a.rr.R;
     const int64_t qrow = (int64_t)b * a.Lq + t;
     const int64_t irow = a.il.row(b, t);
-    const int ke = a.kt[irow];
+    const int ke = clamp_budget(a.kt[irow], a.k_max);
     const int32_t* __restrict__ S = a.idx + irow * a.k_max;
     float* __restrict__ prow = a.pbar + irow * a.k_max;
 
@@ -107,7 +107,7 @@ __global__ void __launch_bounds__(kLossWarps * 32) gsa_attn_probs_mean_kernel(co
     const __nv_bfloat16* const kbase = a.K + ((size_t)b * a.Lk * a.n_kv + g) * DH;
     auto fetch = [&](int j, int stage) {
         if (j < ke) {
-            const int32_t pos16 = S[min(j + (lane & 15), ke - 1)];
+            const int32_t pos16 = clamp_pos(S[min(j + (lane & 15), ke - 1)], a.Lk);
 #pragma unroll
             for (int i = 0; i < 16 * CPR / 32; ++i) {
                 const int chunk = i * 32 + lane;
@@ -229,7 +229,7 @@ __global__ void __launch_bounds__(kLossWarps * 32) gsa_indexer_kl_kernel(const K
     const int b = a.rr.b0 + lr / a.rr.R, t = a.rr.q_begin + lr % a.rr.R;
     const int64_t qrow = (int64_t)b * a.Lq + t;
     const int64_t irow = a.il.row(b, t);
-    const int ke = a.kt[irow];
+    const int ke = clamp_budget(a.kt[irow], a.k_max);
     const int32_t* __restrict__ S = a.idx + irow * a.k_max;
     const float* __restrict__ prow = a.pbar + irow * a.k_max;
 
@@ -260,7 +260,7 @@ __global__ void __launch_bounds__(kLossWarps * 32) gsa_indexer_kl_kernel(const K
     const __nv_bfloat16* const kbase = a.kI + (size_t)b * a.Lk * DI;
     auto fetch = [&](int j, int stage) {
         if (j < ke) {
-            const int32_t pos16 = S[min(j + (lane & 15), ke - 1)];
+            const int32_t pos16 = clamp_pos(S[min(j + (lane & 15), ke - 1)], a.Lk);
 #pragma unroll
             for (int i = 0; i < 16 * CPR / 32; ++i) {
                 const int chunk = i * 32 + lane;
@@ -344,7 +344,7 @@ __global__ void __launch_bounds__(kLossWarps * 32) gsa_indexer_kl_kernel(const K
     float dw_acc[2] = {0.f, 0.f}, db_acc[2] = {0.f, 0.f};
     fetch(0, 0);
     for (int j0 = 0, stage = 0; j0 < ke; j0 += 16, stage ^= 1) {
-        const int32_t pos16 = S[min(j0 + (lane & 15), ke - 1)];
+        const int32_t pos16 = clamp_pos(S[min(j0 + (lane & 15), ke - 1)], a.Lk);
         fetch(j0 + 16, stage ^ 1);
         const bool v0 = j0 + gid < ke, v1 = j0 + gid + 8 < ke;
         const float p0 = v0 ? prow[j0 + gid] : 0.f, p1 = v1 ? prow[j0 + gid + 8] : 0.f;
@@ -498,7 +498,7 @@ cudaError_t launch_indexer_kl(const gsa_params_t& p, RowRange rr, const __nv_bfl
         if (e != cudaSuccess) return e;
     }
     const int64_t want = (n_k / 4 + 255) / 256;
-    gsa_f32_to_bf16_kernel<<<(int)(want < 148 * 16 ? (want > 0 ? want : 1) : 148 * 16), 256, 0, st>>>(dkI32, dkI, n_k);
+    gsa_f32_to_bf16_kernel<<<(int)(want < sm_count() * 16 ? (want > 0 ? want : 1) : sm_count() * 16), 256, 0, st>>>(dkI32, dkI, n_k);
     ++g_launches;
     return cudaGetLastError();
 }

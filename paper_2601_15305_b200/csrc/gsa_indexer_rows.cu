@@ -128,7 +128,7 @@ cudaError_t launch_rows_t(const gsa_params_t& p, RowRange rr, const RowsIdxArgs&
     RowsIdxArgs a = a0;
     const int n_max = p.Lk - p.Lq + rr.q_begin + rr.R;
     // enough CTAs to fill the GPU about four times over, each with a run of keys long enough to stream
-    const int64_t want_ctas = 148 * 4;
+    const int64_t want_ctas = (int64_t)sm_count() * 4;
     int64_t per = ((int64_t)n_max * rr.rows() + want_ctas - 1) / want_ctas;
     const int step = kRowsWarps * 16 * kTilesPerStep;
     per = (per + step - 1) / step * step;

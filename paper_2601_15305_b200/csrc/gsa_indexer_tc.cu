@@ -313,7 +313,7 @@ cudaError_t launch_t(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* qI
     const int tiles_max = (n_vis_max + kTileKeys - 1) / kTileKeys;
     // enough CTAs to fill the GPU a few times over, but runs long enough to amortise the q^I load
     int64_t total_tiles = (int64_t)groups * tiles_max;
-    int tpc = (int)(total_tiles / (148 * 4));
+    int tpc = (int)(total_tiles / (sm_count() * 4));
     tpc = tpc < 4 ? 4 : (tpc > 64 ? 64 : tpc);
     a.tiles_per_cta = tpc;
     dim3 grid((tiles_max + tpc - 1) / tpc, groups);

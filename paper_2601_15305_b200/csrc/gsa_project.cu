@@ -225,8 +225,7 @@ cudaError_t launch_project(const gsa_params_t& p, int d_model, const __nv_bfloat
     if (!make_kblock_tmap(&tm_w, Wt, (uint64_t)a.N, (uint64_t)a.K, kTileN)) return cudaErrorUnknown;
     cudaError_t e = cudaFuncSetAttribute(gsa_project_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal);
     if (e != cudaSuccess) return e;
-    int sms = 148, dev = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = sm_count();
     const int tiles = a.m_tiles * a.n_tiles;
     gsa_project_kernel<<<tiles < sms ? tiles : sms, kPThreads, kSmemTotal, st>>>(tm_h, tm_w, a);
     ++g_launches;
@@ -249,8 +248,7 @@ cudaError_t launch_gemm_bf16(int M, int K, int N, const __nv_bfloat16* A, const 
     if (!make_kblock_tmap(&tm_b, Bt, (uint64_t)N, (uint64_t)K, kTileN)) return cudaErrorUnknown;
     cudaError_t e = cudaFuncSetAttribute(gsa_project_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal);
     if (e != cudaSuccess) return e;
-    int sms = 148, dev = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = sm_count();
     const int tiles = a.m_tiles * a.n_tiles;
     gsa_project_kernel<<<tiles < sms ? tiles : sms, kPThreads, kSmemTotal, st>>>(tm_a, tm_b, a);
     ++g_launches;

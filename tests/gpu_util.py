@@ -78,6 +78,7 @@ def run_forward(cfg, d, slab_rows=0, bI=None, want_idx=True, k_mode=0, **over):
     kt = torch.full((cfg.B, cfg.Lq), -7, device="cuda", dtype=torch.int32)
     var = torch.empty((cfg.B, cfg.Lq), device="cuda", dtype=torch.float32)
     ws = torch.empty(gsa.gsa_workspace_bytes(p, slab_rows), dtype=torch.uint8, device="cuda")
+    ws.fill_(0xFF)        # the path must not rely on a cleared workspace (0xFF..: NaN as fp32, -1 as int32)
     gsa.gsa_forward(p, d["Q"], d["K"], d["V"], d["qI"], d["kI"], d["w"], bI, d["g1"], d["g2"], out, idx, kt, var,
                     slab_rows, ws)
     assert gsa.gsa_device_status(ws) == 0
@@ -121,26 +122,64 @@ def check_out(got: np.ndarray, want: np.ndarray):
     assert (err <= OUT_REL_TO_ROWMAX_TOL * rowmax + 1e-6).all(), (err / (rowmax + 1e-30)).max()
 
 
-def check_e2e_indices(o: dict, idx: np.ndarray, kt: np.ndarray, oracle_scores: np.ndarray, n_vis):
+def check_e2e_indices(o: dict, idx: np.ndarray, kt: np.ndarray, oracle_scores: np.ndarray, n_vis, mism_rows=None):
     """End to end, an index may differ from the oracle's only where the two candidates' oracle scores
-    differ by less than 1e-5 (fp32 vs fp64 scoring)."""
+    differ by less than 1e-5 (fp32 vs fp64 scoring).  Returns the number of rows whose sets differ (their
+    positions are appended to mism_rows)."""
     mism = 0
     for i, n in enumerate(n_vis):
         kg, ko = int(kt[i]), int(o["keff"][i])
-        sg, so = set(idx[i, :kg].tolist()), set(o["idx"][i, :ko].tolist())
+        g_idx = idx[i, :kg]
+        assert (g_idx[1:] > g_idx[:-1]).all() and (kg == 0 or (g_idx[0] >= 0 and g_idx[-1] < n)), i
+        assert (idx[i, kg:] == -1).all(), i
+        sg = set(g_idx.tolist())
+        sc = oracle_scores[i]
         if kg != ko:
-            # budget flipped across an integer because the fp32 scores shift the variance slightly
+            # The budget may flip across an integer because the fp32 scores shift the variance slightly: by one,
+            # and only where k_base * Var / v_bar sits next to an integer.  Top-k sets under a total order are
+            # nested, so the GPU's set is then judged against the oracle's top-k_gpu, taken from the oracle's own
+            # fp64 scores in the oracle's order (score descending, position ascending).
             r = o["r"][i]
-            assert abs(kg - ko) <= 1 and abs(r - round(r)) < 1e-2, (i, kg, ko, r)
+            assert abs(kg - ko) == 1 and abs(r - round(r)) < 1e-2, (i, kg, ko, r)
+            order = np.lexsort((np.arange(n), -sc[:n]))
+            assert set(order[:ko].tolist()) == set(o["idx"][i, :ko].tolist()), i     # same order as the oracle's
+            so = set(order[:kg].tolist())
+        else:
+            so = set(o["idx"][i, :ko].tolist())
         only_g, only_o = sorted(sg - so), sorted(so - sg)
-        if not only_g and not only_o:
+        assert len(only_g) == len(only_o)
+        if not only_g:
             continue
         mism += 1
-        sc = oracle_scores[i]
-        # every swapped pair must be a near-tie at the selection boundary
+        if mism_rows is not None:
+            mism_rows.append(i)
+        # every swapped pair must be a near-tie at the selection boundary: the best score swapped out and
+        # the worst score swapped in bound every pair's gap
         lo = min(sc[j] for j in (only_g + only_o))
         hi = max(sc[j] for j in (only_g + only_o))
-        if kg == ko:
-            assert hi - lo < E2E_SCORE_GAP, (i, only_g, only_o, hi - lo)
-        assert all(0 <= j < n for j in sg)
+        assert hi - lo < E2E_SCORE_GAP, (i, kg, ko, only_g, only_o, hi - lo)
+    return mism
+
+
+def check_forward_rows(p: oracle.OracleParams, x: dict, o: dict, out_rows: np.ndarray, idx_rows: np.ndarray,
+                       kt_rows: np.ndarray, rows_t, rows_b, n_vis):
+    """gsa_forward against the oracle on the listed rows: the index rule, the stated 2e-2 max-abs bound on the
+    outputs end to end, and the tighter bound relative to each row's largest magnitude.  With the workloads'
+    nearly flat attention a row's output is about |v| / sqrt(k), while swapping one selected key for its
+    near-tie (which the index rule allows) moves it by about 2 |v| / k: several per cent of the output at
+    k = 2048..4096.  The tighter bound therefore judges such a row against the oracle's attention stage
+    evaluated on the index set the GPU selected.  o = oracle.forward(..., want_scores=True) for the rows."""
+    rows_t = np.asarray(rows_t)
+    rows_b = np.zeros_like(rows_t) if rows_b is None else np.asarray(rows_b)
+    bad: list = []
+    mism = check_e2e_indices(o, idx_rows, kt_rows, o["scores"], n_vis, mism_rows=bad)
+    got = out_rows.astype(np.float64)
+    assert np.isfinite(got).all()
+    assert np.abs(got - o["out"]).max() <= OUT_MAX_ABS_TOL
+    want = o["out"]
+    if bad:
+        want = want.copy()
+        b = np.asarray(bad)
+        want[b] = oracle.attn(p, x["Q"], x["K"], x["V"], x["g1"], x["g2"], idx_rows[b], kt_rows[b], rows_t[b], rows_b[b])
+    check_out(out_rows, want)
     return mism

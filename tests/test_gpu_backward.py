@@ -297,10 +297,18 @@ def _check_loss_path(cfg, q0, q1, seed, bias=False, act=0, **over):
         assert (got_p[r, kt1[r]:] == 0).all()
 
     bI = torch.tensor([0.3, -0.2, 0.1, 0.0, -0.4, 0.25, 0.05, -0.1][: cfg.HI]) if bias else None
+    _compare_kl(cfg, x, d, p, bI, idx, kt, want_p, q0, q1, act=act, **over)
+
+
+def _compare_kl(cfg, x, d, p, bI, idx, kt, want_p, q0, q1, **over):
+    """gsa_indexer_kl_bwd against the oracle, both fed the oracle's target rounded to fp32."""
+    R = q1 - q0
+    rows_b, rows_t = np.repeat(np.arange(cfg.B), R), np.tile(np.arange(q0, q1), cfg.B)
+    idx2, kt1 = idx.reshape(cfg.B * R, -1).numpy(), kt.reshape(-1).numpy()
     pb32 = want_p.astype(np.float32)
     want = oracle.indexer_kl(p, x["qI"], x["kI"], x["w"], bI, idx2, kt1, pb32.astype(np.float64), rows_t, rows_b)
     got = _run_kl(cfg, d, None if bI is None else bI.cuda(), idx.cuda(), kt.cuda(),
-                  torch.from_numpy(pb32).reshape(cfg.B, R, -1).cuda(), q0, q1, act=act, **over)
+                  torch.from_numpy(pb32).reshape(cfg.B, R, -1).cuda(), q0, q1, **over)
     gl = got["loss"].cpu().numpy().reshape(-1)
     # the loss is a difference of O(log k) terms held in fp32
     assert (np.abs(gl - want["loss"]) <= 2e-3 * np.abs(want["loss"]) + 2e-5).all(), np.abs(gl - want["loss"]).max()
@@ -360,3 +368,43 @@ def test_indexer_warmup_loss_on_all_visible_keys():
     assert (np.abs(gl - want["loss"]) <= 2e-3 * np.abs(want["loss"]) + 2e-5).all()
     g, w = got["dkI"].float().cpu().numpy(), want["dkI"]
     assert np.linalg.norm(g - w) <= GRAD_FROBENIUS_TOL * np.linalg.norm(w)
+
+
+# ------------------------------------------------------------------------- the benchmark's geometry
+def test_backward_and_indexer_loss_at_the_benchmark_geometry():
+    """The launch plan `bench.py --backward` times, checked against the oracle: the l128k workload with the
+    default range sizes (8 key ranges of 16384 keys in the query-major half, 2 query ranges of 4096 rows in
+    the key-major half), index sets taken from the real forward pass, gradients of the last 4200 query rows.
+    dQ and dg1 on every row of the range; dK, dV, dg2, the loss target and dk^I on every key."""
+    cfg = CONFIGS["l128k"]
+    x = make_inputs(cfg)
+    d = U.to_dev(x)
+    _, idx_all, kt_all, _ = U.run_forward(cfg, d)
+    q0, q1 = cfg.Lq - 4200, cfg.Lq
+    idx = idx_all[:, q0:q1].contiguous()
+    kt = kt_all[:, q0:q1].contiguous()
+    del idx_all
+    g = torch.Generator().manual_seed(71)
+    dout = torch.zeros_like(d["Q"])
+    dout_rows = (torch.randn((cfg.B, q1 - q0, cfg.n_h, cfg.d_h), generator=g) * 0.25).to(torch.bfloat16)
+    dout[:, q0:q1] = dout_rows.cuda()
+    got = _run_bwd(cfg, d, idx, kt, dout, q0, q1)
+    idx_c, kt_c = idx.cpu(), kt.cpu()
+    dout_c = torch.zeros((cfg.B, cfg.Lq, cfg.n_h, cfg.d_h), dtype=torch.bfloat16)
+    dout_c[:, q0:q1] = dout_rows
+    _compare(cfg, x, got, idx_c, kt_c, dout_c, q0, q1)
+    # the same gradients when the forward call saved its softmax statistics (first sweep skipped)
+    got2 = _run_bwd(cfg, d, idx, kt, dout, q0, q1, saved_lse=True)
+    for name in ("dQ", "dg1"):
+        a, b = got[name][:, q0:q1].float(), got2[name][:, q0:q1].float()
+        assert (a - b).abs().max().item() <= 2.0 ** -7 * a.abs().max().item(), name
+    for name in ("dK", "dV", "dg2"):
+        a, b = got[name].float(), got2[name].float()
+        assert (a - b).abs().max().item() <= 2.0 ** -7 * a.abs().max().item(), name
+    del got2
+    # the indexer's loss on the same index sets
+    R = q1 - q0
+    p = U.oracle_params(cfg)
+    want_p = oracle.attn_probs_mean(p, x["Q"], x["K"], idx_c.reshape(cfg.B * R, -1).numpy(), kt_c.reshape(-1).numpy(),
+                                    np.tile(np.arange(q0, q1), cfg.B), np.repeat(np.arange(cfg.B), R))
+    _compare_kl(cfg, x, d, p, None, idx_c, kt_c, want_p, q0, q1)

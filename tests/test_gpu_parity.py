@@ -340,8 +340,8 @@ def _forward_and_compare(cfg, x, d, rows, slab_rows=0, **kw):
     sel = torch.from_numpy(rows).cuda()
     p = U.oracle_params(cfg, **kw)
     o = oracle.forward(p, **x, rows_t=rows, want_scores=True)
-    mism = U.check_e2e_indices(o, idx[0][sel].cpu().numpy(), kt[0][sel].cpu().numpy(), o["scores"], _vis(cfg, rows))
-    U.check_out(out[0][sel].float().cpu().numpy(), o["out"])
+    mism = U.check_forward_rows(p, x, o, out[0][sel].float().cpu().numpy(), idx[0][sel].cpu().numpy(),
+                                kt[0][sel].cpu().numpy(), rows, None, _vis(cfg, rows))
     assert not torch.isnan(out.float()).any()
     return mism, kt
 
@@ -420,8 +420,8 @@ def test_forward_batched_chunked_prefill():
     for b in range(cfg.B):
         rows = np.arange(0, cfg.Lq, 5)
         o = oracle.forward(p, **x, rows_t=rows, rows_b=np.full_like(rows, b), want_scores=True)
-        U.check_e2e_indices(o, idx[b][rows].cpu().numpy(), kt[b][rows].cpu().numpy(), o["scores"], _vis(cfg, rows))
-        U.check_out(out[b][rows].float().cpu().numpy(), o["out"])
+        U.check_forward_rows(p, x, o, out[b][rows].float().cpu().numpy(), idx[b][rows].cpu().numpy(),
+                             kt[b][rows].cpu().numpy(), rows, np.full_like(rows, b), _vis(cfg, rows))
 
 
 def test_forward_small_decode_batch():
@@ -433,12 +433,13 @@ def test_forward_small_decode_batch():
     p = U.oracle_params(cfg)
     rows_b = np.arange(cfg.B)
     o = oracle.forward(p, **x, rows_t=np.zeros(cfg.B, np.int32), rows_b=rows_b, want_scores=True)
-    U.check_e2e_indices(o, idx[:, 0].cpu().numpy(), kt[:, 0].cpu().numpy(), o["scores"], [cfg.Lk] * cfg.B)
-    U.check_out(out[:, 0].float().cpu().numpy(), o["out"])
+    U.check_forward_rows(p, x, o, out[:, 0].float().cpu().numpy(), idx[:, 0].cpu().numpy(), kt[:, 0].cpu().numpy(),
+                         np.zeros(cfg.B, np.int64), rows_b, [cfg.Lk] * cfg.B)
 
 
-def test_forward_is_deterministic(tiny):
-    cfg, x, d = tiny
+@pytest.mark.parametrize("which", ["tiny", "l8k"])
+def test_forward_is_deterministic(which, request):
+    cfg, x, d = request.getfixturevalue(which)
     a = U.run_forward(cfg, d)
     b = U.run_forward(cfg, d)
     assert torch.equal(a[1], b[1]) and torch.equal(a[2], b[2])
@@ -484,8 +485,8 @@ def test_forward_many_key_ranges_device_and_host_paths():
     for b in range(cfg.B):
         rows = np.array([0, 5, 1023, 1024, 1500, 2047, 2048, 2999])
         o = oracle.forward(po, **x, rows_t=rows, rows_b=np.full_like(rows, b), want_scores=True)
-        U.check_e2e_indices(o, idx[b][rows].cpu().numpy(), kt[b][rows].cpu().numpy(), o["scores"], _vis(cfg, rows))
-        U.check_out(out[b][rows].float().cpu().numpy(), o["out"])
+        U.check_forward_rows(po, x, o, out[b][rows].float().cpu().numpy(), idx[b][rows].cpu().numpy(),
+                             kt[b][rows].cpu().numpy(), rows, np.full_like(rows, b), _vis(cfg, rows))
 
 
 def test_argument_errors_do_not_launch(tiny):
@@ -515,7 +516,7 @@ def test_forward_l32k_sampled_rows_budgets_span_the_clamp_range():
     cfg = CONFIGS["l32k"]
     x = make_inputs(cfg)
     d = U.to_dev(x)
-    mism, kt = _forward_and_compare(cfg, x, d, sample_rows(cfg, 24).numpy())
+    mism, kt = _forward_and_compare(cfg, x, d, sample_rows(cfg, 256).numpy())
     k = kt[0, cfg.k_max:].cpu().numpy()
     assert k.min() == cfg.k_min and k.max() == cfg.k_max          # heterogeneous variance: both clamps are hit
     assert ((k > cfg.k_min) & (k < cfg.k_max)).mean() > 0.3
@@ -524,10 +525,11 @@ def test_forward_l32k_sampled_rows_budgets_span_the_clamp_range():
 def test_stages_l128k_sampled_rows(l128k):
     """Stage by stage at L = 131072: scores of a block of late rows, bit-exact selection on those fp32 scores."""
     cfg, x, d = l128k
-    for q0 in (70000, cfg.Lq - 48):
+    for q0 in (9000, 40000, 70000, 101000, cfg.Lq - 48):      # 5 blocks x 16 rows = 80 rows
         q1 = q0 + 48
         sc = U.run_scores(cfg, d, q_begin=q0, q_end=q1)
-        rows = np.array([q0, q0 + 17, q1 - 1])
+        rows = q0 + np.arange(0, 48, 3)
+        rows[-1] = q1 - 1
         got = sc[0][torch.from_numpy(rows - q0).cuda()].cpu().numpy()
         want = oracle.scores(U.oracle_params(cfg), x["qI"], x["kI"], x["w"], None, rows)
         U.check_scores(got, want, _vis(cfg, rows))
@@ -539,7 +541,7 @@ def test_stages_l128k_sampled_rows(l128k):
 
 def test_forward_l128k_sampled_rows(l128k):
     cfg, x, d = l128k
-    mism, kt = _forward_and_compare(cfg, x, d, sample_rows(cfg, 16).numpy())
+    mism, kt = _forward_and_compare(cfg, x, d, sample_rows(cfg, 256).numpy())
     k = kt[0, cfg.k_max:].float()
     assert k.min() >= cfg.k_min and k.max() <= cfg.k_max and 1500 < k.mean() < 3000
 
@@ -564,8 +566,8 @@ def test_forward_decode_full_size():
     cfg1 = cfg.with_(B=1)
     for b in checked:
         o = oracle.forward(U.oracle_params(cfg1), **host[b], rows_t=np.zeros(1, np.int32), want_scores=True)
-        U.check_e2e_indices(o, idx[b].cpu().numpy(), kt[b].cpu().numpy(), o["scores"], [cfg.Lk])
-        U.check_out(out[b].float().cpu().numpy(), o["out"])
+        U.check_forward_rows(U.oracle_params(cfg1), host[b], o, out[b].float().cpu().numpy(), idx[b].cpu().numpy(),
+                             kt[b].cpu().numpy(), np.zeros(1, np.int64), None, [cfg.Lk])
     assert (kt >= cfg.k_min).all() and (kt <= cfg.k_max).all()
 
 
