@@ -33,6 +33,12 @@ from paper_2601_15305_b200.inputs import CONFIGS, make_inputs, sample_rows
 
 METRIC = "gsa_fwd_tokens_per_s"
 UNIT = "tokens/s"
+# special-function operations the indexer's epilogue spends per sigmoid: one exp2 each and one reciprocal
+# shared by four heads
+SFU_OPS_PER_SIGMOID = 1.25
+# DRAM bytes (read + written) of the sparse-attention launches of one forward, per workload, from the ncu
+# capture named in profiles/; empty while no capture of the current kernels exists
+ATTN_DRAM_TRAFFIC = {}
 
 
 def measured_peaks():
@@ -105,6 +111,51 @@ def attention_bytes(cfg, kt_sum: int) -> float:
     return float(kt_sum) * per_pair + float(cfg.B * cfg.Lq) * per_tok
 
 
+def measure_rates(gsa, stream):
+    """Ceilings no vendor figure gives, measured here with the library's probe kernels (CUDA events on the
+    launching stream, one warm-up launch, best of three): the rate at which 256-byte and 2048-byte row pieces
+    picked by a random index list are gathered out of a 64 MB table (L2-resident, like one key range of K and
+    V' rows) and out of a 2 GB table (HBM), and the special-function unit's exp2 rate."""
+    gen = torch.Generator(device="cuda").manual_seed(7)
+    sink = torch.zeros(64, dtype=torch.int32, device="cuda")
+    out = {}
+
+    def best_ms(fn, reps=3):
+        fn()
+        ts = []
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            fn()
+            e1.record(stream)
+            e1.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        return min(ts)
+
+    row_bytes = 2048
+    for label, table_bytes in (("l2_64MB", 64 << 20), ("hbm_2GB", 2 << 30)):
+        n_rows = table_bytes // row_bytes
+        table = torch.empty(table_bytes, dtype=torch.uint8, device="cuda")
+        table.random_(0, 255, generator=gen)
+        for piece in (256, 2048):
+            n_idx = (2 << 30) // piece
+            idx = torch.randint(0, n_rows, (n_idx,), generator=gen, device="cuda", dtype=torch.int32)
+            ms = best_ms(lambda: gsa.gsa_probe_gather(table, n_rows, row_bytes, piece, idx, sink, stream))
+            out[f"gather_{label}_piece{piece}_gbs"] = n_idx * piece / (ms * 1e-3) / 1e9
+            del idx
+        del table
+    ops = [0]
+
+    def ex2():
+        ops[0] = gsa.gsa_probe_ex2(4096, sink, stream)
+    ms = best_ms(ex2)
+    out["ex2_per_s"] = ops[0] / (ms * 1e-3)
+    out["how"] = ("gsa_probe_gather: random rows of a 2048-byte-row table, first 256 / 2048 bytes of each, plain 32-byte "
+                  "loads, 8 in flight per thread, 2 GiB gathered per launch; gsa_probe_ex2: 8 independent ex2.approx "
+                  "chains per thread, 2048 threads per SM; best of 3 launches after a warm-up")
+    return out
+
+
 def oracle_sample_rate(cfg, x, n_rows: int):
     """tokens/s of the fp64 oracle on a stratified sample of query rows (mean row cost = mean over the sequence)."""
     import oracle
@@ -174,8 +225,10 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-projection", action="store_true", help="skip timing the upstream projection GEMM")
-    ap.add_argument("--backward", action="store_true",
-                    help="also time gsa_sparse_gated_attn_bwd on the workload's own index sets (adds a 'backward' object)")
+    ap.add_argument("--backward", action="store_true", help="(kept for old command lines: the backward leg is on by default)")
+    ap.add_argument("--no-backward", action="store_true",
+                    help="skip timing gsa_sparse_gated_attn_bwd and the indexer loss on the workload's own index sets")
+    ap.add_argument("--no-rates", action="store_true", help="skip the gather-rate and exp2-rate probes")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "gsa_b200" else args.warmup
     cfg = CONFIGS[args.workload]
@@ -262,6 +315,19 @@ def main():
     clocks = sampler.stop()
     gsa.gsa_profile_set_events(None, None, None)
     assert gsa.gsa_device_status(ws) == 0
+    # one more step, outside the timed region, with an event behind every launch: per-kernel times
+    tl_events = [torch.cuda.Event(enable_timing=True) for _ in range(256)]
+    for e in tl_events:
+        e.record(stream)
+    read_timeline = gsa.gsa_profile_set_timeline(tl_events)
+    step()
+    torch.cuda.synchronize()
+    timeline = read_timeline()
+    gsa.gsa_profile_set_timeline(None)
+    stage_ms = {}
+    for name, ms in timeline:
+        stage_ms[name] = stage_ms.get(name, 0.0) + ms
+    stage_launches = {name: sum(1 for n, _ in timeline if n == name) for name in stage_ms}
     ms_local = t_beg.elapsed_time(t_end)
     ms_total, tokens_total = aggregate_over_ranks(ms_local, float(cfg.B * cfg.Lq * args.steps))
     value = tokens_total / (ms_total * 1e-3)
@@ -269,23 +335,85 @@ def main():
     attn_ms = float(np.mean([tri[1].elapsed_time(tri[2]) for tri in evs]))
 
     peaks = measured_peaks()
+    rates = None if args.no_rates else measure_rates(gsa, stream)
     ab = attention_bytes(cfg, kt_sum)
     achieved = ab / (attn_ms * 1e-3) / 1e9
-    # DRAM bytes of the sparse-attention launches of one forward, from the ncu capture summarised in
-    # profiles/gsa_sparse_attn_kernel_l32k_and_l128k_dram.md (l128k, default key ranges); other workloads: not captured
-    traffic = 48.26e9 if (cfg.name == "l128k" and args.slab_rows == 0) else None
-    roofline = {"kernel": "gsa_sparse_attn_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
-                "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": traffic,
-                "peak_source": f"{peaks['source']} (MEASURED_PEAKS.json hbm_gbs)" if peaks["source"] == "measured"
-                else "fallback 6650 GB/s",
+    hbm_src = f"{peaks['source']} (MEASURED_PEAKS.json hbm_gbs)" if peaks["source"] == "measured" else "fallback 6650 GB/s"
+    # The gather of sparse attention is served by the L2 (key ranges of 16384 keys keep a range's K and V' rows
+    # resident), so the ceiling that binds is the L2's gather rate for 256-byte pieces, measured by the probe
+    # above; the fraction of the HBM copy bandwidth is kept beside it.  `traffic` (DRAM bytes of the launch from
+    # an ncu capture) is null: the kernels changed after the last capture.
+    l2_peak = rates["gather_l2_64MB_piece256_gbs"] if rates else None
+    roofline = {"kernel": "gsa_sparse_attn_kernel", "bound": "l2" if rates else "hbm", "achieved": achieved,
+                "peak": l2_peak if rates else peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / (l2_peak if rates else peaks["hbm_gbs"]), "traffic": ATTN_DRAM_TRAFFIC.get(cfg.name)
+                if args.slab_rows == 0 else None,
+                "peak_source": "measured in this run: gsa_probe_gather, random 256-byte pieces of a 64 MB table (L2-resident)"
+                if rates else hbm_src,
+                "l2_gather_gbs": l2_peak, "frac_l2": achieved / l2_peak if rates else None,
+                "hbm_gbs": peaks["hbm_gbs"], "frac_hbm": achieved / peaks["hbm_gbs"], "hbm_source": hbm_src,
+                "hbm_gather_gbs": rates["gather_hbm_2GB_piece256_gbs"] if rates else None,
                 "algorithmic_bytes_per_launch": ab, "launch_ms": attn_ms,
                 "note": "one 'launch' = the sparse-attention stage of a forward (range cuts, one kernel launch per 16384-key "
-                        "range, finalize); frac exceeds 1 because the 126 MB L2, not HBM, serves the gather "
-                        "(ncu: L2 throughput 72% of peak, DRAM traffic 4% of the algorithmic bytes)"}
+                        "range, finalize).  The 126 MB L2, not HBM, serves the gather, so frac is taken against the L2's "
+                        "measured gather rate; frac_hbm (against the HBM copy bandwidth) exceeds 1 for the same reason"}
     causal_pairs = cfg.B * sum(cfg.Lk - cfg.Lq + t + 1 for t in (0, cfg.Lq - 1)) * cfg.Lq / 2.0
     stages = {"indexer_plus_topk_ms": sel_ms, "sparse_attn_ms": attn_ms,
               "indexer_causal_tflop": 2.0 * cfg.HI * cfg.dI * causal_pairs / 1e12,
               "mean_k_t": kt_sum / float(cfg.B * cfg.Lq), "select_fallback_rows": fallback_rows}
+
+    # ---- one object per kernel of the forward, from the per-launch events of the profiling step ----
+    def per_kernel(name):
+        return stage_ms.get(name, 0.0), stage_launches.get(name, 0)
+    roofline_all = {}
+    ms, n = per_kernel("indexer")
+    if n:
+        flop = 2.0 * cfg.HI * cfg.dI * causal_pairs
+        sig = cfg.HI * causal_pairs
+        tf = flop / (ms * 1e-3) / 1e12
+        roofline_all["indexer"] = {
+            "kernel": "gsa_indexer_tc_kernel" if cfg.Lq > 4 else "gsa_indexer_rows_kernel", "ms": ms, "launches": n,
+            "tflops_causal": tf, "bound": "tensor (nominal)", "peak_tflops": peaks["bf16_tflops_sustained"],
+            "frac": tf / peaks["bf16_tflops_sustained"],
+            "sigmoids_per_s": sig / (ms * 1e-3), "sfu_ops_per_sigmoid": SFU_OPS_PER_SIGMOID if variant["act"] == 0 else 0.0,
+            "ex2_per_s_measured": rates["ex2_per_s"] if rates else None,
+            "frac_sfu": (SFU_OPS_PER_SIGMOID * sig / (ms * 1e-3) / rates["ex2_per_s"]) if (rates and variant["act"] == 0) else None,
+            "note": "flops of causal pairs only (2 * H^I * d^I each); the epilogue's H^I sigmoids per pair run on the "
+                    "special-function unit (one exp2 each and one reciprocal shared by the heads), which binds before the tensor pipe"}
+    ms, n = per_kernel("select")
+    if n:
+        gbs = 4.0 * causal_pairs / (ms * 1e-3) / 1e9
+        roofline_all["select"] = {"kernel": "gsa_select_kernel", "ms": ms, "launches": n, "bound": "hbm",
+                                  "achieved_gbs": gbs, "peak_gbs": peaks["hbm_gbs"], "frac": gbs / peaks["hbm_gbs"],
+                                  "note": "4 bytes per causal pair read once; index sets written"}
+    ms, n = per_kernel("value_gate")
+    if n:
+        gbs = 3.0 * 2 * cfg.B * cfg.Lk * cfg.n_kv * cfg.d_h / (ms * 1e-3) / 1e9
+        roofline_all["value_gate"] = {"kernel": "gsa_value_gate_kernel", "ms": ms, "launches": n, "bound": "hbm",
+                                      "achieved_gbs": gbs, "peak_gbs": peaks["hbm_gbs"], "frac": gbs / peaks["hbm_gbs"]}
+    ms, n = per_kernel("sparse_attn")
+    if n:
+        gb = float(kt_sum) * (2 * cfg.n_kv * cfg.d_h * 2 + 4)
+        gbs = gb / (ms * 1e-3) / 1e9
+        roofline_all["sparse_attn"] = {"kernel": "gsa_sparse_attn_kernel", "ms": ms, "launches": n,
+                                       "bound": "l2" if rates else "hbm", "achieved_gbs": gbs,
+                                       "peak_gbs": l2_peak if rates else peaks["hbm_gbs"],
+                                       "frac": gbs / (l2_peak if rates else peaks["hbm_gbs"]),
+                                       "frac_hbm": gbs / peaks["hbm_gbs"],
+                                       "tflops": float(kt_sum) * cfg.n_h * cfg.d_h * 4 / (ms * 1e-3) / 1e12,
+                                       "note": "gathered K and V' rows (+ indices) of the selected pairs; the kernel launches only"}
+    ms, n = per_kernel("finalize")
+    if n:
+        slots = 1
+        state = cfg.B * cfg.Lq * cfg.n_h * (cfg.d_h + 2) * 4.0 * slots
+        gbs = (state + 2.0 * 2 * cfg.B * cfg.Lq * cfg.n_h * cfg.d_h) / (ms * 1e-3) / 1e9
+        roofline_all["finalize"] = {"kernel": "gsa_attn_finalize_kernel", "ms": ms, "launches": n, "bound": "hbm",
+                                    "achieved_gbs": gbs, "peak_gbs": peaks["hbm_gbs"], "frac": gbs / peaks["hbm_gbs"],
+                                    "note": "fp32 softmax state + g1 read, bf16 out written (one state slot per row counted)"}
+    ms, n = per_kernel("range_cuts")
+    if n:
+        roofline_all["range_cuts"] = {"kernel": "gsa_range_cuts_kernel", "ms": ms, "launches": n}
+    roofline_all["profiled_step_ms"] = sum(ms for _, ms in timeline)
 
     # ---- the upstream projection GEMM (outside the timed step: its outputs are the step's inputs) ----
     projection = None
@@ -317,7 +445,7 @@ def main():
 
     # ---- backward of the sparse gated attention stage, on the index sets this workload selects ----
     backward = None
-    if args.backward:
+    if not args.no_backward and world == 1 and not cfg.decode:
         idx_b = torch.empty((cfg.B, cfg.Lq, cfg.k_max), dtype=torch.int32, device="cuda")
         gsa.gsa_forward(p, d["Q"], d["K"], d["V"], d["qI"], d["kI"], d["w"], None, d["g1"], d["g2"], out, idx_b, kt,
                         None, args.slab_rows, ws, stream)
@@ -436,7 +564,8 @@ def main():
                 "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                 "config": workload_config(cfg), "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
-                "roofline": roofline, "cpu_baseline": cpu_baseline, "stages": stages,
+                "roofline": roofline, "roofline_all": roofline_all, "measured_rates": rates,
+                "cpu_baseline": cpu_baseline, "stages": stages,
                 "upstream_projection": projection, "backward": backward}
         print(json.dumps(line))
     if world > 1:

@@ -18,14 +18,27 @@
  * Conventions common to every call
  *   - Every data pointer is DEVICE memory owned by the caller, 16-byte aligned and
  *     contiguous in the stated layout, unless the argument says "host".
- *   - The library allocates no memory, keeps no state between calls and never
- *     synchronises the device (except gsa_forward_host and gsa_device_status, which
- *     wait for `stream`).  Work is enqueued on `stream` (a cudaStream_t passed as
- *     void*; NULL is the legacy default stream).
+ *   - The library allocates no memory and never synchronises the device (except
+ *     gsa_forward_host, gsa_device_status and gsa_select_fallback_rows, which wait for
+ *     `stream`).  Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is
+ *     the legacy default stream).
+ *   - No data is kept between calls.  The only state the library holds is process-wide
+ *     and set explicitly: the launch counter, the debug / tuning knobs
+ *     (gsa_debug_set_indexer_path, gsa_debug_set_attn_range_keys, gsa_debug_set_wait_limit)
+ *     and the profiling hooks (gsa_profile_set_events, gsa_profile_set_timeline).  A knob
+ *     changes the launch plan -- and with gsa_debug_set_attn_range_keys the workspace
+ *     size -- of every later call on every host thread; set them before the calls they are
+ *     meant for, not concurrently with them.
  *   - Return value: GSA_OK or a negative gsa_status.  Argument errors are detected on
- *     the host before anything is launched.  Conditions only the device can see
- *     (a bounded wait that ran out inside a tensor-core pipeline) are recorded in a
- *     status word at the start of the workspace; read it with gsa_device_status.
+ *     the host before anything is launched.  Conditions only the device can see are
+ *     recorded in a status word at the start of the workspace; read it with
+ *     gsa_device_status: a bounded wait that ran out inside a tensor-core pipeline
+ *     (every device-side wait has a limit of about a second; the kernel then stops issuing
+ *     work, lets what it issued complete, frees what it holds and returns), or an index
+ *     set handed to an attention / backward / loss call with an entry outside [0, Lk) or a
+ *     budget outside [0, k_max].  Such an entry never becomes an address: budgets are
+ *     clamped, a position used for a gather is clamped into the tensor, an entry that
+ *     would be scattered is skipped; the results of that row are then meaningless.
  *   - bf16 tensors are passed as void*; fp32 accumulation everywhere; outputs are
  *     rounded to bf16 once (round to nearest even).
  *   - Query t (0-based, of Lq) may look at keys s = 0 .. Lk-Lq+t ("visible keys",
@@ -51,8 +64,10 @@ typedef enum {
     GSA_ERR_WORKSPACE = -3,        /* workspace missing or smaller than gsa_workspace_bytes  */
     GSA_ERR_CUDA = -4,             /* a CUDA runtime / driver call failed                    */
     GSA_ERR_DEVICE_TIMEOUT = -5,   /* a bounded device-side wait expired (see device status) */
-    GSA_ERR_STATIC_SCRATCH = -6    /* problem larger than the built-in scratch array of the
+    GSA_ERR_STATIC_SCRATCH = -6,   /* problem larger than the built-in scratch array of the
                                       allocation-free entry point                            */
+    GSA_ERR_INDEX_RANGE = -7       /* a kernel met an index set entry outside [0, Lk) or a budget
+                                      outside [0, k_max] (see device status)                 */
 } gsa_status;
 
 /* Hyper-parameters (Table 1 of the paper) plus the call's geometry. */
@@ -85,7 +100,7 @@ typedef struct gsa_params {
 /*
  * Bytes of device workspace gsa_forward (and the per-stage calls) need for `p`.
  * `slab_rows` is the number of query rows whose fp32 score rows gsa_forward keeps
- * resident at a time (0 = library default: about 1 GiB of score rows, at least 32 rows).
+ * resident at a time (0 = library default: about 4 GiB of score rows, at least 32 rows).
  * Host call; writes *bytes.
  */
 int gsa_workspace_bytes(const gsa_params_t *p, int32_t slab_rows, size_t *bytes);
@@ -311,7 +326,8 @@ int gsa_forward_host(const gsa_params_t *p, const void *Q, const void *K, const 
 
 /*
  * Waits for `stream`, reads the device status word at the start of `ws` into
- * *status_out (host) and returns GSA_OK / GSA_ERR_DEVICE_TIMEOUT accordingly.
+ * *status_out (host) and returns GSA_OK, GSA_ERR_DEVICE_TIMEOUT (*status_out 1..3: copy producer,
+ * MMA issuer, epilogue) or GSA_ERR_INDEX_RANGE (*status_out 6) accordingly.
  * The word is cleared by every call that takes `ws`.  ws == NULL reads the status word of
  * gsa_sparse_gated_attn_fwd_static (it lives in the library's built-in array on the current device).
  */
@@ -342,12 +358,50 @@ void gsa_debug_set_indexer_path(int32_t path);
 void gsa_debug_set_attn_range_keys(int32_t keys);
 
 /*
+ * Test knob for the bounded device-side waits: `cycles` is the limit of every wait in SM clock cycles
+ * (<= 0 restores the default of 2^31, about a second).  With withhold_first_copy != 0 the copy producer of
+ * each tensor-core kernel (gsa_indexer_scores / gsa_forward on the tcgen05 path, gsa_project,
+ * gsa_output_projection) leaves out its first copy, so that the wait for it meets a barrier that nothing
+ * completes: the way to see the give-up path work (status word set, kernel returns, context intact).
+ * Process-wide; not meant for production use.
+ */
+void gsa_debug_set_wait_limit(int64_t cycles, int32_t withhold_first_copy);
+
+/*
  * Profiling hook: three cudaEvent_t handles (or NULL to switch off) that every following
  * gsa_forward records on its stream: at entry, after the last indexer/top-k slab (before the
  * sparse-attention launch), and after the sparse-attention launch.  Process-wide; the caller
  * owns the events and reads them after synchronising.
  */
 void gsa_profile_set_events(void *ev_begin, void *ev_selected, void *ev_end);
+
+/*
+ * Profiling hook with one interval per launch: `events` is an array of `capacity` cudaEvent_t handles
+ * (created by the caller, timing enabled).  Every following gsa_forward records events[0] at entry and the
+ * next event behind each stage it enqueues, and writes into the HOST arrays stage_out[i] which stage the
+ * interval events[i] .. events[i + 1] belongs to (0 indexer, 1 budget + top-k, 2 value gate, 3 range cuts,
+ * 4 sparse attention, 5 normalise + output gate) and into *count_out the number of intervals.  The events
+ * serialise nothing but cost a little: use it for a profiling step, not inside a timed loop.  NULL / 0
+ * switches it off.  Process-wide; the caller owns the events and the arrays and reads them after
+ * synchronising.
+ */
+void gsa_profile_set_timeline(void **events, int32_t capacity, int32_t *stage_out, int32_t *count_out);
+
+/*
+ * Rate probes (measurement aids; the paper has no counterpart).  They enqueue one kernel on `stream`; the
+ * caller times it with events and divides.
+ *   gsa_probe_gather: reads the first piece_bytes of table row row_idx[i] for every i < n_idx with plain
+ *     32-byte loads, every thread keeping eight loads in flight: n_idx * piece_bytes bytes gathered.
+ *     table: n_rows rows of row_bytes (device, 32-byte aligned; row_bytes a multiple of 32, piece_bytes
+ *     32 times a power of two);
+ *     row_idx: n_idx int32 on the device (values outside [0, n_rows) are clamped); sink: 4 bytes of device
+ *     memory.  A table smaller than the L2 gives the L2's gather rate, a larger one HBM's.
+ *   gsa_probe_ex2: every resident thread runs `iters` rounds of eight independent 2^x on the
+ *     special-function unit; *ops_out (host) receives the number of 2^x evaluated.  sink: 4 bytes (device).
+ */
+int gsa_probe_gather(const void *table, int32_t n_rows, int64_t row_bytes, int32_t piece_bytes,
+                     const int32_t *row_idx, int64_t n_idx, void *sink, void *stream);
+int gsa_probe_ex2(int32_t iters, int64_t *ops_out, void *sink, void *stream);
 
 /* Static string for a gsa_status value. */
 const char *gsa_status_string(int status);

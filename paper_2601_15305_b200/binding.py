@@ -24,6 +24,7 @@ EXPORTS = (
     "gsa_select_fallback_rows", "gsa_project", "gsa_project_columns", "gsa_output_projection",
     "gsa_attn_bwd_workspace_bytes", "gsa_sparse_gated_attn_bwd", "gsa_vbar_update",
     "gsa_attn_probs_mean", "gsa_indexer_kl_workspace_bytes", "gsa_indexer_kl_bwd", "gsa_sparse_gated_attn_fwd_lse",
+    "gsa_profile_set_timeline", "gsa_probe_gather", "gsa_probe_ex2", "gsa_debug_set_wait_limit",
 )
 
 STATIC_SCRATCH_BYTES = 32 << 20     # GSA_STATIC_SCRATCH_BYTES of include/gsa.h
@@ -243,7 +244,7 @@ def gsa_device_status(ws, stream=None) -> int:
     one of gsa_sparse_gated_attn_fwd_static."""
     v = ctypes.c_int32(0)
     rc = lib().gsa_device_status(_dp(ws), _stream(stream), ctypes.byref(v))
-    if rc not in (0, -5):
+    if rc not in (0, -5, -7):
         _check(rc, "gsa_device_status")
     return v.value
 
@@ -260,6 +261,48 @@ def gsa_launch_count() -> int:
 
 def gsa_debug_set_indexer_path(path: int) -> None:
     lib().gsa_debug_set_indexer_path(ctypes.c_int32(path))
+
+
+def gsa_debug_set_wait_limit(cycles: int = 0, withhold_first_copy: bool = False) -> None:
+    lib().gsa_debug_set_wait_limit(ctypes.c_int64(cycles), ctypes.c_int32(1 if withhold_first_copy else 0))
+
+
+STAGE_NAMES = ("indexer", "select", "value_gate", "range_cuts", "sparse_attn", "finalize")
+_timeline_keep = None        # the arrays the library writes into must outlive the calls
+
+
+def gsa_profile_set_timeline(events=None):
+    """events: list of torch.cuda.Event(enable_timing=True), each recorded once already (so its handle exists),
+    or None to switch the hook off.  Returns a function that, after a synchronize, gives the list of
+    (stage name, milliseconds) intervals of the last gsa_forward."""
+    global _timeline_keep
+    if not events:
+        lib().gsa_profile_set_timeline(None, ctypes.c_int32(0), None, None)
+        _timeline_keep = None
+        return None
+    n = len(events)
+    handles = (ctypes.c_void_p * n)(*[e.cuda_event for e in events])
+    stages = (ctypes.c_int32 * n)()
+    count = ctypes.c_int32(0)
+    _timeline_keep = (handles, stages, count, events)
+    lib().gsa_profile_set_timeline(handles, ctypes.c_int32(n), stages, ctypes.byref(count))
+
+    def read():
+        return [(STAGE_NAMES[stages[i]], events[i].elapsed_time(events[i + 1])) for i in range(count.value)]
+    return read
+
+
+def gsa_probe_gather(table, n_rows: int, row_bytes: int, piece_bytes: int, row_idx, sink, stream=None) -> None:
+    _check(lib().gsa_probe_gather(_dp(table), ctypes.c_int32(n_rows), ctypes.c_int64(row_bytes), ctypes.c_int32(piece_bytes),
+                                  _dp(row_idx, I32), ctypes.c_int64(row_idx.numel()), _dp(sink), _stream(stream)),
+           "gsa_probe_gather")
+
+
+def gsa_probe_ex2(iters: int, sink, stream=None) -> int:
+    """Enqueues the exp2 probe; returns the number of 2^x it evaluates."""
+    ops = ctypes.c_int64(0)
+    _check(lib().gsa_probe_ex2(ctypes.c_int32(iters), ctypes.byref(ops), _dp(sink), _stream(stream)), "gsa_probe_ex2")
+    return ops.value
 
 
 def gsa_profile_set_events(ev_begin=None, ev_selected=None, ev_end=None) -> None:

@@ -21,8 +21,37 @@ int sm_count() {
     }
     return n;
 }
+thread_local int32_t* t_dev_status = nullptr;
 static int32_t g_indexer_path = 0;
+static std::atomic<long long> g_wait_cycles{kSpinCycles};
+static std::atomic<int> g_withhold_first_copy{0};
+
+long long wait_limit_cycles() { return g_wait_cycles.load(std::memory_order_relaxed); }
+bool withhold_first_copy() { return g_withhold_first_copy.load(std::memory_order_relaxed) != 0; }
 static cudaEvent_t g_prof_ev[3] = {nullptr, nullptr, nullptr};
+
+// profiling timeline: the caller's event handles and host arrays; armed only inside gsa_forward
+static cudaEvent_t* g_tl_events = nullptr;
+static int32_t g_tl_cap = 0;
+static int32_t* g_tl_stage = nullptr;
+static int32_t* g_tl_count = nullptr;
+static bool g_tl_armed = false;
+
+static void timeline_begin(cudaStream_t st) {
+    if (!g_tl_events || g_tl_cap < 2) return;
+    *g_tl_count = 0;
+    g_tl_armed = cudaEventRecord(g_tl_events[0], st) == cudaSuccess;
+}
+static void timeline_end() { g_tl_armed = false; }
+
+void timeline_mark(int32_t stage, cudaStream_t st) {
+    if (!g_tl_armed) return;
+    const int32_t n = *g_tl_count;
+    if (n + 1 >= g_tl_cap) return;                       // out of events: the rest of the call is not split up
+    if (cudaEventRecord(g_tl_events[n + 1], st) != cudaSuccess) return;
+    g_tl_stage[n] = stage;
+    *g_tl_count = n + 1;
+}
 
 cudaError_t launch_indexer_simple(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* qI,
                                   const __nv_bfloat16* kI, const float* w, const float* bI,
@@ -152,6 +181,7 @@ int gsa_indexer_scores(const gsa_params_t* p, const void* qI, const void* kI, co
     if (row_stride < p->Lk || row_stride % 4 != 0) return GSA_ERR_INVALID_ARG;
     if (!ws || ws_bytes < (size_t)kStatusBytes || !aligned16(ws)) return GSA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
+    t_dev_status = (int32_t*)ws;
     cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, st);
     if (e != cudaSuccess) return cuda_rc(e);
     return cuda_rc(launch_indexer(*p, rr, (const bf16*)qI, (const bf16*)kI, w, bI, scores, row_stride,
@@ -177,6 +207,7 @@ int gsa_project(const gsa_params_t* p, int32_t d_model, const void* H, const voi
     for (const void* q : ptrs) if (!q || !aligned16(q)) return GSA_ERR_INVALID_ARG;
     if (!ws || ws_bytes < (size_t)kStatusBytes || !aligned16(ws)) return GSA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
+    t_dev_status = (int32_t*)ws;
     cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, st);
     if (e != cudaSuccess) return cuda_rc(e);
     return cuda_rc(launch_project(*p, d_model, (const bf16*)H, (const bf16*)Wt, (bf16*)qI, (bf16*)kI, w,
@@ -193,6 +224,7 @@ int gsa_output_projection(const gsa_params_t* p, int32_t d_model, const void* at
     for (const void* q : ptrs) if (!q || !aligned16(q)) return GSA_ERR_INVALID_ARG;
     if (!ws || ws_bytes < (size_t)kStatusBytes || !aligned16(ws)) return GSA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
+    t_dev_status = (int32_t*)ws;
     cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, st);
     if (e != cudaSuccess) return cuda_rc(e);
     return cuda_rc(launch_gemm_bf16(p->B * p->Lq, p->n_h * p->d_h, d_model, (const bf16*)attn_out, (const bf16*)Wo_t,
@@ -209,10 +241,12 @@ int gsa_adaptive_topk(const gsa_params_t* p, const float* scores, int64_t row_st
     if (row_stride < p->Lk || row_stride % 4 != 0) return GSA_ERR_INVALID_ARG;
     IdxLayout il{0, rr.q_begin, rr.R};
     int32_t* fb = nullptr;
+    t_dev_status = nullptr;
     if (ws && aligned16(ws) && ws_bytes >= (size_t)kStatusBytes) {
         cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, (cudaStream_t)stream);
         if (e != cudaSuccess) return cuda_rc(e);
         fb = (int32_t*)ws + kStatusFallbackWord;
+        t_dev_status = (int32_t*)ws;
     }
     return cuda_rc(launch_select(*p, rr, scores, row_stride, idx, kt, var, il, fb, (cudaStream_t)stream));
 }
@@ -274,6 +308,7 @@ int gsa_sparse_gated_attn_bwd(const gsa_params_t* p, const void* Q, const void* 
     bf16* dOs = (bf16*)(wsb + wp.dos_off);
     float* lse2 = (float*)(wsb + wp.lse_off);
     float* delta = (float*)(wsb + wp.delta_off);
+    t_dev_status = (int32_t*)ws;
     cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, st);
     if (e == cudaSuccess)
         e = launch_value_gate((const bf16*)V, (const bf16*)g2_logits, Vg, (int64_t)p->B * p->Lk * p->n_kv * p->d_h, st);
@@ -301,6 +336,7 @@ int gsa_attn_probs_mean(const gsa_params_t* p, const void* Q, const void* K, con
         return GSA_ERR_INVALID_ARG;
     if (!ws || !aligned16(ws) || ws_bytes < (size_t)kStatusBytes) return GSA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
+    t_dev_status = (int32_t*)ws;
     cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, st);
     IdxLayout il{0, rr.q_begin, rr.R};
     if (e == cudaSuccess) e = launch_attn_probs_mean(*p, rr, (const bf16*)Q, (const bf16*)K, idx, kt, il, pbar, st);
@@ -329,6 +365,7 @@ int gsa_indexer_kl_bwd(const gsa_params_t* p, const void* qI, const void* kI, co
     gsa_indexer_kl_workspace_bytes(p, &need);
     if (!ws || !aligned16(ws) || ws_bytes < need) return GSA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
+    t_dev_status = (int32_t*)ws;
     cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, st);
     IdxLayout il{0, rr.q_begin, rr.R};
     if (e == cudaSuccess)
@@ -363,6 +400,7 @@ static int attn_fwd_impl(const gsa_params_t* p, const void* Q, const void* K, co
         return GSA_ERR_INVALID_ARG;
     if (!ws || !aligned16(ws) || ws_bytes < attn_ws_bytes(*p, false)) return GSA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
+    t_dev_status = (int32_t*)ws;
     cudaError_t e0 = cudaMemsetAsync(ws, 0, kStatusBytes, st);
     if (e0 != cudaSuccess) return cuda_rc(e0);
     IdxLayout il{0, rr.q_begin, rr.R};
@@ -419,6 +457,7 @@ static int forward_impl(const gsa_params_t* p, const void* Q, const void* K, con
     if (!ws || !aligned16(ws) || ws_bytes < wp.total) return GSA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     char* wsb = (char*)ws;
+    t_dev_status = (int32_t*)ws;
     cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, st);
     if (e != cudaSuccess) return cuda_rc(e);
 
@@ -428,6 +467,8 @@ static int forward_impl(const gsa_params_t* p, const void* Q, const void* K, con
     const IdxLayout il{0, 0, p->Lq};
 
     if (g_prof_ev[0]) cudaEventRecord(g_prof_ev[0], st);
+    timeline_begin(st);
+    struct TimelineGuard { ~TimelineGuard() { timeline_end(); } } timeline_guard;
 
     // Eq. 7, 8, 4 slab by slab: score rows live only inside the workspace
     if (dense) {
@@ -439,8 +480,10 @@ static int forward_impl(const gsa_params_t* p, const void* Q, const void* K, con
             RowRange rr{b0, (p->B - b0 < nb_per ? p->B - b0 : nb_per), 0, p->Lq};
             if ((e = launch_indexer(*p, rr, (const bf16*)qI, (const bf16*)kI, w, bI, slab, wp.row_stride,
                                     (int32_t*)ws, st)) != cudaSuccess) return cuda_rc(e);
+            timeline_mark(kStageIndexer, st);
             if ((e = launch_select(*p, rr, slab, wp.row_stride, idx, kt, var_out, il, (int32_t*)ws + kStatusFallbackWord, st)) != cudaSuccess)
                 return cuda_rc(e);
+            timeline_mark(kStageSelect, st);
         }
     } else {
         for (int b = 0; b < p->B; ++b)
@@ -448,8 +491,10 @@ static int forward_impl(const gsa_params_t* p, const void* Q, const void* K, con
                 RowRange rr{b, 1, q0, (p->Lq - q0 < wp.slab_rows ? p->Lq - q0 : wp.slab_rows)};
                 if ((e = launch_indexer(*p, rr, (const bf16*)qI, (const bf16*)kI, w, bI, slab, wp.row_stride,
                                         (int32_t*)ws, st)) != cudaSuccess) return cuda_rc(e);
+                timeline_mark(kStageIndexer, st);
                 if ((e = launch_select(*p, rr, slab, wp.row_stride, idx, kt, var_out, il, (int32_t*)ws + kStatusFallbackWord, st)) != cudaSuccess)
                     return cuda_rc(e);
+                timeline_mark(kStageSelect, st);
             }
     }
 
@@ -463,6 +508,7 @@ static int forward_impl(const gsa_params_t* p, const void* Q, const void* K, con
         e = launch_value_gate((const bf16*)V, (const bf16*)g2_logits, Vg,
                               (int64_t)p->B * p->Lk * p->n_kv * p->d_h, st);
         if (e != cudaSuccess) return cuda_rc(e);
+        timeline_mark(kStageValueGate, st);
         Vuse = Vg;
         g2use = nullptr;
     }
@@ -602,7 +648,7 @@ int gsa_device_status(const void* ws, void* stream, int32_t* status_out) {
     if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
     if (e != cudaSuccess) return cuda_rc(e);
     if (status_out) *status_out = v;
-    return v == kDevOk ? GSA_OK : GSA_ERR_DEVICE_TIMEOUT;
+    return v == kDevOk ? GSA_OK : (v == kDevBadIndex ? GSA_ERR_INDEX_RANGE : GSA_ERR_DEVICE_TIMEOUT);
 }
 
 int gsa_select_fallback_rows(const void* ws, void* stream, int32_t* rows_out) {
@@ -622,6 +668,20 @@ void gsa_debug_set_indexer_path(int32_t path) { g_indexer_path = path; }
 
 void gsa_debug_set_attn_range_keys(int32_t keys) { set_attn_range_keys(keys); }
 
+void gsa_debug_set_wait_limit(int64_t cycles, int32_t withhold_first_copy) {
+    g_wait_cycles.store(cycles > 0 ? (long long)cycles : kSpinCycles, std::memory_order_relaxed);
+    g_withhold_first_copy.store(withhold_first_copy != 0 ? 1 : 0, std::memory_order_relaxed);
+}
+
+void gsa_profile_set_timeline(void** events, int32_t capacity, int32_t* stage_out, int32_t* count_out) {
+    const bool on = events && stage_out && count_out && capacity >= 2;
+    g_tl_events = on ? (cudaEvent_t*)events : nullptr;
+    g_tl_cap = on ? capacity : 0;
+    g_tl_stage = on ? stage_out : nullptr;
+    g_tl_count = on ? count_out : nullptr;
+    g_tl_armed = false;
+}
+
 void gsa_profile_set_events(void* ev_begin, void* ev_selected, void* ev_end) {
     g_prof_ev[0] = (cudaEvent_t)ev_begin;
     g_prof_ev[1] = (cudaEvent_t)ev_selected;
@@ -636,6 +696,7 @@ const char* gsa_status_string(int s) {
         case GSA_ERR_WORKSPACE: return "workspace missing or too small";
         case GSA_ERR_CUDA: return "CUDA error";
         case GSA_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+        case GSA_ERR_INDEX_RANGE: return "an index set entry or a budget was out of range (clamped or skipped on the device)";
         case GSA_ERR_STATIC_SCRATCH: return "problem exceeds the built-in scratch array (GSA_STATIC_SCRATCH_BYTES)";
     }
     return "unknown status";

@@ -64,6 +64,7 @@ struct AttnArgs {
     int32_t range, n_cuts;
     float scale_log2;         // sm_scale * log2(e)
     float* lse;               // optional output [B, Lq, n_h]: natural log of sum_j exp(sm_scale * q.k_j) over S_t
+    int32_t* dev_status;      // where an out-of-range index or budget is reported (may be null)
 };
 
 struct RowId { int32_t b, t; int64_t irow; };
@@ -138,7 +139,7 @@ gsa_sparse_attn_kernel(const AttnArgs a) {
         int part = 0;
         if (a.mode == 1) { part = (int)(rest % a.max_parts); rest /= a.max_parts; }
         const RowId r = row_of(a.rr, a.il, (int)rest);
-        const int k_eff = min(a.kt[r.irow], a.k_max);
+        const int k_eff = checked_budget(a.kt[r.irow], a.k_max, a.dev_status);
         int lo, hi, slot = 0;
         if (a.mode == 0) {
             lo = 0;
@@ -212,11 +213,10 @@ gsa_sparse_attn_kernel(const AttnArgs a) {
         const unsigned char* gbase = reinterpret_cast<const unsigned char*>(a.g2) + head0 + vch * 16;
         const uint32_t vdst = my_s32 + vkey * VSTRIDE + vch * 16;
         const int32_t pad_pos = count > 0 ? idx_seg[0] : 0;          // tail keys re-read a valid row (P = 0 there)
-        const int32_t max_pos = a.Lk - 1;
         auto load_pos = [&](int tile) -> int32_t {
             const int j = tile * kTileKeys + (lane & 15);
             const int32_t p = j < count ? idx_seg[j] : pad_pos;
-            return min(max(p, 0), max_pos);                          // a corrupt index must not leave the tensor
+            return checked_pos(p, a.Lk, a.dev_status);               // a corrupt index must not leave the tensor
         };
         uint4 kb[2 * NC];                                            // K tile = A operand fragments
         auto issue_k = [&](int32_t pos16) {
@@ -368,7 +368,7 @@ __global__ void __launch_bounds__(256) gsa_range_cuts_kernel(const int32_t* __re
     const int c = (int)(i % n_cuts);
     const RowId r = row_of(rr, il, (int)(i / n_cuts));
     const int32_t* __restrict__ row = idx + r.irow * k_max;
-    const int k_eff = min(kt[r.irow], k_max);
+    const int k_eff = clamp_budget(kt[r.irow], k_max);
     const int bound = c * range_keys;
     int lo = 0, hi = k_eff;                      // first position with row[pos] >= bound
     while (lo < hi) {
@@ -434,7 +434,7 @@ __global__ void __launch_bounds__(1024) gsa_attn_finalize_kernel(const float* __
         } else {
             for (int q = 0; q < rows_per_cta && lr0 + q < rows; ++q) {
                 const RowId r = row_of(rr, il, lr0 + q);
-                const int k_eff = min(kt[r.irow], k_max);
+                const int k_eff = clamp_budget(kt[r.irow], k_max);
                 const int np = parts_of(k_eff, max_parts);
                 float acc[G], mx[G], den[G];
 #pragma unroll
@@ -540,6 +540,7 @@ cudaError_t launch_attn_t(AttnArgs a, const gsa_params_t& p, const AttnPlan& pl,
                                                                           pl.n_ranges, g_range_keys);
         ++g_launches;
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        timeline_mark(kStageRangeCuts, st);
     }
     a.cuts = cuts;
     a.n_cuts = pl.n_ranges;
@@ -557,6 +558,7 @@ cudaError_t launch_attn_t(AttnArgs a, const gsa_params_t& p, const AttnPlan& pl,
             a.state, a.kt, g1, out, fr, a.il, a.idx_rows, p.Lq, p.n_h, p.n_kv, p.k_max, pl.mode, pl.slots, a.lse);
         ++g_launches;
         cudaError_t fe = cudaGetLastError();
+        timeline_mark(kStageFinalize, st);
         if (fe == cudaSuccess && prog && prog->n < prog->cap && prog->n < 64) {
             fe = cudaEventRecord(prog->events[prog->n], st);
             prog->t_lo[prog->n] = t_lo; prog->t_hi[prog->n] = t_hi;
@@ -580,6 +582,7 @@ cudaError_t launch_attn_t(AttnArgs a, const gsa_params_t& p, const AttnPlan& pl,
         kern<<<ctas, kWarpsPerCta * 32, smem, st>>>(ar);
         ++g_launches;
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        timeline_mark(kStageAttn, st);
         if (pl.mode == 0 && rg + 1 < pl.n_ranges) {
             // rows whose last visible key lies in this range are complete
             const int64_t t_done = (int64_t)(rg + 1) * g_range_keys - off;
@@ -634,6 +637,7 @@ cudaError_t launch_sparse_attn(const gsa_params_t& p, RowRange rr, const __nv_bf
     const AttnPlan pl = plan_attn(p);
     AttnArgs a;
     a.lse = lse;
+    a.dev_status = t_dev_status;
     a.Q = Q; a.K = K; a.V = V; a.g2 = g2; a.idx = idx; a.kt = kt;
     a.state = reinterpret_cast<float*>(scratch);
     int32_t* cuts = reinterpret_cast<int32_t*>((char*)scratch + (pl.state_bytes + 255) / 256 * 256);

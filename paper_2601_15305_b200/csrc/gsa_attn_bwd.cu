@@ -60,6 +60,7 @@ struct BwdArgs {
     IdxLayout il;
     int32_t Lq, Lk, n_h, n_kv, k_max;
     float scale;
+    int32_t* dev_status;          // where an out-of-range index or budget is reported (may be null)
 };
 
 __device__ __forceinline__ uint32_t movmatrix_t(uint32_t a) {
@@ -167,7 +168,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32, 4) gsa_sparse_attn_bwd_kernel(
     const int t = a.rr.q_begin + lr % a.rr.R;
     const int64_t qrow = (int64_t)b * a.Lq + t;
     const int64_t irow = a.il.row(b, t);
-    const int ke_all = clamp_budget(a.kt[irow], a.k_max);
+    const int ke_all = checked_budget(a.kt[irow], a.k_max, a.dev_status);
     const int32_t* __restrict__ S = a.idx + irow * a.k_max;
     // this item's part of the index set: positions [j_lo, ke)
     int j_lo = 0, ke = ke_all;
@@ -262,7 +263,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32, 4) gsa_sparse_attn_bwd_kernel(
     int32_t pos_fetched = 0;                              // positions of the tile fetched last (lanes 0..15)
     auto fetch = [&](int j, int stage) {
         if (j < ke) {
-            pos_fetched = clamp_pos(S[min(j + (lane & 15), ke - 1)], a.Lk);
+            pos_fetched = checked_pos(S[min(j + (lane & 15), ke - 1)], a.Lk, a.dev_status);
             fetch_tile(kbase, st_s32 + stage * STAGE, pos_fetched);
         }
         cp_async_commit();                                // (possibly empty: keeps the group count uniform)
@@ -540,7 +541,7 @@ cudaError_t launch_sparse_attn_bwd(const gsa_params_t& p, RowRange rr, const __n
     a.part_ml = (float2*)range_ws;
     a.dq32 = (float*)((char*)range_ws + ((size_t)br.n_ranges * a.total_rows * p.n_h * 8 + 255) / 256 * 256);
     a.cuts = (const int32_t*)((char*)a.dq32 + ((size_t)a.total_rows * p.n_h * p.d_h * 4 + 255) / 256 * 256);
-    a.Q = Q; a.K = K; a.Vg = Vg; a.g1 = g1; a.out = out; a.dout = dout; a.idx = idx; a.kt = kt;
+    a.Q = Q; a.K = K; a.Vg = Vg; a.g1 = g1; a.out = out; a.dout = dout; a.idx = idx; a.kt = kt; a.dev_status = t_dev_status;
     a.dQ = dQ; a.dg1 = dg1; a.dOs = dOs; a.lse2 = lse2; a.delta = delta; a.pbar = pbar; a.rr = rr; a.il = il;
     a.Lq = p.Lq; a.Lk = p.Lk; a.n_h = p.n_h; a.n_kv = p.n_kv; a.k_max = p.k_max;
     a.scale = p.sm_scale > 0.f ? p.sm_scale : 1.0f / sqrtf((float)p.d_h);

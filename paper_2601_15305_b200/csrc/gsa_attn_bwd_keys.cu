@@ -41,6 +41,7 @@ struct InvArgs {
     RowRange rr;
     IdxLayout il;
     int32_t Lq, Lk, k_max;
+    int32_t* dev_status;          // where a skipped entry is reported (may be null)
 };
 
 // one warp per query row: cnt[b * Lk + s] += 1 for every selected s
@@ -55,6 +56,7 @@ __global__ void __launch_bounds__(256) gsa_bwd_count_kernel(const InvArgs a, int
     for (int j = lane; j < ke; j += 32) {
         const int32_t s = S[j];
         if (key_in_range(s, a.Lk)) atomicAdd(cnt + (int64_t)b * a.Lk + s, 1);
+        else report_bad_index(a.dev_status);
     }
 }
 
@@ -449,6 +451,7 @@ cudaError_t launch_sparse_attn_bwd_keys(const gsa_params_t& p, RowRange rr, cons
     if (e != cudaSuccess) return e;
     InvArgs ia;
     ia.idx = idx; ia.kt = kt; ia.rr = rr; ia.il = il; ia.Lq = p.Lq; ia.Lk = p.Lk; ia.k_max = p.k_max;
+    ia.dev_status = t_dev_status;
     const unsigned row_ctas = (unsigned)((rr.rows() + 7) / 8);
     if (rr.rows() > 0) {
         gsa_bwd_count_kernel<<<row_ctas, 256, 0, st>>>(ia, cnt);

@@ -30,14 +30,31 @@ struct IdxLayout {
 constexpr int kStatusBytes = 256;   // head of every workspace: device status word, counters, padding
 constexpr int kStatusFallbackWord = 1;   // int32 word: rows on which top-k selection took its whole-row fallback
 
-// device status word values
-enum : int32_t { kDevOk = 0, kDevTimeoutTma = 1, kDevTimeoutMma = 2, kDevTimeoutEpi = 3,
-                 kDevTimeoutGather = 4, kDevTimeoutAttn = 5 };
+// device status word values: which bounded wait of a tensor-core pipeline ran out (copy producer, MMA
+// issuer, epilogue), or that a kernel met an index set entry / budget outside its range
+enum : int32_t { kDevOk = 0, kDevTimeoutTma = 1, kDevTimeoutMma = 2, kDevTimeoutEpi = 3, kDevBadIndex = 6 };
+
+// Status word of the call this host thread is enqueueing: the entry point sets it (the head of the call's
+// workspace, or null when the call has none) and the launchers copy it into their kernels' arguments.
+extern thread_local int32_t* t_dev_status;
+
+// Limit of every bounded device-side wait, in SM clock cycles (about one second unless the debug knob
+// changed it), and the fault-injection switch of the same knob: the copy producers of the tensor-core
+// kernels leave out their first copy, so the barrier it would complete is one that nothing sets.
+long long wait_limit_cycles();
+bool withhold_first_copy();
 
 extern std::atomic<int64_t> g_launches;   // host-side launch counter (any host thread may launch)
 
 // multiprocessors of the current device (cached per device; 148 if the query fails)
 int sm_count();
+
+// Profiling timeline (off unless gsa_profile_set_timeline armed one): while gsa_forward enqueues its work,
+// every launcher records the next event of the caller's array behind the stage it just enqueued and notes
+// which stage the interval that ends there belongs to.
+enum : int32_t { kStageIndexer = 0, kStageSelect = 1, kStageValueGate = 2, kStageRangeCuts = 3, kStageAttn = 4,
+                 kStageFinalize = 5 };
+void timeline_mark(int32_t stage, cudaStream_t st);
 
 // ---- stage launchers (host) ----------------------------------------------------------------
 cudaError_t launch_indexer(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* qI,
@@ -138,6 +155,19 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
 __device__ __forceinline__ int32_t clamp_budget(int32_t kt, int32_t k_max) { return min(max(kt, 0), k_max); }
 __device__ __forceinline__ int32_t clamp_pos(int32_t s, int32_t Lk) { return min(max(s, 0), Lk - 1); }
 __device__ __forceinline__ bool key_in_range(int32_t s, int32_t Lk) { return (uint32_t)s < (uint32_t)Lk; }
+// the same two rules, reporting what they had to correct through the status word (first report wins)
+__device__ __forceinline__ void report_bad_index(int32_t* dev_status) {
+    if (dev_status) atomicCAS(dev_status, kDevOk, kDevBadIndex);
+}
+__device__ __forceinline__ int32_t checked_budget(int32_t kt, int32_t k_max, int32_t* dev_status) {
+    if (kt < 0 || kt > k_max) report_bad_index(dev_status);
+    return clamp_budget(kt, k_max);
+}
+__device__ __forceinline__ int32_t checked_pos(int32_t s, int32_t Lk, int32_t* dev_status) {
+    if (key_in_range(s, Lk)) return s;
+    report_bad_index(dev_status);
+    return clamp_pos(s, Lk);
+}
 
 __device__ __forceinline__ float fast_sigmoid(float x) {
     // 1 / (1 + 2^(-x log2 e)); ex2.approx and rcp.approx are accurate to a few ulp
@@ -189,7 +219,8 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
 
 // ---- mbarrier (shared-memory barrier objects completed by arrivals and by async-copy bytes) --
 constexpr uint32_t kSpinLimit = 1u << 24;        // polls
-constexpr long long kSpinCycles = 1ll << 31;     // ~1 s of SM clock: no wait may last longer
+constexpr long long kSpinCycles = 1ll << 31;     // ~1 s of SM clock: no wait may last longer (default limit)
+constexpr uint32_t kDrainPolls = 1u << 20;       // polls granted to a completion that is already on its way
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
@@ -211,27 +242,27 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// bounded wait; returns false if it gave up (and raises the CTA's abort flag)
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// bounded wait of at most `limit` cycles; returns false if it gave up (and raises the CTA's abort flag)
+// or if another thread of the CTA already had
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long limit) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t_start = clock64();
     for (uint32_t it = 0; it < kSpinLimit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 63u) {
+        if ((it & 15u) == 15u) {
             if (*abort_flag) return false;
-            if (clock64() - t_start > kSpinCycles) break;
+            if (clock64() - t_start > limit) break;
         }
     }
     *abort_flag = 1;
     return false;
 }
-
-// one contiguous run global -> shared by the bulk-copy engine; both addresses 16-byte aligned,
-// bytes a multiple of 16; completion is counted on `bar`
-__device__ __forceinline__ void bulk_copy_g2s(uint32_t smem_dst, const void* gsrc, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_dst), "l"(gsrc), "r"(bytes), "r"(bar)
-                 : "memory");
+// Wait of the give-up path, for a completion that is already on its way (a copy or an MMA issued earlier
+// completes by itself): bounded by a poll count of its own, whatever the limit that ran out was.
+__device__ __forceinline__ bool mbar_drain(uint32_t bar, uint32_t parity) {
+    for (uint32_t p = 0; p < kDrainPolls; ++p)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {

@@ -58,6 +58,7 @@ struct ProbsArgs {
     IdxLayout il;
     int32_t Lq, Lk, n_h, n_kv, k_max;
     float scale;
+    int32_t* dev_status;          // where an out-of-range index or budget is reported (may be null)
 };
 
 template <int DH, int G>
@@ -80,7 +81,7 @@ __global__ void __launch_bounds__(kLossWarps * 32) gsa_attn_probs_mean_kernel(co
     const int b = a.rr.b0 + lr / a.rr.R, t = a.rr.q_begin + lr % a.rr.R;
     const int64_t qrow = (int64_t)b * a.Lq + t;
     const int64_t irow = a.il.row(b, t);
-    const int ke = clamp_budget(a.kt[irow], a.k_max);
+    const int ke = checked_budget(a.kt[irow], a.k_max, a.dev_status);
     const int32_t* __restrict__ S = a.idx + irow * a.k_max;
     float* __restrict__ prow = a.pbar + irow * a.k_max;
 
@@ -107,7 +108,7 @@ __global__ void __launch_bounds__(kLossWarps * 32) gsa_attn_probs_mean_kernel(co
     const __nv_bfloat16* const kbase = a.K + ((size_t)b * a.Lk * a.n_kv + g) * DH;
     auto fetch = [&](int j, int stage) {
         if (j < ke) {
-            const int32_t pos16 = clamp_pos(S[min(j + (lane & 15), ke - 1)], a.Lk);
+            const int32_t pos16 = checked_pos(S[min(j + (lane & 15), ke - 1)], a.Lk, a.dev_status);
 #pragma unroll
             for (int i = 0; i < 16 * CPR / 32; ++i) {
                 const int chunk = i * 32 + lane;
@@ -210,6 +211,7 @@ struct KlArgs {
     RowRange rr;
     IdxLayout il;
     int32_t Lq, Lk, k_max, act;
+    int32_t* dev_status;          // where an out-of-range index or budget is reported (may be null)
 };
 
 template <int DI, int HI>
@@ -229,7 +231,7 @@ __global__ void __launch_bounds__(kLossWarps * 32) gsa_indexer_kl_kernel(const K
     const int b = a.rr.b0 + lr / a.rr.R, t = a.rr.q_begin + lr % a.rr.R;
     const int64_t qrow = (int64_t)b * a.Lq + t;
     const int64_t irow = a.il.row(b, t);
-    const int ke = clamp_budget(a.kt[irow], a.k_max);
+    const int ke = checked_budget(a.kt[irow], a.k_max, a.dev_status);
     const int32_t* __restrict__ S = a.idx + irow * a.k_max;
     const float* __restrict__ prow = a.pbar + irow * a.k_max;
 
@@ -260,7 +262,7 @@ __global__ void __launch_bounds__(kLossWarps * 32) gsa_indexer_kl_kernel(const K
     const __nv_bfloat16* const kbase = a.kI + (size_t)b * a.Lk * DI;
     auto fetch = [&](int j, int stage) {
         if (j < ke) {
-            const int32_t pos16 = clamp_pos(S[min(j + (lane & 15), ke - 1)], a.Lk);
+            const int32_t pos16 = checked_pos(S[min(j + (lane & 15), ke - 1)], a.Lk, a.dev_status);
 #pragma unroll
             for (int i = 0; i < 16 * CPR / 32; ++i) {
                 const int chunk = i * 32 + lane;
@@ -344,7 +346,7 @@ __global__ void __launch_bounds__(kLossWarps * 32) gsa_indexer_kl_kernel(const K
     float dw_acc[2] = {0.f, 0.f}, db_acc[2] = {0.f, 0.f};
     fetch(0, 0);
     for (int j0 = 0, stage = 0; j0 < ke; j0 += 16, stage ^= 1) {
-        const int32_t pos16 = clamp_pos(S[min(j0 + (lane & 15), ke - 1)], a.Lk);
+        const int32_t pos16 = checked_pos(S[min(j0 + (lane & 15), ke - 1)], a.Lk, a.dev_status);
         fetch(j0 + 16, stage ^ 1);
         const bool v0 = j0 + gid < ke, v1 = j0 + gid + 8 < ke;
         const float p0 = v0 ? prow[j0 + gid] : 0.f, p1 = v1 ? prow[j0 + gid + 8] : 0.f;
@@ -465,7 +467,7 @@ cudaError_t launch_attn_probs_mean(const gsa_params_t& p, RowRange rr, const __n
     cudaError_t e = cudaMemsetAsync(pbar, 0, (size_t)rr.rows() * p.k_max * 4, st);
     if (e != cudaSuccess) return e;
     ProbsArgs a;
-    a.Q = Q; a.K = K; a.idx = idx; a.kt = kt; a.pbar = pbar; a.rr = rr; a.il = il;
+    a.Q = Q; a.K = K; a.idx = idx; a.kt = kt; a.dev_status = t_dev_status; a.pbar = pbar; a.rr = rr; a.il = il;
     a.Lq = p.Lq; a.Lk = p.Lk; a.n_h = p.n_h; a.n_kv = p.n_kv; a.k_max = p.k_max;
     a.scale = p.sm_scale > 0.f ? p.sm_scale : 1.0f / sqrtf((float)p.d_h);
     const int G = p.n_h / p.n_kv;
@@ -487,7 +489,7 @@ cudaError_t launch_indexer_kl(const gsa_params_t& p, RowRange rr, const __nv_bfl
     if (e != cudaSuccess) return e;
     if (rr.rows() > 0) {
         KlArgs a;
-        a.qI = qI; a.kI = kI; a.w = w; a.bI = bI; a.idx = idx; a.kt = kt; a.pbar = pbar; a.loss = loss;
+        a.qI = qI; a.kI = kI; a.w = w; a.bI = bI; a.idx = idx; a.kt = kt; a.dev_status = t_dev_status; a.pbar = pbar; a.loss = loss;
         a.dqI = dqI; a.dw = dw; a.dkI32 = dkI32; a.dbI = dbI; a.rr = rr; a.il = il;
         a.Lq = p.Lq; a.Lk = p.Lk; a.k_max = p.k_max; a.act = p.act;
         e = cudaErrorInvalidValue;

@@ -43,6 +43,8 @@ struct TcArgs {
     int32_t Lq, Lk;
     int32_t groups_per_batch;
     int32_t tiles_per_cta;
+    long long wait_cycles;         // limit of every bounded wait
+    int32_t withhold_q;            // fault injection: the q^I copy is left out, so its barrier is never completed
 };
 
 template <int DI>
@@ -54,7 +56,7 @@ struct SmemPlan {
     static constexpr int OFF_W = OFF_K + kStages * K_BYTES;
     static constexpr int OFF_B = OFF_W + kNCols * 4;
     static constexpr int OFF_BAR = OFF_B + 64;                    // 8-byte aligned
-    static constexpr int N_BARS = 2 * kStages + 1 + 4;
+    static constexpr int N_BARS = 2 * kStages + 1 + 4 + 1;
     static constexpr int OFF_TMEM = OFF_BAR + N_BARS * 8;
     static constexpr int OFF_ABORT = OFF_TMEM + 8;
     static constexpr int TOTAL = OFF_ABORT + 8;
@@ -155,6 +157,7 @@ gsa_indexer_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
     const uint32_t bar_q = bar0 + 8u * (2 * kStages);
     auto bar_tfull = [&](int i) { return bar0 + 8u * (2 * kStages + 1 + i); };
     auto bar_tempty = [&](int i) { return bar0 + 8u * (2 * kStages + 3 + i); };
+    const uint32_t bar_drain = bar0 + 8u * (2 * kStages + 5);         // give-up path only
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -162,6 +165,7 @@ gsa_indexer_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         for (int s = 0; s < kStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
         mbar_init(bar_q, 1);
         for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull(i), 1); mbar_init(bar_tempty(i), kEpiWarps); }
+        mbar_init(bar_drain, 1);
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -183,40 +187,37 @@ gsa_indexer_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *s_tmem;
+    // what this thread has put in flight (the copy producer's and the MMA issuer's own counts)
+    int copies_issued = 0, mma_tiles_issued = 0;
+    bool q_issued = false;
 
     if (warp == 0) {
         // ================= TMA producer =======================================================
         if (lane == 0) {
-            mbar_expect_tx(bar_q, P::Q_BYTES);
-            tma_load_2d(sbase + P::OFF_Q, &tm_q, 0, (b * a.Lq + t0) * HI, bar_q);
-            int issued = 0;
-            for (int i = 0; i < ntiles; ++i) {
+            if (!a.withhold_q) {
+                mbar_expect_tx(bar_q, P::Q_BYTES);
+                tma_load_2d(sbase + P::OFF_Q, &tm_q, 0, (b * a.Lq + t0) * HI, bar_q);
+                q_issued = true;
+            }
+            for (int i = 0; i < ntiles && !*s_abort; ++i) {
                 const int s = i % kStages;
-                if (!mbar_wait(bar_empty(s), ((i / kStages) & 1) ^ 1, s_abort)) break;
+                if (!mbar_wait(bar_empty(s), ((i / kStages) & 1) ^ 1, s_abort, a.wait_cycles)) break;
                 mbar_expect_tx(bar_full(s), P::K_BYTES);
                 tma_load_2d(sbase + P::OFF_K + s * P::K_BYTES, &tm_k, 0, b * a.Lk + (tile0 + i) * kTileKeys,
                             bar_full(s));
-                issued = i + 1;
+                copies_issued = i + 1;
             }
-            if (*s_abort) {
-                // drain: wait (bounded) for the copies still in flight before the CTA may exit
-                atomicExch(a.dev_status, kDevTimeoutTma);
-                for (int i = max(0, issued - kStages); i < issued; ++i) {
-                    const uint32_t bar = bar_full(i % kStages), par = (i / kStages) & 1;
-                    for (uint32_t it = 0; it < (1u << 20) && !mbar_try_wait(bar, par); ++it) {}
-                }
-                for (uint32_t it = 0; it < (1u << 20) && !mbar_try_wait(bar_q, 0); ++it) {}
-            }
+            if (copies_issued < ntiles) atomicCAS(a.dev_status, kDevOk, kDevTimeoutTma);
         }
     } else if (warp == 1) {
         // ================= MMA issuer =========================================================
         if (lane == 0) {
-            bool ok = mbar_wait(bar_q, 0, s_abort);
+            bool ok = mbar_wait(bar_q, 0, s_abort, a.wait_cycles);
             const uint64_t bdesc = make_kmajor_desc<ROW_BYTES>(sbase + P::OFF_Q);
             for (int i = 0; ok && i < ntiles; ++i) {
                 const int s = i % kStages, buf = i & 1;
-                if (!mbar_wait(bar_tempty(buf), ((i >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
-                if (!mbar_wait(bar_full(s), (i / kStages) & 1, s_abort)) { ok = false; break; }
+                if (!mbar_wait(bar_tempty(buf), ((i >> 1) & 1) ^ 1, s_abort, a.wait_cycles)) { ok = false; break; }
+                if (!mbar_wait(bar_full(s), (i / kStages) & 1, s_abort, a.wait_cycles)) { ok = false; break; }
                 tc_fence_after();
                 const uint64_t adesc = make_kmajor_desc<ROW_BYTES>(sbase + P::OFF_K + s * P::K_BYTES);
 #pragma unroll
@@ -224,8 +225,9 @@ gsa_indexer_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
                     tc_mma_bf16(tmem_base + buf * kNCols, adesc + 2 * k, bdesc + 2 * k, kIdesc, k > 0);
                 tc_commit(bar_empty(s));                   // stage reusable once these MMAs have read it
                 tc_commit(bar_tfull(buf));                 // accumulator ready for the epilogue
+                mma_tiles_issued = i + 1;
             }
-            if (!ok) atomicExch(a.dev_status, kDevTimeoutMma);
+            if (!ok) atomicCAS(a.dev_status, kDevOk, kDevTimeoutMma);
         }
     } else {
         // ================= epilogue: sigmoid, head weights, head sum, store ===================
@@ -239,8 +241,8 @@ gsa_indexer_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         for (int j = 0; j < HI; ++j) bias[j] = RELU ? s_b[j] : s_b[j] * -1.4426950408889634f;
         for (int i = 0; i < ntiles; ++i) {
             const int buf = i & 1;
-            if (!mbar_wait(bar_tfull(buf), (i >> 1) & 1, s_abort)) {
-                if (lane == 0) atomicExch(a.dev_status, kDevTimeoutEpi);
+            if (!mbar_wait(bar_tfull(buf), (i >> 1) & 1, s_abort, a.wait_cycles)) {
+                if (lane == 0) atomicCAS(a.dev_status, kDevOk, kDevTimeoutEpi);
                 break;
             }
             tc_fence_after();
@@ -288,6 +290,27 @@ gsa_indexer_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
 
     tc_fence_before();
     __syncthreads();
+    if (*s_abort) {
+        // Give-up path.  Every role has left its loop, but what was issued before is still under way: copies
+        // land in this CTA's stages, MMAs read them and write its TMEM, commits arrive on its barriers.  None
+        // of that may outlive the CTA, whose TMEM and shared memory go to the next one.  All of it completes by
+        // itself (nothing issued waits for anything that was not), so these polls end; each is bounded anyway.
+        if (warp == 0 && lane == 0) {
+            if (q_issued) mbar_drain(bar_q, 0);
+            for (int i = max(0, copies_issued - kStages); i < copies_issued; ++i)
+                mbar_drain(bar_full(i % kStages), (i / kStages) & 1);
+        }
+        if (warp == 1 && lane == 0) {
+            tc_commit(bar_drain);                          // arrives once every MMA issued so far has completed
+            mbar_drain(bar_drain, 0);
+            for (int i = max(0, mma_tiles_issued - kStages); i < mma_tiles_issued; ++i)
+                mbar_drain(bar_empty(i % kStages), (i / kStages) & 1);
+            for (int i = max(0, mma_tiles_issued - 2); i < mma_tiles_issued; ++i)
+                mbar_drain(bar_tfull(i & 1), (i >> 1) & 1);
+        }
+        tc_fence_before();
+        __syncthreads();
+    }
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
@@ -316,6 +339,8 @@ cudaError_t launch_t(const gsa_params_t& p, RowRange rr, const __nv_bfloat16* qI
     int tpc = (int)(total_tiles / (sm_count() * 4));
     tpc = tpc < 4 ? 4 : (tpc > 64 ? 64 : tpc);
     a.tiles_per_cta = tpc;
+    a.wait_cycles = wait_limit_cycles();
+    a.withhold_q = withhold_first_copy() ? 1 : 0;
     dim3 grid((tiles_max + tpc - 1) / tpc, groups);
 
     // one CTA per SM: the kernel allocates all 512 TMEM columns, so a second resident CTA would

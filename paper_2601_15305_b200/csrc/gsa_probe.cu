@@ -1,0 +1,102 @@
+// Rate probes: small kernels that measure, on the device at hand, the ceilings two of the path's kernels
+// run against and that no vendor figure gives: the rate at which row pieces selected by an index list can be
+// gathered (out of the L2 when the table fits it, out of HBM otherwise), which bounds sparse attention, and
+// the special-function unit's exp2 rate, which bounds the indexer's sigmoid epilogue.  The benchmark times
+// them with events on the launching stream and prints the rates beside the kernels' own.
+#include "gsa_common.cuh"
+
+namespace gsa {
+namespace {
+
+constexpr int kProbeThreads = 256;
+constexpr int kProbeUnroll = 8;          // independent 32-byte loads in flight per thread
+
+// Piece i is the first (1 << unit_shift) 32-byte units of table row idx[i] (rows are row_bytes apart).  The
+// (piece, unit) pairs are dealt to the threads in order, so a warp-wide load covers whole 128-byte lines of
+// 32 >> unit_shift pieces (or part of one piece); every thread keeps kProbeUnroll loads in flight.  The
+// index of a load's piece is itself loaded (one 4-byte word shared by the lanes of a piece), as in a kernel
+// that walks an index set.
+__global__ void __launch_bounds__(kProbeThreads) gsa_probe_gather_kernel(const unsigned char* __restrict__ table,
+                                                                         int64_t row_bytes, int32_t unit_shift,
+                                                                         int32_t n_rows, const int32_t* __restrict__ idx,
+                                                                         int64_t n_idx, uint32_t* __restrict__ sink) {
+    const int64_t total = n_idx << unit_shift;
+    const int64_t step = (int64_t)gridDim.x * kProbeThreads * kProbeUnroll;
+    const uint32_t unit_mask = (1u << unit_shift) - 1u;
+    uint32_t acc = 0;
+    for (int64_t base = (int64_t)blockIdx.x * kProbeThreads * kProbeUnroll + threadIdx.x; base < total; base += step) {
+        int32_t row[kProbeUnroll];
+#pragma unroll
+        for (int u = 0; u < kProbeUnroll; ++u) {
+            const int64_t e = base + (int64_t)u * kProbeThreads;
+            row[u] = e < total ? clamp_pos(__ldg(idx + (e >> unit_shift)), n_rows) : -1;
+        }
+        uint4 lo[kProbeUnroll], hi[kProbeUnroll];
+#pragma unroll
+        for (int u = 0; u < kProbeUnroll; ++u) {
+            lo[u] = hi[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (row[u] >= 0) {
+                const uint32_t c = (uint32_t)(base + (int64_t)u * kProbeThreads) & unit_mask;
+                const unsigned char* src = table + (int64_t)row[u] * row_bytes + c * 32u;
+                asm volatile("ld.global.nc.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                             : "=r"(lo[u].x), "=r"(lo[u].y), "=r"(lo[u].z), "=r"(lo[u].w), "=r"(hi[u].x), "=r"(hi[u].y),
+                               "=r"(hi[u].z), "=r"(hi[u].w)
+                             : "l"(src));
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kProbeUnroll; ++u)
+            acc ^= lo[u].x ^ lo[u].y ^ lo[u].z ^ lo[u].w ^ hi[u].x ^ hi[u].y ^ hi[u].z ^ hi[u].w;
+    }
+    if (acc == 0x9E3779B9u) sink[0] = acc;             // keeps the loads alive; practically never taken
+}
+
+// Every thread runs 8 independent chains of 2^x; nothing else competes for the special-function unit.
+__global__ void __launch_bounds__(1024) gsa_probe_ex2_kernel(int32_t iters, float* __restrict__ sink) {
+    float x[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) x[u] = -0.001f * (float)(threadIdx.x + u + 1);
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) asm volatile("ex2.approx.ftz.f32 %0, %0;" : "+f"(x[u]));
+#pragma unroll
+        for (int u = 0; u < 8; ++u) x[u] -= 1.0f;      // back into (-1, 0]: 2^x stays in (1/2, 1]
+    }
+    float s = 0.f;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) s += x[u];
+    if (s == 12345.678f) sink[0] = s;
+}
+
+}  // namespace
+}  // namespace gsa
+
+using namespace gsa;
+
+extern "C" int gsa_probe_gather(const void* table, int32_t n_rows, int64_t row_bytes, int32_t piece_bytes,
+                                const int32_t* row_idx, int64_t n_idx, void* sink, void* stream) {
+    if (!table || !row_idx || !sink || n_idx < 1 || n_rows < 1) return GSA_ERR_INVALID_ARG;
+    // pieces of 32 * 2^s bytes, rows a multiple of 32 bytes
+    int unit_shift = 0;
+    while ((32 << unit_shift) < piece_bytes && unit_shift < 20) ++unit_shift;
+    if (piece_bytes < 32 || (32 << unit_shift) != piece_bytes) return GSA_ERR_INVALID_ARG;
+    if (row_bytes < piece_bytes || row_bytes % 32 != 0) return GSA_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(table) & 31u) != 0) return GSA_ERR_INVALID_ARG;
+    const int64_t total = n_idx << unit_shift;
+    int64_t ctas = (total + kProbeThreads * kProbeUnroll - 1) / (kProbeThreads * kProbeUnroll);
+    const int64_t cap = (int64_t)sm_count() * 8;
+    if (ctas > cap) ctas = cap;
+    gsa_probe_gather_kernel<<<(unsigned)ctas, kProbeThreads, 0, (cudaStream_t)stream>>>(
+        (const unsigned char*)table, row_bytes, unit_shift, n_rows, row_idx, n_idx, (uint32_t*)sink);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? GSA_OK : GSA_ERR_CUDA;
+}
+
+extern "C" int gsa_probe_ex2(int32_t iters, int64_t* ops_out, void* sink, void* stream) {
+    if (iters < 1 || !ops_out || !sink) return GSA_ERR_INVALID_ARG;
+    const int ctas = sm_count() * 2;
+    gsa_probe_ex2_kernel<<<ctas, 1024, 0, (cudaStream_t)stream>>>(iters, (float*)sink);
+    ++g_launches;
+    *ops_out = (int64_t)ctas * 1024 * 8 * iters;
+    return cudaGetLastError() == cudaSuccess ? GSA_OK : GSA_ERR_CUDA;
+}

@@ -31,7 +31,7 @@ constexpr int kA_BYTES = kTileM * kBlockK * 2;          // 16 KB
 constexpr int kB_BYTES = kTileN * kBlockK * 2;          // 32 KB
 constexpr int kStageBytes = kA_BYTES + kB_BYTES;
 constexpr int kOffBar = kPStages * kStageBytes;
-constexpr int kNBars = 2 * kPStages + 4;
+constexpr int kNBars = 2 * kPStages + 4 + 1;
 constexpr int kOffTmem = kOffBar + kNBars * 8;
 constexpr int kOffAbort = kOffTmem + 8;
 constexpr int kSmemTotal = kOffAbort + 8 + 1024;        // slack to align the base to 1024
@@ -47,6 +47,8 @@ struct ProjArgs {
     int32_t M, K, N;               // tokens, d_model, stacked output columns
     int32_t n_q, n_k, HI, n_g1, n_g2;
     int32_t m_tiles, n_tiles;
+    long long wait_cycles;         // limit of every bounded wait
+    int32_t withhold_first;        // fault injection: the first stage's copies are left out (its barrier is never completed)
 };
 
 __global__ void __launch_bounds__(kPThreads, 1)
@@ -71,11 +73,13 @@ gsa_project_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
     auto bar_empty = [&](int s) { return bar0 + 8u * (kPStages + s); };
     auto bar_tfull = [&](int i) { return bar0 + 8u * (2 * kPStages + i); };
     auto bar_tempty = [&](int i) { return bar0 + 8u * (2 * kPStages + 2 + i); };
+    const uint32_t bar_drain = bar0 + 8u * (2 * kPStages + 4);        // give-up path only
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (int s = 0; s < kPStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull(i), 1); mbar_init(bar_tempty(i), kPEpiWarps); }
+        mbar_init(bar_drain, 1);
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -91,32 +95,33 @@ gsa_project_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
 
     const int n_tiles_total = a.m_tiles * a.n_tiles;
     const int kblocks = (a.K + kBlockK - 1) / kBlockK;
+    // what this thread has put in flight (the copy producer's and the MMA issuer's own counts)
+    uint32_t copies_issued = 0;                            // stages filled so far (all tiles)
+    uint32_t mma_blocks_issued = 0, mma_tiles_committed = 0;
+    bool first_withheld = false;
 
     if (warp == 0) {
         // ================= TMA producer =======================================================
         if (lane == 0) {
-            uint32_t it = 0;                                   // k-blocks issued so far (all tiles)
-            for (int tile = blockIdx.x; tile < n_tiles_total && !*s_abort; tile += gridDim.x) {
+            bool gave_up = false;
+            for (int tile = blockIdx.x; tile < n_tiles_total && !gave_up && !*s_abort; tile += gridDim.x) {
                 const int m0 = (tile / a.n_tiles) * kTileM, n0 = (tile % a.n_tiles) * kTileN;
-                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    const uint32_t it = copies_issued;
                     const int s = it % kPStages;
-                    if (!mbar_wait(bar_empty(s), ((it / kPStages) & 1) ^ 1, s_abort)) break;
-                    mbar_expect_tx(bar_full(s), kStageBytes);
-                    const uint32_t dst = sbase + s * kStageBytes;
-                    tma_load_2d(dst, &tm_h, kb * kBlockK, m0, bar_full(s));
-                    tma_load_2d(dst + kA_BYTES, &tm_w, kb * kBlockK, n0, bar_full(s));
+                    if (!mbar_wait(bar_empty(s), ((it / kPStages) & 1) ^ 1, s_abort, a.wait_cycles)) { gave_up = true; break; }
+                    if (it == 0 && a.withhold_first) {
+                        first_withheld = true;             // (counted as issued; the give-up path skips it)
+                    } else {
+                        mbar_expect_tx(bar_full(s), kStageBytes);
+                        const uint32_t dst = sbase + s * kStageBytes;
+                        tma_load_2d(dst, &tm_h, kb * kBlockK, m0, bar_full(s));
+                        tma_load_2d(dst + kA_BYTES, &tm_w, kb * kBlockK, n0, bar_full(s));
+                    }
+                    copies_issued = it + 1;
                 }
             }
-            if (*s_abort) {
-                // wait (bounded) for the copies still in flight before the CTA may exit
-                atomicExch(a.dev_status, kDevTimeoutTma);
-                const uint32_t back = it < (uint32_t)kPStages ? it : (uint32_t)kPStages;
-                for (uint32_t i = 0; i < back; ++i) {
-                    const uint32_t f = it - 1 - i;
-                    const uint32_t bar = bar_full(f % kPStages), par = (f / kPStages) & 1;
-                    for (uint32_t p = 0; p < (1u << 20) && !mbar_try_wait(bar, par); ++p) {}
-                }
-            }
+            if (gave_up) atomicCAS(a.dev_status, kDevOk, kDevTimeoutTma);
         }
     } else if (warp == 1) {
         // ================= MMA issuer =========================================================
@@ -125,10 +130,10 @@ gsa_project_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < n_tiles_total; tile += gridDim.x, ++tl) {
                 const int buf = tl & 1;
-                if (!mbar_wait(bar_tempty(buf), ((tl >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
+                if (!mbar_wait(bar_tempty(buf), ((tl >> 1) & 1) ^ 1, s_abort, a.wait_cycles)) { ok = false; break; }
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const int s = it % kPStages;
-                    if (!mbar_wait(bar_full(s), (it / kPStages) & 1, s_abort)) { ok = false; break; }
+                    if (!mbar_wait(bar_full(s), (it / kPStages) & 1, s_abort, a.wait_cycles)) { ok = false; break; }
                     tc_fence_after();
                     const uint64_t adesc = make_kmajor_desc<128>(sbase + s * kStageBytes);
                     const uint64_t bdesc = make_kmajor_desc<128>(sbase + s * kStageBytes + kA_BYTES);
@@ -136,10 +141,14 @@ gsa_project_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
                     for (int k = 0; k < kBlockK / 16; ++k)      // 16 K-elements = 32 bytes = 2 descriptor units
                         tc_mma_bf16(tmem_base + buf * kTileN, adesc + 2 * k, bdesc + 2 * k, kIdescP, (kb | k) != 0);
                     tc_commit(bar_empty(s));                    // stage reusable once these MMAs have read it
+                    mma_blocks_issued = it + 1;
                 }
-                if (ok) tc_commit(bar_tfull(buf));              // accumulator ready for the epilogue
+                if (ok) {
+                    tc_commit(bar_tfull(buf));                  // accumulator ready for the epilogue
+                    mma_tiles_committed = tl + 1;
+                }
             }
-            if (!ok) atomicExch(a.dev_status, kDevTimeoutMma);
+            if (!ok) atomicCAS(a.dev_status, kDevOk, kDevTimeoutMma);
         }
     } else {
         // ================= epilogue: route, round / sigmoid, store =============================
@@ -150,8 +159,8 @@ gsa_project_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
         uint32_t tl = 0;
         for (int tile = blockIdx.x; tile < n_tiles_total; tile += gridDim.x, ++tl) {
             const int buf = tl & 1;
-            if (!mbar_wait(bar_tfull(buf), (tl >> 1) & 1, s_abort)) {
-                if (lane == 0) atomicExch(a.dev_status, kDevTimeoutEpi);
+            if (!mbar_wait(bar_tfull(buf), (tl >> 1) & 1, s_abort, a.wait_cycles)) {
+                if (lane == 0) atomicCAS(a.dev_status, kDevOk, kDevTimeoutEpi);
                 break;
             }
             tc_fence_after();
@@ -199,6 +208,34 @@ gsa_project_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
 
     tc_fence_before();
     __syncthreads();
+    if (*s_abort) {
+        // Give-up path: what was issued before a wait ran out is still under way (copies into this CTA's
+        // stages, MMAs that read them and write its TMEM, commits onto its barriers) and must not outlive the
+        // CTA.  All of it completes by itself, so these polls end; each is bounded anyway.
+        if (warp == 0 && lane == 0) {
+            const uint32_t back = copies_issued < (uint32_t)kPStages ? copies_issued : (uint32_t)kPStages;
+            for (uint32_t i = 0; i < back; ++i) {
+                const uint32_t f = copies_issued - 1 - i;
+                if (f == 0 && first_withheld) continue;    // never issued
+                mbar_drain(bar_full(f % kPStages), (f / kPStages) & 1);
+            }
+        }
+        if (warp == 1 && lane == 0) {
+            tc_commit(bar_drain);                          // arrives once every MMA issued so far has completed
+            mbar_drain(bar_drain, 0);
+            const uint32_t back = mma_blocks_issued < (uint32_t)kPStages ? mma_blocks_issued : (uint32_t)kPStages;
+            for (uint32_t i = 0; i < back; ++i) {
+                const uint32_t f = mma_blocks_issued - 1 - i;
+                mbar_drain(bar_empty(f % kPStages), (f / kPStages) & 1);
+            }
+            for (uint32_t i = 0; i < 2 && i < mma_tiles_committed; ++i) {
+                const uint32_t f = mma_tiles_committed - 1 - i;
+                mbar_drain(bar_tfull(f & 1), (f >> 1) & 1);
+            }
+        }
+        tc_fence_before();
+        __syncthreads();
+    }
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
@@ -220,6 +257,8 @@ cudaError_t launch_project(const gsa_params_t& p, int d_model, const __nv_bfloat
     a.n_q = p.HI * p.dI; a.n_k = p.dI; a.HI = p.HI; a.n_g1 = p.n_h * p.d_h; a.n_g2 = p.n_kv * p.d_h;
     a.m_tiles = (a.M + kTileM - 1) / kTileM;
     a.n_tiles = (a.N + kTileN - 1) / kTileN;
+    a.wait_cycles = wait_limit_cycles();
+    a.withhold_first = withhold_first_copy() ? 1 : 0;
     CUtensorMap tm_h, tm_w;
     if (!make_kblock_tmap(&tm_h, H, (uint64_t)a.M, (uint64_t)a.K, kTileM)) return cudaErrorUnknown;
     if (!make_kblock_tmap(&tm_w, Wt, (uint64_t)a.N, (uint64_t)a.K, kTileN)) return cudaErrorUnknown;
@@ -243,6 +282,8 @@ cudaError_t launch_gemm_bf16(int M, int K, int N, const __nv_bfloat16* A, const 
     a.n_q = N; a.n_k = 0; a.HI = 0; a.n_g1 = 0; a.n_g2 = 0;
     a.m_tiles = (M + kTileM - 1) / kTileM;
     a.n_tiles = (N + kTileN - 1) / kTileN;
+    a.wait_cycles = wait_limit_cycles();
+    a.withhold_first = withhold_first_copy() ? 1 : 0;
     CUtensorMap tm_a, tm_b;
     if (!make_kblock_tmap(&tm_a, A, (uint64_t)M, (uint64_t)K, kTileM)) return cudaErrorUnknown;
     if (!make_kblock_tmap(&tm_b, Bt, (uint64_t)N, (uint64_t)K, kTileN)) return cudaErrorUnknown;

@@ -90,6 +90,7 @@ extern "C" int gsa_sparse_gated_attn_fwd_static(const gsa_params_t* p, const voi
     // The array keeps what the previous call left in it.  The status word must start at zero and is
     // cleared here; the pre-pass overwrites every gated value the attention kernel will read, and the
     // attention kernels write every state slot before they read it.
+    t_dev_status = (int32_t*)scratch;
     e = cudaMemsetAsync(scratch, 0, kStatusBytes, st);
     if (e == cudaSuccess)
         e = launch_value_gate((const __nv_bfloat16*)V, (const __nv_bfloat16*)g2_logits, Vg,
