@@ -41,6 +41,9 @@ namespace {
 constexpr int kTileKeys = 16;
 constexpr int kWarpsPrefill = 16;          // warps per CTA, V' pre-gated
 constexpr int kWarpsFused = 12;            // warps per CTA when V and g2 pass through registers
+constexpr float kRefSlack = 8.0f;          // a score may exceed the softmax reference by 2^8 before the reference moves
+constexpr int kVStages = 2;                // shared-memory stages of a warp's V' tiles (one being read, the others in flight;
+                                           // measured at L = 128K: 2 stages 90.2 ms, 3 stages 94.7 ms)
 constexpr int kRangeKeysDefault = 16384;   // keys per L2 range: K + V' rows of 16K tokens = 64 MB at the 1.7B shape
 constexpr int kMaxRanges = 48;
 constexpr int kPartKeys = 128;             // decode: fewest keys worth a parallel segment
@@ -113,7 +116,7 @@ gsa_sparse_attn_kernel(const AttnArgs a) {
     constexpr int MT = DH / 16;                         // output m-tiles
     constexpr int VSTRIDE = HEAD_BYTES + 16;            // padded row of the staged V' tile
     constexpr int VTILE = kTileKeys * VSTRIDE;
-    constexpr int VSTAGES = FUSE_G2 ? 1 : 2;
+    constexpr int VSTAGES = FUSE_G2 ? 1 : kVStages;
     constexpr int CHUNKS = HEAD_BYTES / 16;             // 16-byte chunks per head row
     constexpr int KPI = 32 / CHUNKS;                    // keys one warp-wide 16-byte copy covers
     constexpr int ITS = kTileKeys / KPI;
@@ -244,16 +247,24 @@ gsa_sparse_attn_kernel(const AttnArgs a) {
             }
         };
 
-        int32_t pos_nxt = load_pos(1);
+        // positions of the tile whose K loads are issued next (tile + 1) and of the tile whose V' copies are
+        // issued next (tile + VSTAGES - 1)
+        int32_t pos_nxt = load_pos(1), pos_vahead = load_pos(VSTAGES - 1);
         {
             const int32_t pos0 = load_pos(0);
             issue_v(pos0, 0);
             cp_async_commit();
+            if (!FUSE_G2) {
+#pragma unroll
+                for (int t = 1; t < VSTAGES - 1; ++t) {
+                    if (t < ntiles) issue_v(load_pos(t), t);
+                    cp_async_commit();                                   // (possibly empty: one group per tile)
+                }
+            }
             issue_k(pos0);
         }
 
-        for (int tile = 0; tile < ntiles; ++tile) {
-            const int stage = FUSE_G2 ? 0 : (tile & 1);
+        for (int tile = 0, stage = 0; tile < ntiles; ++tile, stage = (FUSE_G2 || stage == VSTAGES - 1) ? 0 : stage + 1) {
             const bool more = tile + 1 < ntiles;
             if (FUSE_G2) {
                 // Eq. 9 in registers, then the gated tile goes to shared memory for the transposed read
@@ -272,53 +283,71 @@ gsa_sparse_attn_kernel(const AttnArgs a) {
                 }
                 if (more) issue_v(pos_nxt, 0);
             } else {
-                if (more) issue_v(pos_nxt, stage ^ 1);
+                // the stage consumed by the previous tile takes the tile after the next one
+                if (tile + VSTAGES - 1 < ntiles) issue_v(pos_vahead, stage == 0 ? VSTAGES - 1 : stage - 1);
                 cp_async_commit();
             }
 
             // ---- S^T = K Q^T : rows = 16 keys, columns = heads --------------------------------
-            float s[4] = {0.f, 0.f, 0.f, 0.f};
+            // (two accumulators: half the length of the dependent MMA chain)
+            float s[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int c = 0; c < NC; ++c) {
                 mma_bf16_16816(s, kb[c].x, kb[NC + c].x, kb[c].y, kb[NC + c].y, qb[c].x, qb[c].y);
-                mma_bf16_16816(s, kb[c].z, kb[NC + c].z, kb[c].w, kb[NC + c].w, qb[c].z, qb[c].w);
+                mma_bf16_16816(s2, kb[c].z, kb[NC + c].z, kb[c].w, kb[NC + c].w, qb[c].z, qb[c].w);
             }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) s[e] += s2[e];
             if (more) issue_k(pos_nxt);
             pos_nxt = load_pos(tile + 2);
+            pos_vahead = VSTAGES == 2 ? pos_nxt : load_pos(tile + VSTAGES);
 
             // ---- online softmax per head (column) ------------------------------------------------
+            // The reference value m_run that the exponentials are taken against need not be the running
+            // maximum itself: any value that no score exceeds by more than kRefSlack (in the log2 domain) keeps
+            // 2^(s - m_run) <= 2^kRefSlack, harmless in fp32 and bf16, and the normalisation at the end divides
+            // it out.  So the reduction over the tile's keys (shuffles across the lanes of a column) and the
+            // rescaling run only when some score jumps above the reference: on a row's first tiles.
             const int j0 = tile * kTileKeys + gid;
             const bool v0 = j0 < count, v1 = j0 + 8 < count;
-            float p[4];
-            float alpha[2];
+            float sc[4];
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
-                const float s0 = v0 ? s[e] * a.scale_log2 : -INFINITY;
-                const float s1 = v1 ? s[2 + e] * a.scale_log2 : -INFINITY;
-                float mx = fmaxf(s0, s1);
-                mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 4));
-                mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 8));
-                mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 16));
-                const float m_new = fmaxf(m_run[e], mx);              // finite: key 0 of every tile is valid
-                alpha[e] = ex2_fast(m_run[e] - m_new);
-                m_run[e] = m_new;
-                p[e] = ex2_fast(s0 - m_new);
-                p[2 + e] = ex2_fast(s1 - m_new);
-                l_run[e] = fmaf(l_run[e], alpha[e], p[e] + p[2 + e]);
+                sc[e] = v0 ? s[e] * a.scale_log2 : -INFINITY;
+                sc[2 + e] = v1 ? s[2 + e] * a.scale_log2 : -INFINITY;
             }
-            // the running maximum settles after a few tiles; rescale only when it moved
-            if (__any_sync(0xFFFFFFFFu, alpha[0] != 1.f || alpha[1] != 1.f)) {
+            const bool jump = fmaxf(sc[0], sc[2]) > m_run[0] + kRefSlack || fmaxf(sc[1], sc[3]) > m_run[1] + kRefSlack;
+            if (__any_sync(0xFFFFFFFFu, jump)) {
+                float alpha[2];
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    float mx = fmaxf(sc[e], sc[2 + e]);
+                    mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 4));
+                    mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 8));
+                    mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 16));
+                    const float m_new = fmaxf(m_run[e], mx);          // finite: key 0 of every tile is valid
+                    alpha[e] = ex2_fast(m_run[e] - m_new);
+                    m_run[e] = m_new;
+                    l_run[e] *= alpha[e];
+                }
 #pragma unroll
                 for (int mt = 0; mt < MT; ++mt) {
                     o[mt][0] *= alpha[0]; o[mt][1] *= alpha[1]; o[mt][2] *= alpha[0]; o[mt][3] *= alpha[1];
                 }
+            }
+            float p[4];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                p[e] = ex2_fast(sc[e] - m_run[e]);
+                p[2 + e] = ex2_fast(sc[2 + e] - m_run[e]);
+                l_run[e] += p[e] + p[2 + e];
             }
             // P^T[key, head] as the B operand: transpose the two 8x8 bf16 blocks of the fragment
             const uint32_t pb0 = movmatrix_trans(pack_bf16(p[0], p[1]));     // keys 0..7
             const uint32_t pb1 = movmatrix_trans(pack_bf16(p[2], p[3]));     // keys 8..15
 
             // ---- O^T += V'^T P^T -------------------------------------------------------------------
-            if (!FUSE_G2) cp_async_wait<1>();
+            if (!FUSE_G2) cp_async_wait<VSTAGES - 1>();              // all but the newest groups: this tile's has landed
             __syncwarp();
             {
                 const int mi = lane >> 3;
@@ -330,7 +359,7 @@ gsa_sparse_attn_kernel(const AttnArgs a) {
                     mma_bf16_16816(o[mt], a0, a1, a2, a3, pb0, pb1);
                 }
             }
-            __syncwarp();                                             // the stage is rewritten two tiles on
+            __syncwarp();                                             // the stage is refilled at the top of the next tile
         }
         if (!FUSE_G2) cp_async_wait<0>();
 
@@ -519,7 +548,7 @@ AttnPlan plan_attn(const gsa_params_t& p) {
 template <int DH, int G, bool FUSE_G2>
 cudaError_t launch_attn_t(AttnArgs a, const gsa_params_t& p, const AttnPlan& pl, const __nv_bfloat16* g1,
                           __nv_bfloat16* out, int32_t* cuts, cudaStream_t st, AttnProgress* prog) {
-    constexpr int VSTAGES = FUSE_G2 ? 1 : 2;
+    constexpr int VSTAGES = FUSE_G2 ? 1 : kVStages;
     constexpr int kWarpsPerCta = FUSE_G2 ? kWarpsFused : kWarpsPrefill;
     constexpr size_t smem = (size_t)kWarpsPerCta * VSTAGES * kTileKeys * (DH * 2 + 16);
     auto kern = gsa_sparse_attn_kernel<DH, G, FUSE_G2>;
