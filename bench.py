@@ -29,6 +29,7 @@ if ROOT not in sys.path:
 import numpy as np
 import torch
 
+from paper_2601_15305_b200 import cost_model
 from paper_2601_15305_b200.inputs import CONFIGS, make_inputs, sample_rows
 
 METRIC = "gsa_fwd_tokens_per_s"
@@ -360,7 +361,9 @@ def main():
     causal_pairs = cfg.B * sum(cfg.Lk - cfg.Lq + t + 1 for t in (0, cfg.Lq - 1)) * cfg.Lq / 2.0
     stages = {"indexer_plus_topk_ms": sel_ms, "sparse_attn_ms": attn_ms,
               "indexer_causal_tflop": 2.0 * cfg.HI * cfg.dI * causal_pairs / 1e12,
-              "mean_k_t": kt_sum / float(cfg.B * cfg.Lq), "select_fallback_rows": fallback_rows}
+              "mean_k_t": kt_sum / float(cfg.B * cfg.Lq), "select_fallback_rows": fallback_rows,
+              "paper_cost_model_speedup_vs_dense": cost_model.theoretical_speedup(cfg.Lk, cfg.n_h * cfg.d_h, cfg.dI, cfg.HI,
+                                                                                 cfg.k_base)}
 
     # ---- one object per kernel of the forward, from the per-launch events of the profiling step ----
     def per_kernel(name):

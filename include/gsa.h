@@ -260,6 +260,14 @@ int gsa_sparse_gated_attn_fwd(const gsa_params_t *p, const void *Q, const void *
                               void *stream);
 
 /*
+ * The value gate on its own, Eq. 9:  V_gated = bf16(V * sigmoid(g2_logits)), elementwise over n_elems
+ * bf16 values (a multiple of 8; three distinct device buffers, 16-byte aligned).
+ * What gsa_forward runs as its pre-pass; exposed for callers that gate their own shard of the values
+ * before exchanging them (context-parallel prefill) and then pass g2_logits = NULL.
+ */
+int gsa_value_gate(const void *V, const void *g2_logits, void *V_gated, int64_t n_elems, void *stream);
+
+/*
  * The same call for training: also saves the softmax statistics the backward pass needs,
  *     lse[b, t, h] = log sum_{j in S_t} exp(sm_scale * q_h . k_j)      (natural logarithm, fp32),
  * for rows [q_begin, q_end) of [B, Lq, n_h]; gsa_sparse_gated_attn_bwd takes them back.

@@ -18,7 +18,7 @@
  *   Eq. 12  aggregation                 O[t] = sum_{s in S_t} A[t,s] V'[s]
  *   Eq. 10  output gate G1              out[t,h] = O[t,h] * sigmoid(g1[t,h]) (elementwise)
  *
- * Readings where the paper is silent (each is also listed in the design notes):
+ * Readings where the paper is silent (listed with the library's documentation as well):
  *   - query t of Lq sees keys s = 0 .. Lk-Lq+t (causal; decode is Lq = 1);
  *   - Var is the population variance over the visible scores only;
  *   - k_eff = min(k_t, number of visible keys);

@@ -24,7 +24,7 @@ EXPORTS = (
     "gsa_select_fallback_rows", "gsa_project", "gsa_project_columns", "gsa_output_projection",
     "gsa_attn_bwd_workspace_bytes", "gsa_sparse_gated_attn_bwd", "gsa_vbar_update",
     "gsa_attn_probs_mean", "gsa_indexer_kl_workspace_bytes", "gsa_indexer_kl_bwd", "gsa_sparse_gated_attn_fwd_lse",
-    "gsa_profile_set_timeline", "gsa_probe_gather", "gsa_probe_ex2", "gsa_debug_set_wait_limit",
+    "gsa_profile_set_timeline", "gsa_probe_gather", "gsa_probe_ex2", "gsa_debug_set_wait_limit", "gsa_value_gate",
 )
 
 STATIC_SCRATCH_BYTES = 32 << 20     # GSA_STATIC_SCRATCH_BYTES of include/gsa.h
@@ -193,6 +193,11 @@ def gsa_vbar_update(var, momentum: float, v_bar, mean_var=None, stream=None) -> 
     """v_bar (one fp32 on the device) <- momentum * v_bar + (1 - momentum) * mean(var)."""
     _check(lib().gsa_vbar_update(_dp(var, F32), ctypes.c_int64(var.numel()), ctypes.c_float(momentum),
                                  _dp(v_bar, F32), _dp(mean_var, F32), _stream(stream)), "gsa_vbar_update")
+
+
+def gsa_value_gate(V, g2, V_gated, stream=None) -> None:
+    _check(lib().gsa_value_gate(_dp(V, BF16), _dp(g2, BF16), _dp(V_gated, BF16), ctypes.c_int64(V.numel()), _stream(stream)),
+           "gsa_value_gate")
 
 
 def gsa_sparse_gated_attn_fwd_lse(p, Q, K, V, g1, g2, idx, kt, out, lse, ws, stream=None) -> None:

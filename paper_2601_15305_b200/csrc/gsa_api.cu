@@ -379,6 +379,12 @@ int gsa_vbar_update(const float* var, int64_t n, float momentum, float* v_bar, f
     return cuda_rc(launch_vbar_update(var, n, momentum, v_bar, mean_var, (cudaStream_t)stream));
 }
 
+int gsa_value_gate(const void* V, const void* g2_logits, void* V_gated, int64_t n_elems, void* stream) {
+    if (!V || !g2_logits || !V_gated || n_elems < 1 || n_elems % 8 != 0) return GSA_ERR_INVALID_ARG;
+    if (!aligned16(V) || !aligned16(g2_logits) || !aligned16(V_gated)) return GSA_ERR_INVALID_ARG;
+    return cuda_rc(launch_value_gate((const bf16*)V, (const bf16*)g2_logits, (bf16*)V_gated, n_elems, (cudaStream_t)stream));
+}
+
 int gsa_attn_workspace_bytes(const gsa_params_t* p, int32_t with_value_gate_prepass, size_t* bytes) {
     int rc = check_params(p);
     if (rc) return rc;

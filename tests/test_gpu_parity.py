@@ -489,6 +489,36 @@ def test_forward_many_key_ranges_device_and_host_paths():
                              kt[b][rows].cpu().numpy(), rows, np.full_like(rows, b), _vis(cfg, rows))
 
 
+def test_context_parallel_row_blocks_match_the_whole_sequence(l8k):
+    """The context-parallel split on one GPU: the shares of two ranks (four row blocks in the chunked-prefill
+    geometry Lq = block rows, Lk = block end, values gated by gsa_value_gate before the exchange) computed one
+    after another from the gathered keys, against gsa_forward over the whole sequence and against the oracle."""
+    from paper_2601_15305_b200 import context_parallel as cp
+    cfg, x, d = l8k
+    out_full, idx_full, kt_full, _ = U.run_forward(cfg, d)
+    Vg = torch.empty_like(d["V"])
+    gsa.gsa_value_gate(d["V"], d["g2"], Vg)
+    keys = {"kI": d["kI"], "K": d["K"], "Vg": Vg}
+    world = 2
+    n0 = gsa.gsa_launch_count()
+    for rank in range(world):
+        blocks = cp.plan_row_blocks(cfg.Lk, world, rank)
+        local = cp.shard(d, blocks)
+        out, kt = cp.forward_context_parallel(cfg, local, world, rank, gathered_keys=keys)
+        at = 0
+        for blk in blocks:
+            assert torch.equal(kt[0, at:at + blk.rows], kt_full[0, blk.t0:blk.t1])
+            a, b = out[0, at:at + blk.rows].float(), out_full[0, blk.t0:blk.t1].float()
+            assert (a - b).abs().max().item() <= 2.0 ** -8 * b.abs().max().item()       # one bf16 ulp of the largest value
+            at += blk.rows
+    assert gsa.gsa_launch_count() - n0 >= 4 * 4          # per block: indexer, selection, attention, finalize at least
+    rows = sample_rows(cfg, 16).numpy()
+    o = oracle.forward(U.oracle_params(cfg), **x, rows_t=rows, want_scores=True)
+    sel = torch.from_numpy(rows).cuda()
+    U.check_forward_rows(U.oracle_params(cfg), x, o, out_full[0][sel].float().cpu().numpy(), idx_full[0][sel].cpu().numpy(),
+                         kt_full[0][sel].cpu().numpy(), rows, None, _vis(cfg, rows))
+
+
 def test_argument_errors_do_not_launch(tiny):
     cfg, x, d = tiny
     p = gsa.make_params(cfg)

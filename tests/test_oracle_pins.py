@@ -681,14 +681,23 @@ def test_indexer_kl_closed_forms_and_central_differences():
 
 
 def test_paper_printed_cost_model():
-    """Appendix A prints d^I H^I/(d n_h) ~ 0.002 and a 12.8x speed-up for its parameters."""
+    """The cost-model functions the benchmark prints from, against the two numbers Appendix A prints for its
+    parameters (d^I H^I / (d n_h) ~ 0.002 and a 12.8x speed-up) and against the closed form of Corollary 2."""
+    from paper_2601_15305_b200 import cost_model as cm
     vals = {}
     with open(__file__.rsplit("/", 1)[0] + "/golden/paper_cost_model.txt") as f:
         for line in f:
             if line.strip() and not line.startswith("#"):
                 k, v = line.split("=")
                 vals[k.strip()] = float(v.split("#")[0])
-    ratio = vals["dI"] * vals["HI"] / (vals["d"] * vals["n_h"])
-    assert abs(ratio - vals["printed_ratio"]) < 5e-4
-    sp = (vals["d"] / (vals["dI"] * vals["HI"])) / (1.0 + vals["k"] * vals["d"] / (vals["L"] * vals["dI"] * vals["HI"]))
-    assert abs(sp - vals["printed_speedup"]) < 0.1
+    d, n_h, dI, HI, k, L = (int(vals[n]) for n in ("d", "n_h", "dI", "HI", "k", "L"))
+    assert abs(cm.indexer_to_attention_ratio(d, n_h, dI, HI) - vals["printed_ratio"]) < 5e-4
+    assert abs(cm.theoretical_speedup(L, d, dI, HI, k) - vals["printed_speedup"]) < 0.1
+    # Corollary 2's closed form, and its two limits: no selection cost -> d / (d^I H^I); k = L -> below 1
+    for (L_, d_, dI_, HI_, k_) in ((L, d, dI, HI, k), (131072, 2048, 64, 8, 2048), (4096, 2048, 64, 8, 2048)):
+        closed = (d_ / (dI_ * HI_)) / (1.0 + k_ * d_ / (L_ * dI_ * HI_))
+        assert abs(cm.theoretical_speedup(L_, d_, dI_, HI_, k_) - closed) < 1e-9 * closed
+    assert abs(cm.theoretical_speedup(L, d, dI, HI, 0) - d / (dI * HI)) < 1e-9
+    assert cm.theoretical_speedup(1000, 2048, 64, 8, 1000) < 1.0
+    # the benchmark's layer shape (n_h d_h = 2048, H^I d^I = 512, k = 2048, L = 131072): 3.8x, not 12.8x
+    assert abs(cm.theoretical_speedup(131072, 2048, 64, 8, 2048) - 3.76) < 0.05
