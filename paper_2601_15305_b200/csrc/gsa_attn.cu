@@ -29,9 +29,10 @@
 // (few tokens) the same state slots hold the partial results of segments that run in parallel.
 // A last small kernel merges the slots, normalises, applies G1 and rounds to bf16 once.
 //
-// G2 is either applied by a streaming pre-pass (V' = bf16(V * sigmoid(g2)), prefill) or in
-// registers on the gathered rows (decode, where gating the whole cache would cost more than the
-// attention): V and g2 slices are then loaded to registers, gated, and stored to the shared tile.
+// G2 is either applied by a streaming pre-pass (V' = bf16(V * sigmoid(g2)), prefill) or on the gathered
+// rows (decode, where gating the whole cache would cost more than the attention): the V and the g2 slices
+// of a tile then arrive in two shared-memory tiles, both are read transposed into the same A-fragment
+// layout, and the gate is applied to the fragments in registers right before the MMA.
 #include "gsa_common.cuh"
 
 namespace gsa {
@@ -40,7 +41,7 @@ namespace {
 
 constexpr int kTileKeys = 16;
 constexpr int kWarpsPrefill = 16;          // warps per CTA, V' pre-gated
-constexpr int kWarpsFused = 12;            // warps per CTA when V and g2 pass through registers
+constexpr int kWarpsFused = 16;            // warps per CTA when V and g2 are gathered raw and gated in the fragments
 constexpr float kRefSlack = 8.0f;          // a score may exceed the softmax reference by 2^8 before the reference moves
 constexpr int kVStages = 2;                // shared-memory stages of a warp's V' tiles (one being read, the others in flight;
                                            // measured at L = 128K: 2 stages 90.2 ms, 3 stages 94.7 ms)
@@ -116,7 +117,7 @@ gsa_sparse_attn_kernel(const AttnArgs a) {
     constexpr int MT = DH / 16;                         // output m-tiles
     constexpr int VSTRIDE = HEAD_BYTES + 16;            // padded row of the staged V' tile
     constexpr int VTILE = kTileKeys * VSTRIDE;
-    constexpr int VSTAGES = FUSE_G2 ? 1 : kVStages;
+    constexpr int VSTAGES = FUSE_G2 ? 2 : kVStages;     // fused G2: one tile of V and one of g2, each single-staged
     constexpr int CHUNKS = HEAD_BYTES / 16;             // 16-byte chunks per head row
     constexpr int KPI = 32 / CHUNKS;                    // keys one warp-wide 16-byte copy covers
     constexpr int ITS = kTileKeys / KPI;
@@ -232,15 +233,15 @@ gsa_sparse_attn_kernel(const AttnArgs a) {
                 ldg_stream32(k1 + (c >> 1) * 128, kb[NC + c], kb[NC + c + 1]);
             }
         };
-        uint4 vreg[FUSE_G2 ? ITS : 1], greg[FUSE_G2 ? ITS : 1];
+        // (fused G2: `stage` is ignored; the V tile sits at stage 0 and the g2 tile at stage 1)
         auto issue_v = [&](int32_t pos16, int stage) {
 #pragma unroll
             for (int i = 0; i < ITS; ++i) {
                 const uint32_t p = __shfl_sync(0xFFFFFFFFu, pos16, i * KPI + vkey);
                 const uint64_t goff = (uint64_t)p * row_bytes;
                 if (FUSE_G2) {
-                    vreg[i] = ldg_stream(vbase + goff);
-                    greg[i] = ldg_stream(gbase + goff);
+                    cp_async16(vdst + i * KPI * VSTRIDE, vbase + goff);
+                    cp_async16(vdst + VTILE + i * KPI * VSTRIDE, gbase + goff);
                 } else {
                     cp_async16(vdst + stage * VTILE + i * KPI * VSTRIDE, vbase + goff);
                 }
@@ -266,23 +267,8 @@ gsa_sparse_attn_kernel(const AttnArgs a) {
 
         for (int tile = 0, stage = 0; tile < ntiles; ++tile, stage = (FUSE_G2 || stage == VSTAGES - 1) ? 0 : stage + 1) {
             const bool more = tile + 1 < ntiles;
-            if (FUSE_G2) {
-                // Eq. 9 in registers, then the gated tile goes to shared memory for the transposed read
-#pragma unroll
-                for (int i = 0; i < ITS; ++i) {
-                    uint4 vv = vreg[i];
-                    const uint4 gg = greg[i];
-                    __nv_bfloat162* v2 = reinterpret_cast<__nv_bfloat162*>(&vv);
-                    const __nv_bfloat162* g2v = reinterpret_cast<const __nv_bfloat162*>(&gg);
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float2 vf = __bfloat1622float2(v2[e]), gf = __bfloat1622float2(g2v[e]);
-                        v2[e] = __floats2bfloat162_rn(vf.x * gate_sigmoid(gf.x), vf.y * gate_sigmoid(gf.y));
-                    }
-                    *reinterpret_cast<uint4*>(my_smem + (i * KPI + vkey) * VSTRIDE + vch * 16) = vv;
-                }
-                if (more) issue_v(pos_nxt, 0);
-            } else {
+            const int32_t pos_v = pos_nxt;                            // fused G2: the next tile's V / g2 copies go out after this tile's product
+            if (!FUSE_G2) {
                 // the stage consumed by the previous tile takes the tile after the next one
                 if (tile + VSTAGES - 1 < ntiles) issue_v(pos_vahead, stage == 0 ? VSTAGES - 1 : stage - 1);
                 cp_async_commit();
@@ -347,21 +333,36 @@ gsa_sparse_attn_kernel(const AttnArgs a) {
             const uint32_t pb1 = movmatrix_trans(pack_bf16(p[2], p[3]));     // keys 8..15
 
             // ---- O^T += V'^T P^T -------------------------------------------------------------------
-            if (!FUSE_G2) cp_async_wait<VSTAGES - 1>();              // all but the newest groups: this tile's has landed
+            if (FUSE_G2) cp_async_wait<0>(); else cp_async_wait<kVStages - 1>();   // this tile's copies have landed
             __syncwarp();
             {
                 const int mi = lane >> 3;
-                const uint32_t vaddr = my_s32 + stage * VTILE + ((lane & 7) + (mi >> 1) * 8) * VSTRIDE + (mi & 1) * 16;
+                const uint32_t vaddr = my_s32 + (FUSE_G2 ? 0 : stage) * VTILE + ((lane & 7) + (mi >> 1) * 8) * VSTRIDE + (mi & 1) * 16;
 #pragma unroll
                 for (int mt = 0; mt < MT; ++mt) {
                     uint32_t a0, a1, a2, a3;
                     ldmatrix_x4_trans(a0, a1, a2, a3, vaddr + mt * 32);
+                    if constexpr (FUSE_G2) {
+                        // Eq. 9 on the fragments: the g2 tile read the same way has the same layout
+                        uint32_t g0, g1r, g2r, g3;
+                        ldmatrix_x4_trans(g0, g1r, g2r, g3, vaddr + VTILE + mt * 32);
+                        auto gate = [](uint32_t v, uint32_t g) -> uint32_t {
+                            const float2 vf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v));
+                            const float2 gf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&g));
+                            return pack_bf16(vf.x * gate_sigmoid(gf.x), vf.y * gate_sigmoid(gf.y));
+                        };
+                        a0 = gate(a0, g0); a1 = gate(a1, g1r); a2 = gate(a2, g2r); a3 = gate(a3, g3);
+                    }
                     mma_bf16_16816(o[mt], a0, a1, a2, a3, pb0, pb1);
                 }
             }
-            __syncwarp();                                             // the stage is refilled at the top of the next tile
+            __syncwarp();                                             // the tiles are refilled from here on
+            if (FUSE_G2) {
+                if (more) issue_v(pos_v, 0);
+                cp_async_commit();
+            }
         }
-        if (!FUSE_G2) cp_async_wait<0>();
+        cp_async_wait<0>();
 
         // ---- write the state slot ---------------------------------------------------------------
 #pragma unroll
@@ -548,7 +549,7 @@ AttnPlan plan_attn(const gsa_params_t& p) {
 template <int DH, int G, bool FUSE_G2>
 cudaError_t launch_attn_t(AttnArgs a, const gsa_params_t& p, const AttnPlan& pl, const __nv_bfloat16* g1,
                           __nv_bfloat16* out, int32_t* cuts, cudaStream_t st, AttnProgress* prog) {
-    constexpr int VSTAGES = FUSE_G2 ? 1 : kVStages;
+    constexpr int VSTAGES = FUSE_G2 ? 2 : kVStages;
     constexpr int kWarpsPerCta = FUSE_G2 ? kWarpsFused : kWarpsPrefill;
     constexpr size_t smem = (size_t)kWarpsPerCta * VSTAGES * kTileKeys * (DH * 2 + 16);
     auto kern = gsa_sparse_attn_kernel<DH, G, FUSE_G2>;
