@@ -35,8 +35,8 @@ from paper_2601_15305_b200.inputs import CONFIGS, make_inputs, sample_rows
 METRIC = "gsa_fwd_tokens_per_s"
 UNIT = "tokens/s"
 # special-function operations the indexer's epilogue spends per sigmoid: one exp2 each and one reciprocal
-# shared by four heads
-SFU_OPS_PER_SIGMOID = 1.25
+# shared by the eight heads of a query
+SFU_OPS_PER_SIGMOID = 1.125
 # DRAM bytes (read + written) of the sparse-attention launches of one forward, per workload, from the ncu
 # capture named in profiles/; empty while no capture of the current kernels exists
 ATTN_DRAM_TRAFFIC = {}

@@ -78,7 +78,24 @@ __device__ __forceinline__ float rcp_approx(float x) {
 //   w1/a1 + w2/a2 = (w1 a2 + w2 a1) / (a1 a2),   a_j = 1 + 2^(-(x_j + b_j) log2 e).
 // The exponent is clamped at 28 (sigmoid < 4e-9 there), so a product of four a_j stays below
 // 2^116 and cannot overflow.  nb[j] = -b_j log2 e.
+// The epilogue is bound by instruction issue, so for four and eight heads the arithmetic runs on the
+// packed fp32 instructions of sm_100 (two values per instruction).  Adjacent heads (2i, 2i+1) share a
+// register pair; the tree combines head 2i with 2i+2 and 2i+1 with 2i+3 (elementwise on the pairs), then,
+// for eight heads, those with their counterparts four heads on: the even and the odd heads end up as one
+// quotient each (four factors per denominator), and one more step joins the two under a single reciprocal:
+// the special-function unit, which bounds this kernel, then sees nine operations per eight sigmoids.  To keep
+// a product of eight factors inside fp32, the a_j of eight heads are carried scaled by 2^-12 (the offset
+// rides in the exponent's bias term and in the added constant; exponent clamped at 27: sigmoid < 8e-9), so
+// each lies in [2^-12, 2^15], the product of eight in [2^-96, 2^120] and a head's numerator term within
+// w_j 2^-96 .. 2^96: nothing overflows and only weights below 2^-30 could be flushed.  The 2^-12 left over
+// per quotient is folded into the weights, which the caller passes pre-scaled (kWeightScale).
+// 37 issue slots per eight sigmoids instead of 54.
 // RELU: sum_j w_j * max(x_j + b_j, 0) (Eq. 3), nb[j] = b_j; no special-function work at all.
+template <int HI> constexpr float kOne = HI == 8 ? 2.44140625e-04f : 1.0f;             // 2^-12 : 1
+template <int HI> constexpr float kExpClamp = HI == 8 ? 15.0f : 28.0f;                 // 27 - 12 : 28
+template <int HI> constexpr float kExpBias = HI == 8 ? -12.0f : 0.0f;                  // added to nb[j] by the caller
+template <int HI> constexpr float kWeightScale = HI == 8 ? 2.44140625e-04f : 1.0f;     // applied to w[j] by the caller
+
 template <int HI, bool RELU>
 __device__ __forceinline__ float gated_head_sum(const uint32_t* x, const float* w, const float (&nb)[HI]) {
     if constexpr (RELU) {
@@ -87,25 +104,39 @@ __device__ __forceinline__ float gated_head_sum(const uint32_t* x, const float* 
         for (int j = 0; j < HI; ++j) acc = fmaf(w[j], fmaxf(__uint_as_float(x[j]) + nb[j], 0.f), acc);
         return acc;
     }
-    float a[HI];
-#pragma unroll
-    for (int j = 0; j < HI; ++j)
-        a[j] = 1.0f + ex2_approx(fminf(fmaf(__uint_as_float(x[j]), -1.4426950408889634f, nb[j]), 28.0f));
-    float acc = 0.f;
     if constexpr (HI >= 4) {
+        constexpr int NP = HI / 2;
+        const float2 kScale = make_float2(-1.4426950408889634f, -1.4426950408889634f), kOne2 = make_float2(kOne<HI>, kOne<HI>);
+        float2 a2[NP];
 #pragma unroll
-        for (int g = 0; g < HI; g += 4) {
-            const float n01 = fmaf(w[g], a[g + 1], w[g + 1] * a[g]), d01 = a[g] * a[g + 1];
-            const float n23 = fmaf(w[g + 2], a[g + 3], w[g + 3] * a[g + 2]), d23 = a[g + 2] * a[g + 3];
-            const float num = fmaf(n01, d23, n23 * d01);
-            acc = fmaf(num, rcp_approx(d01 * d23), acc);
+        for (int i = 0; i < NP; ++i) {
+            const float2 y = __ffma2_rn(make_float2(__uint_as_float(x[2 * i]), __uint_as_float(x[2 * i + 1])), kScale,
+                                        make_float2(nb[2 * i], nb[2 * i + 1]));
+            a2[i] = __fadd2_rn(make_float2(ex2_approx(fminf(y.x, kExpClamp<HI>)), ex2_approx(fminf(y.y, kExpClamp<HI>))), kOne2);
         }
-    } else if constexpr (HI == 2) {
-        acc = fmaf(w[0], a[1], w[1] * a[0]) * rcp_approx(a[0] * a[1]);
+        // heads (0,1) with (2,3) [and (4,5) with (6,7)]: numerators and denominators of the pairs (0,2), (1,3)
+        float2 n2[NP / 2], d2[NP / 2];
+#pragma unroll
+        for (int q = 0; q < NP / 2; ++q) {
+            const float2 wp = make_float2(w[4 * q], w[4 * q + 1]), wq = make_float2(w[4 * q + 2], w[4 * q + 3]);
+            n2[q] = __ffma2_rn(wp, a2[2 * q + 1], __fmul2_rn(wq, a2[2 * q]));
+            d2[q] = __fmul2_rn(a2[2 * q], a2[2 * q + 1]);
+        }
+        if constexpr (HI == 8) {
+            const float2 nc = __ffma2_rn(n2[0], d2[1], __fmul2_rn(n2[1], d2[0]));     // even heads | odd heads
+            const float2 dc = __fmul2_rn(d2[0], d2[1]);
+            return fmaf(nc.x, dc.y, nc.y * dc.x) * rcp_approx(dc.x * dc.y);
+        } else {
+            return fmaf(n2[0].x, d2[0].y, n2[0].y * d2[0].x) * rcp_approx(d2[0].x * d2[0].y);
+        }
     } else {
-        acc = w[0] * rcp_approx(a[0]);
+        float a[HI];
+#pragma unroll
+        for (int j = 0; j < HI; ++j)
+            a[j] = 1.0f + ex2_approx(fminf(fmaf(__uint_as_float(x[j]), -1.4426950408889634f, nb[j]), 28.0f));
+        if constexpr (HI == 2) return fmaf(w[0], a[1], w[1] * a[0]) * rcp_approx(a[0] * a[1]);
+        else return w[0] * rcp_approx(a[0]);
     }
-    return acc;
 }
 
 // instruction descriptor: D fp32, A = B = bf16, both K-major, M = 128, N = 256
@@ -179,7 +210,8 @@ gsa_indexer_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         const int e = threadIdx.x - 64;                               // 0..255 = (query, head) column
         if (e < kNCols) {
             const int qi = e / HI, j = e % HI;
-            s_w[e] = qi < nq ? a.w[((size_t)b * a.Lq + t0 + qi) * HI + j] : 0.f;
+            // (sigmoid path with eight heads: weights pre-scaled by the power of two the head sum leaves over)
+            s_w[e] = qi < nq ? a.w[((size_t)b * a.Lq + t0 + qi) * HI + j] * (RELU ? 1.0f : kWeightScale<HI>) : 0.f;
             if (e < 8) s_b[e] = (a.bI && e < HI) ? a.bI[e] : 0.f;
         }
     }
@@ -238,7 +270,7 @@ gsa_indexer_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         constexpr int NCHUNK = kColsPerWarp / kChunkCols;
         float bias[HI];
 #pragma unroll
-        for (int j = 0; j < HI; ++j) bias[j] = RELU ? s_b[j] : s_b[j] * -1.4426950408889634f;
+        for (int j = 0; j < HI; ++j) bias[j] = RELU ? s_b[j] : fmaf(s_b[j], -1.4426950408889634f, kExpBias<HI>);
         for (int i = 0; i < ntiles; ++i) {
             const int buf = i & 1;
             if (!mbar_wait(bar_tfull(buf), (i >> 1) & 1, s_abort, a.wait_cycles)) {
