@@ -37,9 +37,10 @@ UNIT = "tokens/s"
 # special-function operations the indexer's epilogue spends per sigmoid: one exp2 each and one reciprocal
 # shared by the eight heads of a query
 SFU_OPS_PER_SIGMOID = 1.125
-# DRAM bytes (read + written) of the sparse-attention launches of one forward, per workload, from the ncu
-# capture named in profiles/; empty while no capture of the current kernels exists
-ATTN_DRAM_TRAFFIC = {}
+# DRAM bytes (read + written) of the sparse-attention launches of one forward, per workload, from the one-pass
+# ncu capture summarised in profiles/gsa_sparse_attn_kernel_l128k_dram.md (taken with the current kernel,
+# default slab and key ranges); a workload without a capture reports null
+ATTN_DRAM_TRAFFIC = {"l128k": 47.06e9}
 
 
 def measured_peaks():
@@ -342,8 +343,8 @@ def main():
     hbm_src = f"{peaks['source']} (MEASURED_PEAKS.json hbm_gbs)" if peaks["source"] == "measured" else "fallback 6650 GB/s"
     # The gather of sparse attention is served by the L2 (key ranges of 16384 keys keep a range's K and V' rows
     # resident), so the ceiling that binds is the L2's gather rate for 256-byte pieces, measured by the probe
-    # above; the fraction of the HBM copy bandwidth is kept beside it.  `traffic` (DRAM bytes of the launch from
-    # an ncu capture) is null: the kernels changed after the last capture.
+    # above; the fraction of the HBM copy bandwidth is kept beside it.  `traffic`: DRAM bytes of the launch from
+    # an ncu capture of this kernel (ATTN_DRAM_TRAFFIC), null for workloads without one.
     l2_peak = rates["gather_l2_64MB_piece256_gbs"] if rates else None
     roofline = {"kernel": "gsa_sparse_attn_kernel", "bound": "l2" if rates else "hbm", "achieved": achieved,
                 "peak": l2_peak if rates else peaks["hbm_gbs"], "unit": "GB/s",
