@@ -153,7 +153,7 @@ def measure_rates(gsa, stream):
     ms = best_ms(ex2)
     out["ex2_per_s"] = ops[0] / (ms * 1e-3)
     out["how"] = ("gsa_probe_gather: random rows of a 2048-byte-row table, first 256 / 2048 bytes of each, plain 32-byte "
-                  "loads, 8 in flight per thread, 2 GiB gathered per launch; gsa_probe_ex2: 8 independent ex2.approx "
+                  "loads, 4 in flight per thread at 2048 threads per SM, 2 GiB gathered per launch; gsa_probe_ex2: 8 independent ex2.approx "
                   "chains per thread, 2048 threads per SM; best of 3 launches after a warm-up")
     return out
 

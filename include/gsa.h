@@ -399,7 +399,8 @@ void gsa_profile_set_timeline(void **events, int32_t capacity, int32_t *stage_ou
  * Rate probes (measurement aids; the paper has no counterpart).  They enqueue one kernel on `stream`; the
  * caller times it with events and divides.
  *   gsa_probe_gather: reads the first piece_bytes of table row row_idx[i] for every i < n_idx with plain
- *     32-byte loads, every thread keeping eight loads in flight: n_idx * piece_bytes bytes gathered.
+ *     32-byte loads, every thread keeping four loads in flight (2048 threads per SM): n_idx * piece_bytes bytes
+ *     gathered.
  *     table: n_rows rows of row_bytes (device, 32-byte aligned; row_bytes a multiple of 32, piece_bytes
  *     32 times a power of two);
  *     row_idx: n_idx int32 on the device (values outside [0, n_rows) are clamped); sink: 4 bytes of device
