@@ -280,6 +280,25 @@ def test_attn_given_oracle_indices_tiny(tiny):
         U.check_out(out[0].float().cpu().numpy(), o["out"])
 
 
+@pytest.mark.parametrize("n_h,n_kv,d_h", [(8, 8, 128), (1, 1, 128), (16, 2, 128), (2, 1, 64), (32, 8, 64), (64, 8, 64)])
+def test_attn_head_layouts(n_h, n_kv, d_h):
+    """One, two, four and eight query heads per KV head at both head widths, with the value gate as a pre-pass
+    and inside the gather; index sets are the oracle's (budgets from k_min up to everything visible)."""
+    cfg = CONFIGS["tiny"].with_(name=f"attn_h{n_h}_{n_kv}_{d_h}", B=2, Lq=70, Lk=150, n_h=n_h, n_kv=n_kv, d_h=d_h,
+                                k_base=40, k_min=5, k_max=61, seed=90 + n_h)
+    x = make_inputs(cfg)
+    d = U.to_dev(x)
+    p = U.oracle_params(cfg)
+    rows_t = np.tile(np.arange(cfg.Lq), cfg.B)
+    rows_b = np.repeat(np.arange(cfg.B), cfg.Lq)
+    o = oracle.forward(p, **x, rows_t=rows_t, rows_b=rows_b)
+    idx = torch.from_numpy(o["idx"]).reshape(cfg.B, cfg.Lq, -1).cuda()
+    kt = torch.from_numpy(o["keff"]).reshape(cfg.B, cfg.Lq).cuda()
+    for use_prepass in (True, False):
+        out = U.run_attn(cfg, d, idx, kt, prepass=use_prepass)
+        U.check_out(out.reshape(cfg.B * cfg.Lq, n_h, d_h).float().cpu().numpy(), o["out"])
+
+
 def test_attn_pregated_values_and_custom_scale(tiny):
     cfg, x, d = tiny
     rows = np.arange(0, cfg.Lq, 7)
