@@ -426,11 +426,13 @@ __global__ void __launch_bounds__(1024) gsa_attn_finalize_kernel(const float* __
     const int rows_per_cta = mode == 0 ? kFinRows : 1;
     const int lr0 = blockIdx.x * rows_per_cta;
     const int i_begin = gridDim.y > 1 ? blockIdx.y * DH : 0, i_end = gridDim.y > 1 ? i_begin + DH : n_kv * DH;
-    for (int i = i_begin + threadIdx.x; i < i_end; i += blockDim.x) {
-        const int d = i % DH;
-        const int g = i / DH;
-        if (mode == 0) {
-            float o[kFinRows][G], l[kFinRows][G], gl[kFinRows][G];
+    if (mode == 0) {
+        // thread = (KV head, two consecutive d): 2 G consecutive floats of the state, bf16 pairs of g1 and out
+        for (int i = threadIdx.x; i < n_kv * (DH / 2); i += blockDim.x) {
+            const int d = (i % (DH / 2)) * 2;
+            const int g = i / (DH / 2);
+            float o[kFinRows][2 * G], l[kFinRows][G];
+            __nv_bfloat162 gl[kFinRows][G];
             int keff[kFinRows];
             size_t at0[kFinRows];
 #pragma unroll
@@ -440,11 +442,20 @@ __global__ void __launch_bounds__(1024) gsa_attn_finalize_kernel(const float* __
                 const float* st = state + ((int64_t)r.irow * n_kv + g) * STATE_F;
                 keff[q] = kt[r.irow];
                 at0[q] = (((size_t)r.b * Lq + r.t) * n_h + g * G) * DH + d;
+                if constexpr (G == 1) {
+                    const float2 v = *reinterpret_cast<const float2*>(st + d);
+                    o[q][0] = v.x; o[q][1] = v.y;
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 2 * G / 4; ++c) {
+                        const float4 v = *reinterpret_cast<const float4*>(st + d * G + 4 * c);
+                        o[q][4 * c] = v.x; o[q][4 * c + 1] = v.y; o[q][4 * c + 2] = v.z; o[q][4 * c + 3] = v.w;
+                    }
+                }
 #pragma unroll
                 for (int e = 0; e < G; ++e) {
-                    o[q][e] = st[d * G + e];
                     l[q][e] = st[G * DH + G + e];
-                    gl[q][e] = __bfloat162float(g1[at0[q] + (size_t)e * DH]);
+                    gl[q][e] = *reinterpret_cast<const __nv_bfloat162*>(g1 + at0[q] + (size_t)e * DH);
                 }
             }
 #pragma unroll
@@ -452,8 +463,11 @@ __global__ void __launch_bounds__(1024) gsa_attn_finalize_kernel(const float* __
                 if (lr0 + q >= rows) break;
 #pragma unroll
                 for (int e = 0; e < G; ++e) {
-                    const float v = (keff[q] > 0 && l[q][e] > 0.f) ? o[q][e] / l[q][e] * fast_sigmoid(gl[q][e]) : 0.f;
-                    out[at0[q] + (size_t)e * DH] = __float2bfloat16_rn(v);
+                    const bool live = keff[q] > 0 && l[q][e] > 0.f;
+                    const float2 gf = __bfloat1622float2(gl[q][e]);
+                    const float v0 = live ? o[q][e] / l[q][e] * fast_sigmoid(gf.x) : 0.f;          // (d, head e)
+                    const float v1 = live ? o[q][G + e] / l[q][e] * fast_sigmoid(gf.y) : 0.f;      // (d + 1, head e)
+                    *reinterpret_cast<__nv_bfloat162*>(out + at0[q] + (size_t)e * DH) = __floats2bfloat162_rn(v0, v1);
                     if (lse && d == 0) {               // the running maximum sits in front of the sums (log2 domain)
                         const RowId r = row_of(rr, il, lr0 + q);
                         const float m = state[((int64_t)r.irow * n_kv + g) * STATE_F + G * DH + e];
@@ -461,7 +475,13 @@ __global__ void __launch_bounds__(1024) gsa_attn_finalize_kernel(const float* __
                     }
                 }
             }
-        } else {
+        }
+        return;
+    }
+    for (int i = i_begin + threadIdx.x; i < i_end; i += blockDim.x) {
+        const int d = i % DH;
+        const int g = i / DH;
+        {
             for (int q = 0; q < rows_per_cta && lr0 + q < rows; ++q) {
                 const RowId r = row_of(rr, il, lr0 + q);
                 const int k_eff = clamp_budget(kt[r.irow], k_max);
@@ -577,7 +597,7 @@ cudaError_t launch_attn_t(AttnArgs a, const gsa_params_t& p, const AttnPlan& pl,
     a.n_cuts = pl.n_ranges;
     a.mode = pl.mode;
     a.max_parts = pl.slots;
-    const int fin_threads = a.n_kv * DH < 1024 ? a.n_kv * DH : 1024;
+    const int fin_threads = a.n_kv * (DH / 2) < 1024 ? a.n_kv * (DH / 2) : 1024;     // range mode: two d per thread
     // normalise + G1 + bf16 for rows t_lo <= t < t_hi of every batch element, then tell the caller
     auto finalize = [&](int t_lo, int t_hi) -> cudaError_t {
         if (t_hi <= t_lo) return cudaSuccess;
