@@ -246,6 +246,8 @@ int gsa_adaptive_topk(const gsa_params_t *p, const float *scores, int64_t row_st
  *   Q, g1_logits [B, Lq, n_h, d_h] bf16;  K, V, g2_logits [B, Lk, n_kv, d_h] bf16
  *   g2_logits may be NULL: V is then taken as already gated.
  *   idx [B, R, k_max], kt [B, R] as written by gsa_adaptive_topk (R = q_end - q_begin)
+ *       A row with kt = 0 (an empty S_t; gsa_adaptive_topk never writes one) has an empty sum: its
+ *       out row is written as zeros.
  *   out [B, Lq, n_h, d_h] bf16 (rows outside q_begin..q_end untouched)
  *   ws  workspace of at least gsa_attn_workspace_bytes(p, 0) bytes (status word, the fp32
  *       online-softmax state that is carried between key ranges or merged across parallel

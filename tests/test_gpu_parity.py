@@ -299,6 +299,32 @@ def test_attn_head_layouts(n_h, n_kv, d_h):
         U.check_out(out.reshape(cfg.B * cfg.Lq, n_h, d_h).float().cpu().numpy(), o["out"])
 
 
+@pytest.mark.parametrize("Lq", [40, 2])
+def test_attn_empty_index_sets_give_zero_rows(Lq):
+    """kt = 0 for some rows (an empty S_t): their outputs are zeros, the other rows are unaffected; with many
+    query rows (one launch per key range) and with few (parallel segments merged at the end)."""
+    cfg = CONFIGS["tiny"].with_(name="attn_empty", B=2, Lq=Lq, Lk=200, k_base=40, k_min=5, k_max=61, seed=95)
+    x = make_inputs(cfg)
+    d = U.to_dev(x)
+    p = U.oracle_params(cfg)
+    rows_t = np.tile(np.arange(cfg.Lq), cfg.B)
+    rows_b = np.repeat(np.arange(cfg.B), cfg.Lq)
+    o = oracle.forward(p, **x, rows_t=rows_t, rows_b=rows_b)
+    idx = torch.from_numpy(o["idx"]).reshape(cfg.B, cfg.Lq, -1).clone()
+    kt = torch.from_numpy(o["keff"]).reshape(cfg.B, cfg.Lq).clone()
+    empty = [(0, 0), (1, cfg.Lq - 1)]
+    for b, t in empty:
+        kt[b, t] = 0
+        idx[b, t] = -1
+    for use_prepass in (True, False):
+        out = U.run_attn(cfg, d, idx.cuda(), kt.cuda(), prepass=use_prepass).float().cpu().numpy()
+        want = o["out"].reshape(cfg.B, cfg.Lq, cfg.n_h, cfg.d_h).copy()
+        for b, t in empty:
+            assert (out[b, t] == 0.0).all()
+            want[b, t] = 0.0
+        U.check_out(out.reshape(-1, cfg.n_h, cfg.d_h), want.reshape(-1, cfg.n_h, cfg.d_h))
+
+
 def test_attn_pregated_values_and_custom_scale(tiny):
     cfg, x, d = tiny
     rows = np.arange(0, cfg.Lq, 7)
