@@ -9,10 +9,10 @@
 //      are dealt to the 16 warps round-robin, so each warp sees an even sample of the row.  Loads are
 //      fully coalesced float4s, one chunk ahead, turned through shared memory so that a lane holds 16
 //      consecutive scores; every score goes into fp64 sum and sum of squares; the position of a score
-//      that reaches tau (one float compare) goes into the candidate list in shared memory: a warp scan
+//      that reaches tau (one float compare) goes into the candidate list in shared memory, with its order key: a warp scan
 //      of the lanes' counts orders the chunk's candidates, one shared-memory atomic claims their space,
 //      and a table remembers where each chunk's entries start and how many there are.   -> Var, k_t
-//   2  on chip: the candidates' keys are fetched (one per thread and round); radix rounds over them give
+//   2  on chip: radix rounds over the candidates' keys give
 //      the exact threshold key T of the k_t-th largest score and how many keys equal to T are taken;
 //      the chunks are then walked in position order (counts per thread, one block scan, emission) to
 //      write S_t ascending.
@@ -35,8 +35,8 @@ constexpr int kListCap = 8192;                        // entries of the candidat
 constexpr int kListPerThread = kListCap / kSelThreads;  // 16
 constexpr int kIter = 512;                            // scores a warp takes per iteration (= one chunk)
 constexpr int kMaxChunks = 2048;                      // rows of up to kIter * kMaxChunks = 1 Mi scores are listed
-constexpr int kStageFloats = kListCap / kSelWarps;    // a warp's staging area inside list_key: 512 floats
-static_assert(kStageFloats == kIter, "one iteration must fit the warp's staging area");
+constexpr int kKeysInScan = kListCap - kBins;         // list entries below this get their key during pass 1
+static_assert(kListCap - kKeysInScan + kBins == kSelWarps * kIter, "upper half of list_key + hist hold one chunk per warp");
 constexpr int kSampleChunks = 256;                    // sample = 256 chunks of 32 scores
 constexpr int kSamplePerThread = kSampleChunks * 32 / kSelThreads;   // 16
 
@@ -61,9 +61,9 @@ __device__ __forceinline__ uint32_t order_key(float x) {
 }
 
 struct SelShared {
-    uint32_t hist[kBins];
     uint32_t list_pos[kListCap];      // candidate positions; the entries of one chunk are consecutive and ascending
-    uint32_t list_key[kListCap];      // their order keys (pass 1 stages scores in here first)
+    uint32_t list_key[kListCap];      // their order keys; pass 1 stages scores in the upper half and in hist (next member)
+    uint32_t hist[kBins];
     double red_a[kSelWarps];
     double red_b[kSelWarps];
     uint32_t red_min[kSelWarps];
@@ -322,9 +322,13 @@ __global__ void __launch_bounds__(kSelThreads, 2) gsa_select_kernel(const Select
         // The 512 scores of an iteration arrive by coalesced 16-byte loads (lane l gets scores 4l..4l+3 of
         // each 128) and are turned, through shared memory, so that lane l holds scores 16l..16l+15: a
         // lane's candidates are then consecutive in position order and one warp scan of the counts places
-        // them.  The staging buffer is the warp's part of list_key, which is filled only after this pass.
+        // them.  The staging buffer is the upper half of list_key and the histogram behind it (idle during this
+        // pass); a candidate's score is read back from it for the order key that goes into the list with the
+        // position, as long as the list has not grown into the staging area (entries from kKeysInScan on, rare:
+        // they get their keys after the pass).
         // 16-byte slot q (= position / 4) is kept at q ^ ((q >> 3) & 3): no bank conflicts either way.
-        float4* const tb = reinterpret_cast<float4*>(sh.list_key + wid * kStageFloats);
+        float4* const tb = reinterpret_cast<float4*>(sh.list_key + kKeysInScan + wid * kIter);
+        const float* const tbf = reinterpret_cast<const float*>(tb);
         const int wslot = lane ^ ((lane >> 3) & 3);
         const int rsw = (lane >> 1) & 3;
         // loads run one iteration ahead
@@ -408,6 +412,22 @@ __global__ void __launch_bounds__(kSelThreads, 2) gsa_select_kernel(const Select
                             sh.list_pos[pos++] = ib + (uint32_t)(__ffs(f) - 1);
                             f &= f - 1;
                         }
+                        __syncwarp();
+                        // the chunk's order keys, all lanes side by side: the scores are still in the staging area
+                        // (slot q = offset / 4, swizzled) or, for the row's partial last chunk, in global memory
+                        for (uint32_t q = lane; q < iter_total && base + q < (uint32_t)kKeysInScan; q += 32) {
+                            const uint32_t at = sh.list_pos[base + q];
+                            float x;
+                            if (rs0 + kIter <= n) {
+                                const uint32_t off = at - (uint32_t)rs0, slot = off >> 2;
+                                x = tbf[4 * (slot ^ ((slot >> 3) & 3)) + (off & 3)];
+                            } else {
+                                x = __ldg(grow + at);
+                            }
+                            const uint32_t key = order_key(x);
+                            sh.list_key[base + q] = key;
+                            kmax = max(kmax, key);
+                        }
                     } else {
                         w_over = true;
                     }
@@ -423,17 +443,13 @@ __global__ void __launch_bounds__(kSelThreads, 2) gsa_select_kernel(const Select
     }
     if (lane == 0) { sh.red_a[wid] = s1; sh.red_b[wid] = s2; }
     __syncthreads();
-    // keys of the listed candidates (the staging buffers inside list_key are free now)
-    int m = 0;                                  // candidates found (all of them listed unless overflow)
-    if (listed) {
-        m = (int)min(sh.list_total, (uint32_t)kListCap);
-        if (sh.overflow == 0u)
-            for (int q = tid; q < m; q += kSelThreads) {
-                const uint32_t key = order_key(__ldg(grow + sh.list_pos[q]));
-                sh.list_key[q] = key;
-                kmax = max(kmax, key);
-            }
-    }
+    const int m = listed ? (int)min(sh.list_total, (uint32_t)kListCap) : 0;   // candidates found (all listed unless overflow)
+    if (listed && sh.overflow == 0u)                                          // entries that pass 1 left without a key
+        for (int q = kKeysInScan + tid; q < m; q += kSelThreads) {
+            const uint32_t key = order_key(__ldg(grow + sh.list_pos[q]));
+            sh.list_key[q] = key;
+            kmax = max(kmax, key);
+        }
     if (tid == 0) {
         double ta = 0.0, tb = 0.0;
         for (int i = 0; i < kSelWarps; ++i) { ta += sh.red_a[i]; tb += sh.red_b[i]; }
