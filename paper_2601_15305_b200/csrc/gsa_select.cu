@@ -76,6 +76,7 @@ struct SelShared {
     uint32_t list_total;              // entries handed out so far
     uint32_t found_bin;
     uint32_t found_above;
+    uint32_t found_count;             // entries in the found bin
     uint32_t overflow;
     uint32_t bc_want;                 // pass 0: sample rank of the candidate threshold
     int32_t bc_k;                     // the row's k_t (Eq. 8), computed by one thread
@@ -125,7 +126,7 @@ __device__ __forceinline__ void find_bin(SelShared& sh, uint32_t want, uint32_t&
         uint32_t acc = above_mine;
         for (int j = kBinsPerThread - 1; j >= 0; --j) {
             const uint32_t c = sh.hist[tid * kBinsPerThread + j];
-            if (want <= acc + c) { sh.found_bin = tid * kBinsPerThread + j; sh.found_above = acc; break; }
+            if (want <= acc + c) { sh.found_bin = tid * kBinsPerThread + j; sh.found_above = acc; sh.found_count = c; break; }
             acc += c;
         }
     }
@@ -143,10 +144,10 @@ __device__ __forceinline__ int shift_for(uint32_t span) {
 }
 
 // Radix rounds over `count` keys fetched by `key_of(i)`: narrows [lo, hi] onto the want-th largest
-// key.  Returns T = that key, need_eq = how many keys == T belong to the top set.
+// key.  Returns T = that key, need_eq = how many keys == T belong to the top set, eq_total = how many there are.
 template <class KeyOf>
 __device__ __forceinline__ void radix_rounds(SelShared& sh, int count, KeyOf key_of, uint32_t lo, uint32_t hi,
-                                             uint32_t want, uint32_t& T, uint32_t& need_eq) {
+                                             uint32_t want, uint32_t& T, uint32_t& need_eq, uint32_t& eq_total) {
     const int tid = threadIdx.x;
     while (true) {
         const uint32_t span = hi - lo;          // inclusive range has span + 1 keys
@@ -168,6 +169,7 @@ __device__ __forceinline__ void radix_rounds(SelShared& sh, int count, KeyOf key
     }
     T = lo;
     need_eq = want;
+    eq_total = sh.found_count;               // the last round's bins are single keys: all keys equal to T
 }
 
 // block-wide exclusive scan of one value per thread; returns the exclusive prefix and the total.
@@ -472,10 +474,10 @@ __global__ void __launch_bounds__(kSelThreads, 2) gsa_select_kernel(const Select
         return;
     }
 
-    uint32_t T, need_eq;
+    uint32_t T, need_eq, eq_total;
     if (short_row) {
         // ---- the row is the list: radix rounds, then one ordered compaction -------------------
-        radix_rounds(sh, n, [&](int i) { return sh.list_key[i]; }, kmin, kmax, (uint32_t)k, T, need_eq);
+        radix_rounds(sh, n, [&](int i) { return sh.list_key[i]; }, kmin, kmax, (uint32_t)k, T, need_eq, eq_total);
         uint32_t gt = 0, eq = 0;
         const int j0 = tid * kListPerThread;
 #pragma unroll
@@ -506,7 +508,38 @@ __global__ void __launch_bounds__(kSelThreads, 2) gsa_select_kernel(const Select
 
     if (!overflow && m >= k) {
         // ---- exact threshold among the candidates ------------------------------------------------
-        radix_rounds(sh, m, [&](int i) { return sh.list_key[i]; }, kmin, kmax, (uint32_t)k, T, need_eq);
+        radix_rounds(sh, m, [&](int i) { return sh.list_key[i]; }, kmin, kmax, (uint32_t)k, T, need_eq, eq_total);
+
+        if (eq_total == need_eq && n <= kBins * 32) {
+            // ---- emission through a bitmap of the row's positions (every key equal to T is taken, so the
+            // selected candidates are simply those with key >= T): the candidates mark their positions, all
+            // threads side by side, then every thread turns its stretch of the bitmap into ascending positions.
+            // The bitmap is the histogram's space: one bit per position, rows of up to 32 * kBins scores.
+            const int words = (n + 31) >> 5;
+            for (int i = tid; i < words; i += kSelThreads) sh.hist[i] = 0u;
+            __syncthreads();
+            for (int q = tid; q < m; q += kSelThreads)
+                if (sh.list_key[q] >= T) {
+                    const uint32_t pos = sh.list_pos[q];
+                    atomicOr(&sh.hist[pos >> 5], 1u << (pos & 31u));
+                }
+            __syncthreads();
+            const int wpt = (words + kSelThreads - 1) / kSelThreads;            // 1 .. 8
+            const int w_lo = min(words, tid * wpt), w_hi = min(words, w_lo + wpt);
+            uint32_t mine = 0;
+            for (int w = w_lo; w < w_hi; ++w) mine += __popc(sh.hist[w]);
+            uint32_t total;
+            uint32_t at = block_excl_scan(sh, mine, 0, total);
+            for (int w = w_lo; w < w_hi; ++w) {
+                uint32_t bits = sh.hist[w];
+                while (bits) {
+                    out_idx[at++] = (int32_t)((w << 5) + __ffs(bits) - 1);
+                    bits &= bits - 1u;
+                }
+            }
+            for (int i = k + tid; i < a.k_max; i += kSelThreads) out_idx[i] = -1;
+            return;
+        }
 
         // ---- emission in position order: thread t owns table chunks t*cpt .. t*cpt + cpt - 1 -------
         const int cpt = (ntab + kSelThreads - 1) / kSelThreads;             // 1 .. 4
@@ -542,7 +575,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) gsa_select_kernel(const Select
         // ---- fallback: radix rounds over the whole row, then ordered emission ----------------
         if (tid == 0 && a.fallback_rows) atomicAdd(a.fallback_rows, 1);
         radix_rounds(sh, n, [&](int i) { return order_key(__ldg(grow + i)); }, 0u, 0xFFFFFFFFu,
-                     (uint32_t)k, T, need_eq);
+                     (uint32_t)k, T, need_eq, eq_total);
         const int seg = ((n + kSelWarps - 1) / kSelWarps + 31) & ~31;
         const int seg_lo = min(n, wid * seg), seg_hi = min(n, seg_lo + seg);
         uint32_t cg = 0, ce = 0;
