@@ -9,13 +9,15 @@
 //      are dealt to the 16 warps round-robin, so each warp sees an even sample of the row.  Loads are
 //      fully coalesced float4s, one chunk ahead, turned through shared memory so that a lane holds 16
 //      consecutive scores; every score goes into fp64 sum and sum of squares; the position of a score
-//      that reaches tau (one float compare) goes into the candidate list in shared memory, with its order key: a warp scan
-//      of the lanes' counts orders the chunk's candidates, one shared-memory atomic claims their space,
-//      and a table remembers where each chunk's entries start and how many there are.   -> Var, k_t
-//   2  on chip: radix rounds over the candidates' keys give
-//      the exact threshold key T of the k_t-th largest score and how many keys equal to T are taken;
-//      the chunks are then walked in position order (counts per thread, one block scan, emission) to
-//      write S_t ascending.
+//      that reaches tau (one float compare) goes into the candidate list in shared memory, with its
+//      order key: a warp scan of the lanes' counts orders the chunk's candidates, one shared-memory
+//      atomic claims their space, and a table remembers where each chunk's entries start and how many
+//      there are.   -> Var, k_t
+//   2  on chip: radix rounds over the candidates' keys give the exact threshold key T of the k_t-th
+//      largest score and how many keys equal to T are taken.  S_t is then written ascending: if every
+//      key equal to T is taken (no tie is cut) and the row has at most 131072 scores, the selected
+//      candidates mark their positions in a bitmap and the threads turn stretches of it into positions;
+//      otherwise the chunks are walked in position order (counts per thread, one block scan, emission).
 // Equal keys go to the lower position, so the output is unique.  If the list overflows or comes out
 // shorter than k_t (the sample misjudged the row: huge ties, scores sorted by position, ...) the CTA
 // falls back to radix rounds over the whole row in global memory: slower, same result.  Rows of more
