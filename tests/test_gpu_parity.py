@@ -239,6 +239,23 @@ def test_topk_long_rows_that_defeat_the_sample():
         _select_and_compare(cfg, sc.cuda(), k_mode=k_mode, v_bar=v_bar)
 
 
+def test_topk_long_rows_with_a_tie_cut_and_rows_beyond_the_bitmap():
+    """The two cases in which a long row's set is written by walking the candidate table instead of through
+    the position bitmap: the budget cuts a group of equal scores (scores quantised to 4096 levels: a few equal
+    scores per level, the candidate list does not overflow), and a row of more than 131072 visible scores."""
+    cfg = CONFIGS["l8k"].with_(name="tiecut", B=1, Lq=5, Lk=30011, k_base=900, k_min=100, k_max=3000)
+    st = U.row_stride(cfg)
+    g = torch.Generator().manual_seed(10)
+    sc = torch.floor(torch.rand((1, cfg.Lq, st), generator=g) * 4096.0) / 4096.0
+    for k_mode, v_bar in ((2, 1.0), (0, 0.08)):
+        _select_and_compare(cfg, sc.cuda(), k_mode=k_mode, v_bar=v_bar)
+    cfg = CONFIGS["l8k"].with_(name="beyond_bitmap", B=1, Lq=3, Lk=131072 + 4099, k_base=1500, k_min=100, k_max=4096)
+    st = U.row_stride(cfg)
+    sc = torch.rand((1, cfg.Lq, st), generator=g) ** 3
+    for k_mode, v_bar in ((2, 1.0), (0, 0.05)):
+        _select_and_compare(cfg, sc.cuda(), k_mode=k_mode, v_bar=v_bar)
+
+
 def test_topk_row_lengths_around_the_chunk_and_list_boundaries():
     """Visible lengths n just below / at / above the short-row limit (8192) and multiples of the 512-score
     chunk, and rows whose last chunk holds a single score."""
